@@ -1,0 +1,215 @@
+/*
+ * ddd.h - C ABI of the Dynamic Depth Decoding draft-tree library (single GPU, sm_100a).
+ *
+ * One call of ddd_draft runs Algorithm 1 of the paper ("Dynamic Depth Decoding") for a
+ * batch of B independent sequences, entirely on the device and without a host
+ * synchronisation between draft-model calls:
+ *
+ *   for pass d = 1 .. n:                              (Algorithm 1, the for-loop; n = max_depth)
+ *     logits  = s * h W^T + bias   for the beam rows  (Section 1: the draft model ends in the
+ *                                                      target's LM head; "Run draft model on beam")
+ *     logprob = log-softmax(logits), clamped to <= 0  (Section 2: draft output goes through logsoftmax)
+ *     per-row top-k tokens; candidate score = parent's logprobsum + logprob
+ *                                                     (Section 1: sum of logprobs ranks token sequences;
+ *                                                      Algorithm 1: logprobsum update)
+ *     new beam = top-k of the k*k candidates          (Algorithm 1: "produce the new beam")
+ *     H = log sum_i exp(logprobsum[i])                (Eq. 1)
+ *     stop if d == n, or if step d is in S and H < x  (Algorithm 1: "if step in S", "if H < x: break")
+ *     h_child = RMSNorm(h_parent + E[token])          (stands in for the trained draft head of Section 1)
+ *   rerank: keep the m best tree nodes by logprobsum, emit tokens, parents, depths, position
+ *   ids and a bit-packed ancestor mask                (Section 1: the tree goes to the target model
+ *                                                      with an adjusted attention mask)
+ *
+ * Conventions
+ *   - Every pointer argument says whether it is a HOST or a DEVICE pointer.  The library
+ *     never allocates device memory: weights, workspace, inputs and outputs are allocated by
+ *     the caller and only borrowed.  W, E, bias, plant_next and the workspace must stay valid
+ *     and unchanged until ddd_destroy.
+ *   - All functions return DDD_OK (0) or a negative DDD_ERR_* code; nothing throws, traps or
+ *     aborts.  ddd_strerror maps a code to a static string.
+ *   - ddd_draft only enqueues work on the given stream.  Outputs are valid once that stream
+ *     has been synchronised.  Problems found on the device (a bounded wait that ran out)
+ *     are reported through ddd_output.status, never as a fault.
+ *   - One draft in flight per handle; a handle is not thread-safe.
+ */
+#ifndef DDD_H_
+#define DDD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ddd_handle ddd_handle; /* opaque */
+
+enum {
+  DDD_OK = 0,
+  DDD_ERR_INVALID_ARG = -1, /* NULL pointer, size out of range, unknown enum value          */
+  DDD_ERR_ALIGNMENT = -2,   /* a pointer is not aligned as documented                        */
+  DDD_ERR_WORKSPACE = -3,   /* workspace smaller than ddd_workspace_bytes()                  */
+  DDD_ERR_CUDA = -4,        /* a CUDA runtime / driver call failed                           */
+  DDD_ERR_TIMEOUT = -5,     /* device status: a bounded wait inside a kernel ran out         */
+  DDD_ERR_UNSUPPORTED = -6  /* valid request this build cannot serve (e.g. kernel / dtype)   */
+};
+
+enum { DDD_DTYPE_FP32 = 0, DDD_DTYPE_BF16 = 1 };
+
+/* Which LM-head kernel runs a pass.  AUTO picks TCGEN05 for bf16 and SIMT for fp32. */
+enum { DDD_LM_HEAD_AUTO = 0, DDD_LM_HEAD_SIMT = 1, DDD_LM_HEAD_TCGEN05 = 2 };
+
+/* How a draft is enqueued.  GRAPH replays one captured CUDA graph per draft. */
+enum { DDD_LAUNCH_STREAM = 0, DDD_LAUNCH_GRAPH = 1 };
+
+#define DDD_MAX_K 32          /* beam width limit                                  */
+#define DDD_MAX_DEPTH 32      /* check_mask has one bit per step                   */
+#define DDD_MAX_TOTAL 1023    /* m limit (output rows = m + 1)                     */
+#define DDD_MAX_ROWS 256      /* B * k limit                                       */
+#define DDD_MAX_NODES 24576   /* 1 + k + (n-1) k^2 limit                           */
+#define DDD_CHECK_EVERY_STEP 0xFFFFFFFFu
+
+/* Parameters of Algorithm 1 (n, w, S, x) and the tensor shapes. */
+typedef struct {
+  int32_t batch;        /* B >= 1 independent sequences                                           */
+  int32_t hidden;       /* Hd, multiple of 8 (multiple of 64 for the TCGEN05 kernel)              */
+  int32_t vocab;        /* V > k                                                                  */
+  int32_t k;            /* beam width w, 1..DDD_MAX_K                                             */
+  int32_t max_depth;    /* n: maximum number of draft-model calls, 1..DDD_MAX_DEPTH               */
+  int32_t total_tokens; /* m: draft nodes kept by the rerank (the root is extra), 1..DDD_MAX_TOTAL */
+  int32_t dtype;        /* DDD_DTYPE_*: storage type of W, E and every hidden state               */
+  float threshold;      /* x: after a checked step, drafting continues iff H >= x                 */
+  uint32_t check_mask;  /* S: bit (s-1) set <=> the heuristic is checked after step s             */
+  float logit_scale;    /* s in logits = s * h W^T + bias                                         */
+  float rms_eps;        /* eps inside the square root of RMSNorm                                  */
+  float plant_delta;    /* see plant_next in ddd_create                                           */
+  int32_t device;       /* CUDA device ordinal                                                    */
+  int32_t lm_head_kernel; /* DDD_LM_HEAD_*                                                        */
+  int32_t launch_mode;    /* DDD_LAUNCH_*                                                         */
+} ddd_config;
+
+/*
+ * Results of one draft.  With T = total_tokens + 1 and W32 = ceil(T / 32), per sequence b:
+ *   n_out[b]        rows used: 1 + min(m, N), N = k + (D-1) k^2 nodes generated in D passes
+ *   stop_depth[b]   D: number of draft-model calls made (1..n)
+ *   row 0 is the root; rows 1..n_out-1 are the kept nodes in ascending generation order,
+ *   so a parent always precedes its children.  Rows >= n_out hold token = parent = depth =
+ *   position = -1, cum = 0 and an all-zero mask row.
+ *   token[b][i], parent[b][i] (row index of the parent, -1 for the root), depth[b][i],
+ *   position[b][i] = root_pos[b] + depth, cum[b][i] = summed logprob of the path (root 0)
+ *   mask[b][i][w]   bit j of row i (word j / 32, bit j % 32, LSB first) is set iff row j is
+ *                   row i itself or one of its ancestors
+ *   H_trace[b][d-1] Eq. 1 evaluated after pass d, for every pass that ran (others untouched)
+ *   status[0]       DDD_OK, or the first DDD_ERR_* a kernel recorded during this draft
+ * Every field is required and is a DEVICE pointer for ddd_draft, a HOST pointer for
+ * ddd_draft_host.  Layout is dense row-major in the index order shown.
+ */
+typedef struct {
+  int32_t *n_out;      /* [B]         */
+  int32_t *stop_depth; /* [B]         */
+  int32_t *token;      /* [B][T]      */
+  int32_t *parent;     /* [B][T]      */
+  int32_t *depth;      /* [B][T]      */
+  int32_t *position;   /* [B][T]      */
+  float *cum;          /* [B][T]      */
+  uint32_t *mask;      /* [B][T][W32] */
+  float *H_trace;      /* [B][n]      */
+  int32_t *status;     /* [1]         */
+} ddd_output;
+
+/*
+ * Optional record of the search itself (all DEVICE pointers, each may be NULL), used to
+ * replay the decisions in another implementation.  Nn = 1 + k + (n-1) k^2 node slots per
+ * sequence; node 0 is the root, pass 1 creates nodes 1..k, pass d >= 2 creates node
+ * 1 + k + (d-2) k^2 + p k + c for the c-th best token of beam row p.
+ *   node_id[b][i]      tree node shown in output row i (-1 beyond n_out)
+ *   tree_token[b][j], tree_parent[b][j] (node id), tree_cum[b][j]   for generated nodes
+ *   beam_sel[b][d-1][i] candidate index p k + c that became beam entry i after pass d
+ *   row_lse[b][d-1][p]  logsumexp of the logits of beam row p in pass d
+ */
+typedef struct {
+  int32_t *node_id;     /* [B][T]    */
+  int32_t *tree_token;  /* [B][Nn]   */
+  int32_t *tree_parent; /* [B][Nn]   */
+  float *tree_cum;      /* [B][Nn]   */
+  int32_t *beam_sel;    /* [B][n][k] */
+  float *row_lse;       /* [B][n][k] */
+} ddd_trace;
+
+/*
+ * Bytes of device workspace a handle with this configuration needs (0 if the configuration
+ * is invalid).  Pure host function; makes no CUDA call.
+ */
+size_t ddd_workspace_bytes(const ddd_config *cfg /* HOST */);
+
+/*
+ * Creates a handle.  (Algorithm 1's Require line: n, w, S, x arrive in cfg.)
+ *   W           DEVICE [V][Hd], row-major (hidden contiguous), cfg->dtype, 16-byte aligned:
+ *               the LM head, logits[r][v] = s * sum_j W[v][j] h[r][j] + bias[v]
+ *   E           DEVICE [V][Hd], same layout and type: embedding rows for the draft step
+ *   bias        DEVICE [V] fp32 or NULL
+ *   plant_next  DEVICE [V] int32 or NULL.  If given and c = plant_next[t] >= 0 for the last
+ *               token t of a beam row, that row's logit of column c is replaced by
+ *               (maximum of the row's other logits) + plant_delta before the log-softmax.
+ *   workspace   DEVICE, 256-byte aligned, at least ddd_workspace_bytes(cfg) bytes; its
+ *               contents are owned by the handle until ddd_destroy.
+ * Makes cfg->device current, creates no stream, allocates no device memory.
+ * Errors: INVALID_ARG, ALIGNMENT, WORKSPACE, UNSUPPORTED, CUDA.  *out is NULL on error.
+ */
+int ddd_create(const ddd_config *cfg /* HOST */, const void *W, const void *E, const float *bias,
+               const int32_t *plant_next, void *workspace, size_t workspace_bytes,
+               ddd_handle **out /* HOST */);
+
+/*
+ * Enqueues one draft of the whole batch on `cuda_stream` (a cudaStream_t; NULL = the legacy
+ * default stream) and returns without waiting.  (Algorithm 1, all lines; then the rerank.)
+ *   root_hidden DEVICE [B][Hd], cfg->dtype, 16-byte aligned: hidden state fed to pass 1
+ *   root_token  DEVICE [B] int32: last accepted token of each sequence (tree node 0)
+ *   root_pos    DEVICE [B] int32: its position id
+ *   out         HOST struct of DEVICE pointers, all required
+ *   trace       HOST struct of DEVICE pointers or NULL
+ * In DDD_LAUNCH_GRAPH mode the captured graph is reused while these pointers and the stream
+ * stay the same, and re-captured when they change.
+ * Errors: INVALID_ARG, ALIGNMENT, CUDA.
+ */
+int ddd_draft(ddd_handle *h, const void *root_hidden, const int32_t *root_token,
+              const int32_t *root_pos, const ddd_output *out, const ddd_trace *trace,
+              void *cuda_stream);
+
+/*
+ * Same draft with HOST buffers: copies the inputs to staging space inside the workspace,
+ * runs the draft, copies every ddd_output field back and synchronises the stream before
+ * returning.  All pointers (inputs and the fields of `out`) are HOST pointers; pinned
+ * memory makes the copies asynchronous but is not required.  Returns the device status
+ * (e.g. DDD_ERR_TIMEOUT) if the draft itself reported one.
+ */
+int ddd_draft_host(ddd_handle *h, const void *root_hidden, const int32_t *root_token,
+                   const int32_t *root_pos, const ddd_output *out, void *cuda_stream);
+
+/*
+ * Enqueues ONE LM-head pass (logits, online max / sum-exp and per-row top-k partials, the
+ * kernel that streams W) over all B*k beam rows currently held by the handle, for timing
+ * and profiling that kernel alone.  It reads the hidden rows left by the last draft and
+ * writes only workspace scratch.  (Section 1: the draft model call; Algorithm 1 "Run draft
+ * model on beam".)  Errors: INVALID_ARG, CUDA.
+ */
+int ddd_lm_head_pass(ddd_handle *h, void *cuda_stream);
+
+/*
+ * Number of kernels one ddd_draft enqueues (they all launch even if the gate stops early;
+ * kernels of skipped passes exit at once), and the number of thread blocks the LM-head
+ * kernel uses.  Pure host queries; negative on a NULL handle.
+ */
+int ddd_launches_per_draft(const ddd_handle *h);
+int ddd_lm_head_blocks(const ddd_handle *h);
+
+/* Releases host state (and the captured graph).  Device memory stays with the caller. */
+int ddd_destroy(ddd_handle *h);
+
+/* Static description of a DDD_* code. */
+const char *ddd_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DDD_H_ */
