@@ -1,0 +1,166 @@
+// Shared device-side definitions of the draft-tree kernels: the parameter block, the
+// order-preserving 64-bit (score, index) keys used by every top-k, and the per-row
+// tile update (online max / sum-exp and running top-k) used by both LM-head kernels.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "ddd.h"
+
+namespace ddd {
+
+constexpr int kMaxLmCtas = 512;   // upper bound on LM-head thread blocks (sizes the partial buffers)
+constexpr int kTile = 128;        // vocab rows handled per epilogue tile
+constexpr unsigned kFullMask = 0xFFFFFFFFu;
+
+// Everything a kernel needs that does not change between drafts.
+struct Params {
+  int B, Hd, V, k, n, m, dtype;
+  int R;              // B * k beam rows
+  int Nn;             // node slots per sequence: 1 + k + (n-1) k^2
+  int T, W32;         // output rows per sequence (m + 1) and mask words per row
+  float x;            // threshold
+  uint32_t check_mask;
+  float s, eps, plant_delta;
+  const void* W;
+  const void* E;
+  const float* bias;
+  const int* plant_next;
+  void* hbuf[2];                  // [R][Hd] hidden rows, double-buffered by pass parity
+  unsigned long long* part_key;   // [lm_ctas][R][k] per-block top-k keys, descending, 0 = empty
+  float2* part_ms;                // [lm_ctas][R]    per-block (max, sum exp(z - max))
+  int lm_ctas;
+  int* tree_token;                // [B][Nn]
+  int* tree_parent;               // [B][Nn] node id
+  float* tree_cum;                // [B][Nn]
+  int* beam_node;                 // [B][k]
+  int* beam_tok;                  // [B][k]
+  float* beam_cum;                // [B][k]
+  int* row_plant;                 // [R] planted column of each beam row, -1 = none
+  int* active;                    // [B]
+  int* n_active;                  // [1]
+  int* stop_depth;                // [B]
+  int* root_pos;                  // [B] copy of the caller's root positions
+  int* dev_status;                // [1] first error recorded by a kernel during this draft
+};
+
+// Per-draft pointers (caller-owned device memory).
+struct DraftIO {
+  ddd_output out;
+  ddd_trace trace;
+};
+
+// ---------------------------------------------------------------------------- keys
+// Maps a float to a uint32 whose unsigned order equals the float order (-inf lowest).
+__device__ __forceinline__ uint32_t float_to_ordered(float f) {
+  uint32_t u = __float_as_uint(f + 0.0f);   // +0.0f turns -0 into +0
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float ordered_to_float(uint32_t o) {
+  uint32_t u = (o & 0x80000000u) ? (o & 0x7FFFFFFFu) : ~o;
+  return __uint_as_float(u);
+}
+// Larger key <=> larger value, ties broken towards the smaller index.  Key 0 means "empty".
+__device__ __forceinline__ unsigned long long make_key(float v, uint32_t idx) {
+  return ((unsigned long long)float_to_ordered(v) << 32) | (unsigned long long)(0xFFFFFFFFu - idx);
+}
+__device__ __forceinline__ float key_value(unsigned long long key) {
+  return ordered_to_float((uint32_t)(key >> 32));
+}
+__device__ __forceinline__ uint32_t key_index(unsigned long long key) {
+  return 0xFFFFFFFFu - (uint32_t)key;
+}
+
+// Maximum of one 64-bit key per lane over the warp (two 32-bit redux steps).
+__device__ __forceinline__ unsigned long long warp_max_key(unsigned long long key) {
+  const uint32_t hi = (uint32_t)(key >> 32);
+  const uint32_t mhi = __reduce_max_sync(kFullMask, hi);
+  const uint32_t lo = (hi == mhi) ? (uint32_t)key : 0u;
+  const uint32_t mlo = __reduce_max_sync(kFullMask, lo);
+  return ((unsigned long long)mhi << 32) | mlo;
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFullMask, v, o);
+  return v;
+}
+
+__device__ __forceinline__ float neg_inf() { return __uint_as_float(0xFF800000u); }
+
+// Is beam row r part of pass d?  Pass 1 has one row per sequence (the root, slot 0).
+__device__ __forceinline__ bool row_live(const Params& p, int r, int d, int force_all) {
+  if (force_all) return true;
+  const int b = r / p.k, i = r - b * p.k;
+  return p.active[b] != 0 && (d > 1 || i == 0);
+}
+
+// ---------------------------------------------------------------------------- per-row tile update
+// One warp folds kTile logits of one beam row (tokens tok0 .. tok0 + kTile - 1, -inf where
+// the column does not exist or is excluded) into that row's running state:
+//   (m, s)    online max and sum exp(z - m), identical in all lanes
+//   list_key  lane j < k holds the j-th best (logit, token) key seen so far, 0 = empty
+__device__ __forceinline__ void row_tile_update(const float* zrow, int tok0, int k, float& m, float& s,
+                                                unsigned long long& list_key) {
+  const int lane = threadIdx.x & 31;
+  const float4 z4 = *reinterpret_cast<const float4*>(zrow + 4 * lane);
+  const float z[4] = {z4.x, z4.y, z4.z, z4.w};
+  const float lm = fmaxf(fmaxf(z[0], z[1]), fmaxf(z[2], z[3]));
+  const float mt = ordered_to_float(__reduce_max_sync(kFullMask, float_to_ordered(lm)));
+  if (mt == neg_inf()) return;   // nothing valid in this tile (uniform across the warp)
+
+  float ls = 0.f;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) ls += __expf(z[i] - mt);
+  const float st = warp_sum(ls);
+  if (mt > m) {
+    s = s * __expf(m - mt) + st;
+    m = mt;
+  } else {
+    s += st * __expf(mt - m);
+  }
+
+  unsigned long long keys[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+    keys[i] = (z[i] == neg_inf()) ? 0ull : make_key(z[i], (uint32_t)(tok0 + 4 * lane + i));
+  // Nothing to do unless some entry beats the current k-th best (0 while the list is not full).
+  const unsigned long long kth = __shfl_sync(kFullMask, list_key, k - 1);
+  const bool beats = keys[0] > kth || keys[1] > kth || keys[2] > kth || keys[3] > kth;
+  if (!__any_sync(kFullMask, beats)) return;
+
+  unsigned long long carry = list_key;
+  unsigned long long best = carry;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) best = keys[i] > best ? keys[i] : best;
+  unsigned long long new_list = 0ull;
+  for (int j = 0; j < k; ++j) {
+    const unsigned long long wk = warp_max_key(best);
+    if (wk == 0ull) break;               // pool exhausted (uniform)
+    if (lane == j) new_list = wk;
+    if (best == wk) {                    // keys are unique (distinct tokens): exactly one owner
+      if (carry == wk) carry = 0ull;
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        if (keys[i] == wk) keys[i] = 0ull;
+      best = carry;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) best = keys[i] > best ? keys[i] : best;
+    }
+  }
+  list_key = new_list;
+}
+
+// ---------------------------------------------------------------------------- launchers (host)
+// Each returns the cudaError_t of its launch / attribute call.
+cudaError_t prepare_simt(const Params& p);
+cudaError_t prepare_tree(const Params& p);
+cudaError_t launch_init(const Params& p, const DraftIO& io, const void* root_hidden, const int* root_token,
+                        const int* root_pos, cudaStream_t st);
+cudaError_t launch_lm_head_simt(const Params& p, int d, int force_all, int ctas, cudaStream_t st);
+cudaError_t launch_select(const Params& p, const DraftIO& io, int d, cudaStream_t st);
+cudaError_t launch_rerank(const Params& p, const DraftIO& io, cudaStream_t st);
+
+}  // namespace ddd

@@ -1,0 +1,448 @@
+// Kernels around the LM head: draft initialisation, the per-pass select / gate / draft
+// step, and the final rerank with the bit-packed tree mask.  One thread block per sequence.
+#include "ddd_common.cuh"
+
+namespace ddd {
+
+namespace {
+
+constexpr int kSelThreads = 1024;
+constexpr int kRerankThreads = 1024;
+
+// ---------------------------------------------------------------------------- init
+// Resets the per-draft state and loads the root: tree node 0, beam slot 0 and hidden row b*k.
+template <typename T>
+__global__ void init_kernel(const Params p, const T* __restrict__ root_hidden,
+                            const int* __restrict__ root_token, const int* __restrict__ root_pos) {
+  const int b = blockIdx.x;
+  T* dst = static_cast<T*>(p.hbuf[0]) + (size_t)b * p.k * p.Hd;
+  const T* src = root_hidden + (size_t)b * p.Hd;
+  for (int j = threadIdx.x; j < p.Hd; j += blockDim.x) dst[j] = src[j];
+  if (threadIdx.x == 0) {
+    const int tok = root_token[b];
+    p.tree_token[(size_t)b * p.Nn] = tok;
+    p.tree_parent[(size_t)b * p.Nn] = -1;
+    p.tree_cum[(size_t)b * p.Nn] = 0.f;
+    p.beam_node[b * p.k] = 0;
+    p.beam_tok[b * p.k] = tok;
+    p.beam_cum[b * p.k] = 0.f;
+    const bool tok_ok = tok >= 0 && tok < p.V;
+    p.row_plant[b * p.k] = (p.plant_next && tok_ok) ? p.plant_next[tok] : -1;
+    p.active[b] = 1;
+    p.stop_depth[b] = 0;
+    p.root_pos[b] = root_pos[b];
+    if (b == 0) {
+      *p.n_active = p.B;
+      *p.dev_status = DDD_OK;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------- select / gate / step
+// Dynamic shared memory: first-entry keys of every LM-head block for each of the k rows.
+__global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Params p, const DraftIO io,
+                                                                       const int d) {
+  const int b = blockIdx.x;
+  if (p.active[b] == 0) return;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  unsigned long long* firsts = reinterpret_cast<unsigned long long*>(smem_raw);   // [k][lm_ctas]
+  __shared__ unsigned long long cand_key[DDD_MAX_K * DDD_MAX_K];
+  __shared__ float cand_val[DDD_MAX_K * DDD_MAX_K];
+  __shared__ int cand_tok[DDD_MAX_K * DDD_MAX_K];
+  __shared__ int sel_flat[DDD_MAX_K];
+  __shared__ int sel_tok[DDD_MAX_K];
+  __shared__ int s_stop;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int k = p.k, nc = p.lm_ctas, R = p.R;
+  const int P = (d == 1) ? 1 : k;                            // beam rows of this sequence in pass d
+  const int base = (d == 1) ? 1 : 1 + k + (d - 2) * k * k;   // node id of candidate (0, 0)
+
+  // ---- phase 1: one warp per beam row merges the per-block partials of the LM-head pass
+  if (warp < P) {
+    const int pr = warp, r = b * k + pr;
+    // log-sum-exp over all blocks (fixed lane-strided order, then a butterfly: deterministic)
+    float M = neg_inf();
+    for (int c = lane; c < nc; c += 32) M = fmaxf(M, p.part_ms[(size_t)c * R + r].x);
+    M = ordered_to_float(__reduce_max_sync(kFullMask, float_to_ordered(M)));
+    float S = 0.f;
+    for (int c = lane; c < nc; c += 32) {
+      const float2 ms = p.part_ms[(size_t)c * R + r];
+      if (ms.y > 0.f) S += ms.y * expf(ms.x - M);
+    }
+    S = warp_sum(S);
+    // planted column: its logit is (max of the others) + delta and it was left out of the partials
+    const int pc = p.row_plant[r];
+    unsigned long long plant_key = 0ull;
+    if (pc >= 0) {
+      const float zc = M + p.plant_delta;
+      const float M2 = fmaxf(M, zc);
+      S = S * expf(M - M2) + expf(zc - M2);
+      M = M2;
+      plant_key = make_key(zc, (uint32_t)pc);
+    }
+    const float lse = M + logf(S);
+
+    // the k blocks with the best first entries are the only ones that can hold a top-k entry
+    unsigned long long* my_first = firsts + (size_t)pr * nc;
+    for (int c = lane; c < nc; c += 32) my_first[c] = p.part_key[((size_t)c * R + r) * k];
+    __syncwarp();
+    unsigned long long prev = ~0ull, cur = 0ull, nxt = 0ull;
+    int my_cta = -1;
+    for (int j = 0; j < k; ++j) {
+      unsigned long long best = 0ull;
+      int best_c = -1;
+      for (int c = lane; c < nc; c += 32) {
+        const unsigned long long key = my_first[c];
+        if (key < prev && key > best) { best = key; best_c = c; }
+      }
+      const unsigned long long wk = warp_max_key(best);
+      if (wk == 0ull) break;
+      const unsigned owner = __ballot_sync(kFullMask, best == wk);
+      const int win_c = __shfl_sync(kFullMask, best_c, __ffs(owner) - 1);
+      if (lane == j) { cur = wk; my_cta = win_c; }
+      prev = wk;
+    }
+    // k-way merge of those blocks' sorted lists; lane j walks the list of block my_cta
+    const unsigned long long* my_list =
+        my_cta >= 0 ? p.part_key + ((size_t)my_cta * R + r) * k : nullptr;
+    int pos = 1;
+    if (my_list && pos < k) nxt = my_list[pos];
+    unsigned long long res = 0ull;
+    for (int j = 0; j < k; ++j) {
+      const unsigned long long wk = warp_max_key(cur);
+      if (wk == 0ull) break;
+      if (lane == j) res = wk;
+      if (cur == wk) {
+        cur = nxt;
+        ++pos;
+        nxt = (my_list && pos < k) ? my_list[pos] : 0ull;
+      }
+    }
+    // insert the planted candidate into the sorted result
+    if (pc >= 0) {
+      const int ins = __popc(__ballot_sync(kFullMask, lane < k && res > plant_key));
+      const unsigned long long up = __shfl_up_sync(kFullMask, res, 1);
+      if (lane == ins) res = plant_key;
+      else if (lane > ins) res = up;
+    }
+    if (lane < k) {
+      const float lp = (res != 0ull) ? fminf(key_value(res) - lse, 0.f) : neg_inf();
+      const int tok = (res != 0ull) ? (int)key_index(res) : -1;
+      const float cand = p.beam_cum[b * k + pr] + lp;
+      const int flat = pr * k + lane;
+      const size_t node = (size_t)b * p.Nn + base + flat;
+      p.tree_token[node] = tok;
+      p.tree_parent[node] = p.beam_node[b * k + pr];
+      p.tree_cum[node] = cand;
+      cand_key[flat] = (res != 0ull) ? make_key(cand, (uint32_t)flat) : 0ull;
+      cand_val[flat] = cand;
+      cand_tok[flat] = tok;
+    }
+    if (lane == 0 && io.trace.row_lse) io.trace.row_lse[((size_t)b * p.n + (d - 1)) * k + pr] = lse;
+  }
+  __syncthreads();
+
+  // ---- phase 2: warp 0 picks the new beam, evaluates Eq. 1 and takes the stop decision
+  if (warp == 0) {
+    const int n_cand = P * k;
+    unsigned long long prev = ~0ull, mine = 0ull;
+    for (int j = 0; j < k; ++j) {
+      unsigned long long best = 0ull;
+      for (int c = lane; c < n_cand; c += 32) {
+        const unsigned long long key = cand_key[c];
+        if (key < prev && key > best) best = key;
+      }
+      const unsigned long long wk = warp_max_key(best);
+      if (lane == j) mine = wk;
+      prev = wk;
+    }
+    const bool have = lane < k && mine != 0ull;
+    const int flat = have ? (int)key_index(mine) : 0;
+    const float cum = have ? cand_val[flat] : neg_inf();
+    const float M = __shfl_sync(kFullMask, cum, 0);           // sorted descending: entry 0 is the max
+    const float sum = warp_sum(have ? expf(cum - M) : 0.f);
+    const float H = M + logf(sum);
+    bool stop = (d == p.n);
+    if (!stop && ((p.check_mask >> (d - 1)) & 1u)) stop = H < p.x;
+    if (lane < k) {
+      const int tok = cand_tok[flat];
+      sel_flat[lane] = flat;
+      sel_tok[lane] = tok;
+      p.beam_node[b * k + lane] = base + flat;
+      p.beam_tok[b * k + lane] = tok;
+      p.beam_cum[b * k + lane] = cum;
+      p.row_plant[b * k + lane] = (p.plant_next && tok >= 0 && tok < p.V) ? p.plant_next[tok] : -1;
+      if (io.trace.beam_sel) io.trace.beam_sel[((size_t)b * p.n + (d - 1)) * k + lane] = flat;
+    }
+    if (lane == 0) {
+      io.out.H_trace[(size_t)b * p.n + (d - 1)] = H;
+      s_stop = stop ? 1 : 0;
+      if (stop) {
+        p.stop_depth[b] = d;
+        p.active[b] = 0;
+        atomicSub(p.n_active, 1);
+      }
+    }
+  }
+  __syncthreads();
+  if (s_stop) return;
+
+  // ---- phase 3: synthetic draft step, one warp per new beam row:
+  //      h_child = round( u / sqrt(mean(u^2) + eps) ),  u = h_parent + E[token]
+  if (warp < k) {
+    const int i = warp;
+    const int parent_slot = sel_flat[i] / k;
+    const int tok = sel_tok[i];
+    const size_t src_row = (size_t)(b * k + parent_slot) * p.Hd;
+    const size_t dst_row = (size_t)(b * k + i) * p.Hd;
+    const size_t e_row = (size_t)(tok >= 0 && tok < p.V ? tok : 0) * p.Hd;
+    if (p.dtype == DDD_DTYPE_BF16) {
+      const __nv_bfloat16* hp = static_cast<const __nv_bfloat16*>(p.hbuf[(d - 1) & 1]) + src_row;
+      const __nv_bfloat16* e = static_cast<const __nv_bfloat16*>(p.E) + e_row;
+      __nv_bfloat16* out = static_cast<__nv_bfloat16*>(p.hbuf[d & 1]) + dst_row;
+      float ss = 0.f;
+      for (int j = lane * 8; j < p.Hd; j += 256) {
+        const uint4 a = *reinterpret_cast<const uint4*>(hp + j);
+        const uint4 c = *reinterpret_cast<const uint4*>(e + j);
+        const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, cw[4] = {c.x, c.y, c.z, c.w};
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const float u0 = __uint_as_float(aw[q] << 16) + __uint_as_float(cw[q] << 16);
+          const float u1 = __uint_as_float(aw[q] & 0xFFFF0000u) + __uint_as_float(cw[q] & 0xFFFF0000u);
+          ss = fmaf(u0, u0, ss);
+          ss = fmaf(u1, u1, ss);
+        }
+      }
+      ss = warp_sum(ss);
+      const float inv = 1.0f / sqrtf(ss / (float)p.Hd + p.eps);
+      for (int j = lane * 8; j < p.Hd; j += 256) {
+        const uint4 a = *reinterpret_cast<const uint4*>(hp + j);
+        const uint4 c = *reinterpret_cast<const uint4*>(e + j);
+        const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, cw[4] = {c.x, c.y, c.z, c.w};
+        uint32_t ow[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const float u0 = __uint_as_float(aw[q] << 16) + __uint_as_float(cw[q] << 16);
+          const float u1 = __uint_as_float(aw[q] & 0xFFFF0000u) + __uint_as_float(cw[q] & 0xFFFF0000u);
+          const __nv_bfloat162 y = __floats2bfloat162_rn(u0 * inv, u1 * inv);
+          ow[q] = *reinterpret_cast<const uint32_t*>(&y);
+        }
+        *reinterpret_cast<uint4*>(out + j) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+      }
+    } else {
+      const float* hp = static_cast<const float*>(p.hbuf[(d - 1) & 1]) + src_row;
+      const float* e = static_cast<const float*>(p.E) + e_row;
+      float* out = static_cast<float*>(p.hbuf[d & 1]) + dst_row;
+      float ss = 0.f;
+      for (int j = lane; j < p.Hd; j += 32) {
+        const float u = hp[j] + e[j];
+        ss = fmaf(u, u, ss);
+      }
+      ss = warp_sum(ss);
+      const float inv = 1.0f / sqrtf(ss / (float)p.Hd + p.eps);
+      for (int j = lane; j < p.Hd; j += 32) out[j] = (hp[j] + e[j]) * inv;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------- rerank + mask
+__device__ __forceinline__ int node_depth(int id, int k) {
+  if (id == 0) return 0;
+  if (id <= k) return 1;
+  return 2 + (id - 1 - k) / (k * k);
+}
+
+// Block-wide exclusive prefix sum of one int per thread (kRerankThreads threads).
+__device__ int block_exclusive_scan(int v, int* warp_tot /* [32] shared */, int* total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(kFullMask, inc, o);
+    if (lane >= o) inc += t;
+  }
+  __syncthreads();                 // protect warp_tot from its previous use
+  if (lane == 31) warp_tot[warp] = inc;
+  __syncthreads();
+  int offset = 0, tot = 0;
+  for (int w = 0; w < kRerankThreads / 32; ++w) {
+    const int t = warp_tot[w];
+    if (w < warp) offset += t;
+    tot += t;
+  }
+  *total = tot;
+  return offset + inc - v;
+}
+
+// Dynamic shared memory: ordered cum keys [Nn], selection flags / output rows [Nn].
+__global__ void __launch_bounds__(kRerankThreads) rerank_mask_kernel(const Params p, const DraftIO io) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int b = blockIdx.x, tid = threadIdx.x;
+  const int k = p.k, T = p.T;
+  const int D = p.stop_depth[b];
+  const int N = (D >= 1) ? k + (D - 1) * k * k : 0;     // generated non-root nodes
+  uint32_t* key = reinterpret_cast<uint32_t*>(smem_raw);           // key of node id i+1 at [i]
+  int* slot_of = reinterpret_cast<int*>(key + p.Nn);                // output row of node id, -1 = dropped
+  __shared__ int hist[256];
+  __shared__ int warp_tot[32];
+  __shared__ uint32_t s_prefix;
+  __shared__ int s_remaining;
+  __shared__ int out_parent[DDD_MAX_TOTAL + 1];
+
+  const float* cum = p.tree_cum + (size_t)b * p.Nn;
+  const int* tparent = p.tree_parent + (size_t)b * p.Nn;
+  const int* ttoken = p.tree_token + (size_t)b * p.Nn;
+  for (int i = tid; i < N; i += kRerankThreads) key[i] = float_to_ordered(cum[i + 1]);
+  const int m_eff = min(p.m, N);
+  if (tid == 0) { s_prefix = 0u; s_remaining = m_eff; }
+  __syncthreads();
+
+  // ---- radix select: value of the m_eff-th largest key and how many of its ties to keep
+  uint32_t known_mask = 0u;
+  for (int pass = 3; pass >= 0 && m_eff > 0; --pass) {
+    const int shift = 8 * pass;
+    for (int i = tid; i < 256; i += kRerankThreads) hist[i] = 0;
+    __syncthreads();
+    const uint32_t prefix = s_prefix;
+    for (int i = tid; i < N; i += kRerankThreads) {
+      const uint32_t q = key[i];
+      if ((q & known_mask) == prefix) atomicAdd(&hist[(q >> shift) & 0xFF], 1);
+    }
+    __syncthreads();
+    if (tid == 0) {
+      int remaining = s_remaining, bin = 255;
+      for (; bin > 0; --bin) {
+        if (hist[bin] >= remaining) break;
+        remaining -= hist[bin];
+      }
+      s_prefix = prefix | ((uint32_t)bin << shift);
+      s_remaining = remaining;
+    }
+    known_mask |= 0xFFu << shift;
+    __syncthreads();
+  }
+  const uint32_t thr = s_prefix;
+  const int keep_ties = s_remaining;      // among keys equal to thr, the lowest node ids win
+
+  // ---- selection flags in node-id order; each thread owns a contiguous chunk of ids
+  const int chunk = (N + kRerankThreads - 1) / kRerankThreads;
+  const int lo = min(N, tid * chunk), hi = min(N, lo + chunk);
+  int n_eq = 0;
+  for (int i = lo; i < hi; ++i) n_eq += (key[i] == thr);
+  int tot_unused;
+  int eq_before = block_exclusive_scan(n_eq, warp_tot, &tot_unused);
+  int n_sel = 0;
+  for (int i = lo; i < hi; ++i) {
+    const uint32_t q = key[i];
+    bool sel = false;
+    if (m_eff > 0) {
+      if (q > thr) sel = true;
+      else if (q == thr) sel = (eq_before++ < keep_ties);
+    }
+    slot_of[i + 1] = sel ? 1 : 0;
+    n_sel += sel;
+  }
+  int n_selected;
+  int sel_before = block_exclusive_scan(n_sel, warp_tot, &n_selected);
+  for (int i = lo; i < hi; ++i) {
+    const bool sel = slot_of[i + 1] != 0;
+    slot_of[i + 1] = sel ? 1 + sel_before : -1;
+    sel_before += sel;
+  }
+  if (tid == 0) slot_of[0] = 0;
+  __syncthreads();
+
+  // ---- emit rows: the root, then the kept nodes in ascending node id
+  const int n_out = 1 + n_selected;
+  const size_t ob = (size_t)b * T;
+  for (int id = tid; id <= N; id += kRerankThreads) {
+    const int slot = slot_of[id];
+    if (slot < 0 || slot >= T) continue;
+    const int dep = node_depth(id, k);
+    const int par = (id == 0) ? -1 : slot_of[tparent[id]];
+    out_parent[slot] = par;
+    io.out.token[ob + slot] = ttoken[id];
+    io.out.parent[ob + slot] = par;
+    io.out.depth[ob + slot] = dep;
+    io.out.position[ob + slot] = p.root_pos[b] + dep;
+    io.out.cum[ob + slot] = cum[id];
+    if (io.trace.node_id) io.trace.node_id[ob + slot] = id;
+  }
+  for (int slot = n_out + tid; slot < T; slot += kRerankThreads) {
+    io.out.token[ob + slot] = -1;
+    io.out.parent[ob + slot] = -1;
+    io.out.depth[ob + slot] = -1;
+    io.out.position[ob + slot] = -1;
+    io.out.cum[ob + slot] = 0.f;
+    if (io.trace.node_id) io.trace.node_id[ob + slot] = -1;
+  }
+  if (tid == 0) {
+    io.out.n_out[b] = n_out;
+    io.out.stop_depth[b] = D;
+    if (b == 0) *io.out.status = *p.dev_status;
+  }
+  __syncthreads();
+
+  // ---- ancestor mask: row i has bit j set iff j is i or an ancestor of i
+  for (int slot = tid; slot < T; slot += kRerankThreads) {
+    uint32_t* row = io.out.mask + (ob + slot) * p.W32;
+    for (int w = 0; w < p.W32; ++w) {
+      uint32_t bits = 0u;
+      if (slot < n_out) {
+        int a = slot;
+        for (int guard = 0; a >= 0 && guard <= DDD_MAX_DEPTH; ++guard) {
+          if ((a >> 5) == w) bits |= 1u << (a & 31);
+          a = out_parent[a];
+        }
+      }
+      row[w] = bits;
+    }
+  }
+  // copy the generated tree for replay, if asked for
+  if (io.trace.tree_token) {
+    for (int id = tid; id < p.Nn; id += kRerankThreads) {
+      const bool gen = id <= N;
+      const size_t o = (size_t)b * p.Nn + id;
+      io.trace.tree_token[o] = gen ? ttoken[id] : -1;
+      if (io.trace.tree_parent) io.trace.tree_parent[o] = gen ? tparent[id] : -1;
+      if (io.trace.tree_cum) io.trace.tree_cum[o] = gen ? cum[id] : 0.f;
+    }
+  }
+}
+
+size_t select_smem(const Params& p) { return (size_t)p.k * p.lm_ctas * sizeof(unsigned long long); }
+size_t rerank_smem(const Params& p) { return (size_t)p.Nn * (sizeof(uint32_t) + sizeof(int)); }
+
+}  // namespace
+
+// ---------------------------------------------------------------------------- launchers
+cudaError_t prepare_tree(const Params& p) {
+  cudaError_t e = cudaFuncSetAttribute(select_gate_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)select_smem(p));
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(rerank_mask_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              (int)rerank_smem(p));
+}
+
+cudaError_t launch_init(const Params& p, const DraftIO&, const void* root_hidden, const int* root_token,
+                        const int* root_pos, cudaStream_t st) {
+  if (p.dtype == DDD_DTYPE_FP32)
+    init_kernel<float><<<p.B, 256, 0, st>>>(p, static_cast<const float*>(root_hidden), root_token, root_pos);
+  else
+    init_kernel<__nv_bfloat16><<<p.B, 256, 0, st>>>(p, static_cast<const __nv_bfloat16*>(root_hidden),
+                                                    root_token, root_pos);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_select(const Params& p, const DraftIO& io, int d, cudaStream_t st) {
+  select_gate_step_kernel<<<p.B, kSelThreads, select_smem(p), st>>>(p, io, d);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_rerank(const Params& p, const DraftIO& io, cudaStream_t st) {
+  rerank_mask_kernel<<<p.B, kRerankThreads, rerank_smem(p), st>>>(p, io);
+  return cudaGetLastError();
+}
+
+}  // namespace ddd
