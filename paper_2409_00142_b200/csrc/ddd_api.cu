@@ -1,0 +1,394 @@
+// Host side of the C ABI declared in ddd.h: argument checking, workspace carving, the
+// launch sequence of one draft (optionally replayed from a CUDA graph) and the host-buffer
+// variant.  No device memory is allocated here; the only allocation is a small pinned host
+// bounce buffer used by ddd_draft_host.
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "ddd_common.cuh"
+#include "lm_head_tc.cuh"
+
+using namespace ddd;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
+
+struct Layout {
+  size_t hbuf[2], part_key, part_ms, tree_token, tree_parent, tree_cum, beam_node, beam_tok, beam_cum,
+      row_plant, active, stop_depth, root_pos, n_active, dev_status;
+  // staging for ddd_draft_host: inputs, then the packed output block
+  size_t in_hidden, in_token, in_pos, out_block;
+  size_t o_n_out, o_stop, o_token, o_parent, o_depth, o_position, o_cum, o_mask, o_H, o_status, out_bytes;
+  size_t in_bytes;   // in_hidden .. in_pos are contiguous: one copy
+  size_t total;
+};
+
+int validate(const ddd_config* c) {
+  if (!c) return DDD_ERR_INVALID_ARG;
+  if (c->batch < 1 || c->hidden < 8 || c->vocab < 2) return DDD_ERR_INVALID_ARG;
+  if (c->hidden % 8 != 0) return DDD_ERR_INVALID_ARG;
+  if (c->k < 1 || c->k > DDD_MAX_K || c->vocab <= c->k) return DDD_ERR_INVALID_ARG;
+  if (c->max_depth < 1 || c->max_depth > DDD_MAX_DEPTH) return DDD_ERR_INVALID_ARG;
+  if (c->total_tokens < 1 || c->total_tokens > DDD_MAX_TOTAL) return DDD_ERR_INVALID_ARG;
+  if (c->dtype != DDD_DTYPE_FP32 && c->dtype != DDD_DTYPE_BF16) return DDD_ERR_INVALID_ARG;
+  if ((long long)c->batch * c->k > DDD_MAX_ROWS) return DDD_ERR_INVALID_ARG;
+  const long long nn = 1 + (long long)c->k + (long long)(c->max_depth - 1) * c->k * c->k;
+  if (nn > DDD_MAX_NODES) return DDD_ERR_INVALID_ARG;
+  if (!(c->logit_scale == c->logit_scale) || !(c->threshold == c->threshold)) return DDD_ERR_INVALID_ARG;
+  if (!(c->rms_eps >= 0.f)) return DDD_ERR_INVALID_ARG;
+  if (c->device < 0) return DDD_ERR_INVALID_ARG;
+  if (c->lm_head_kernel < DDD_LM_HEAD_AUTO || c->lm_head_kernel > DDD_LM_HEAD_TCGEN05) return DDD_ERR_INVALID_ARG;
+  if (c->launch_mode != DDD_LAUNCH_STREAM && c->launch_mode != DDD_LAUNCH_GRAPH) return DDD_ERR_INVALID_ARG;
+  if (c->lm_head_kernel == DDD_LM_HEAD_TCGEN05 && (c->dtype != DDD_DTYPE_BF16 || c->hidden % 64 != 0))
+    return DDD_ERR_UNSUPPORTED;
+  return DDD_OK;
+}
+
+Layout make_layout(const ddd_config* c) {
+  Layout L{};
+  const size_t elt = c->dtype == DDD_DTYPE_FP32 ? 4 : 2;
+  const size_t B = c->batch, k = c->k, R = B * k, n = c->max_depth, T = c->total_tokens + 1;
+  const size_t W32 = (T + 31) / 32, Nn = 1 + k + (n - 1) * k * k;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+  L.hbuf[0] = take(R * c->hidden * elt);
+  L.hbuf[1] = take(R * c->hidden * elt);
+  L.part_key = take((size_t)kMaxLmCtas * R * k * 8);
+  L.part_ms = take((size_t)kMaxLmCtas * R * 8);
+  L.tree_token = take(B * Nn * 4);
+  L.tree_parent = take(B * Nn * 4);
+  L.tree_cum = take(B * Nn * 4);
+  L.beam_node = take(R * 4);
+  L.beam_tok = take(R * 4);
+  L.beam_cum = take(R * 4);
+  L.row_plant = take(R * 4);
+  L.active = take(B * 4);
+  L.stop_depth = take(B * 4);
+  L.root_pos = take(B * 4);
+  L.n_active = take(4);
+  L.dev_status = take(4);
+  // host-variant staging: inputs packed back to back (each 16-byte aligned), one output block
+  L.in_hidden = take(0);
+  size_t in = 0;
+  auto in_take = [&](size_t bytes) { size_t o = in; in = (in + bytes + 15) / 16 * 16; return o; };
+  const size_t ih = in_take(B * c->hidden * elt), it = in_take(B * 4), ip = in_take(B * 4);
+  L.in_bytes = in;
+  L.in_token = L.in_hidden + it;
+  L.in_pos = L.in_hidden + ip;
+  (void)ih;
+  take(in);
+  L.out_block = take(0);
+  size_t o = 0;
+  auto o_take = [&](size_t bytes) { size_t r = o; o = (o + bytes + 15) / 16 * 16; return r; };
+  L.o_n_out = o_take(B * 4);
+  L.o_stop = o_take(B * 4);
+  L.o_token = o_take(B * T * 4);
+  L.o_parent = o_take(B * T * 4);
+  L.o_depth = o_take(B * T * 4);
+  L.o_position = o_take(B * T * 4);
+  L.o_cum = o_take(B * T * 4);
+  L.o_mask = o_take(B * T * W32 * 4);
+  L.o_H = o_take(B * n * 4);
+  L.o_status = o_take(4);
+  L.out_bytes = o;
+  take(o);
+  L.total = off;
+  return L;
+}
+
+struct GraphKey {
+  const void* root_hidden;
+  const int32_t* root_token;
+  const int32_t* root_pos;
+  ddd_output out;
+  ddd_trace trace;
+  cudaStream_t stream;
+};
+
+}  // namespace
+
+struct ddd_handle {
+  ddd_config cfg;
+  Params p;
+  Layout L;
+  unsigned char* ws;
+  int sm_count;
+  int lm_kind;     // DDD_LM_HEAD_SIMT or DDD_LM_HEAD_TCGEN05
+  TcPlan tc;
+  // graph cache (one entry)
+  cudaGraphExec_t exec;
+  GraphKey key;
+  bool have_graph;
+  // pinned host bounce buffer for ddd_draft_host
+  unsigned char* bounce;
+  size_t bounce_bytes;
+};
+
+namespace {
+
+cudaError_t launch_lm_head(const ddd_handle* h, int d, int force_all, cudaStream_t st) {
+  if (h->lm_kind == DDD_LM_HEAD_TCGEN05) return launch_lm_head_tc(h->p, h->tc, d, force_all, st);
+  return launch_lm_head_simt(h->p, d, force_all, h->p.lm_ctas, st);
+}
+
+cudaError_t enqueue_draft(const ddd_handle* h, const DraftIO& io, const void* root_hidden,
+                          const int32_t* root_token, const int32_t* root_pos, cudaStream_t st) {
+  cudaError_t e = launch_init(h->p, io, root_hidden, root_token, root_pos, st);
+  for (int d = 1; d <= h->p.n && e == cudaSuccess; ++d) {
+    e = launch_lm_head(h, d, 0, st);
+    if (e == cudaSuccess) e = launch_select(h->p, io, d, st);
+  }
+  if (e == cudaSuccess) e = launch_rerank(h->p, io, st);
+  return e;
+}
+
+bool aligned16(const void* q) { return (reinterpret_cast<uintptr_t>(q) & 15u) == 0; }
+
+}  // namespace
+
+extern "C" {
+
+size_t ddd_workspace_bytes(const ddd_config* cfg) {
+  if (validate(cfg) != DDD_OK) return 0;
+  return make_layout(cfg).total;
+}
+
+int ddd_create(const ddd_config* cfg, const void* W, const void* E, const float* bias,
+               const int32_t* plant_next, void* workspace, size_t workspace_bytes, ddd_handle** out) {
+  if (out) *out = nullptr;
+  if (!out) return DDD_ERR_INVALID_ARG;
+  const int v = validate(cfg);
+  if (v != DDD_OK) return v;
+  if (!W || !E || !workspace) return DDD_ERR_INVALID_ARG;
+  if (!aligned16(W) || !aligned16(E)) return DDD_ERR_ALIGNMENT;
+  if (reinterpret_cast<uintptr_t>(workspace) % kAlign != 0) return DDD_ERR_ALIGNMENT;
+  const Layout L = make_layout(cfg);
+  if (workspace_bytes < L.total) return DDD_ERR_WORKSPACE;
+
+  if (cudaSetDevice(cfg->device) != cudaSuccess) return DDD_ERR_CUDA;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, cfg->device) != cudaSuccess) return DDD_ERR_CUDA;
+
+  ddd_handle* h = new (std::nothrow) ddd_handle();
+  if (!h) return DDD_ERR_CUDA;
+  h->cfg = *cfg;
+  h->L = L;
+  h->ws = static_cast<unsigned char*>(workspace);
+  h->sm_count = prop.multiProcessorCount;
+  h->have_graph = false;
+  h->exec = nullptr;
+  h->bounce = nullptr;
+  h->bounce_bytes = 0;
+
+  Params& p = h->p;
+  p.B = cfg->batch; p.Hd = cfg->hidden; p.V = cfg->vocab; p.k = cfg->k; p.n = cfg->max_depth;
+  p.m = cfg->total_tokens; p.dtype = cfg->dtype;
+  p.R = p.B * p.k;
+  p.Nn = 1 + p.k + (p.n - 1) * p.k * p.k;
+  p.T = p.m + 1;
+  p.W32 = (p.T + 31) / 32;
+  p.x = cfg->threshold; p.check_mask = cfg->check_mask;
+  p.s = cfg->logit_scale; p.eps = cfg->rms_eps; p.plant_delta = cfg->plant_delta;
+  p.W = W; p.E = E; p.bias = bias; p.plant_next = plant_next;
+  unsigned char* ws = h->ws;
+  p.hbuf[0] = ws + L.hbuf[0];
+  p.hbuf[1] = ws + L.hbuf[1];
+  p.part_key = reinterpret_cast<unsigned long long*>(ws + L.part_key);
+  p.part_ms = reinterpret_cast<float2*>(ws + L.part_ms);
+  p.tree_token = reinterpret_cast<int*>(ws + L.tree_token);
+  p.tree_parent = reinterpret_cast<int*>(ws + L.tree_parent);
+  p.tree_cum = reinterpret_cast<float*>(ws + L.tree_cum);
+  p.beam_node = reinterpret_cast<int*>(ws + L.beam_node);
+  p.beam_tok = reinterpret_cast<int*>(ws + L.beam_tok);
+  p.beam_cum = reinterpret_cast<float*>(ws + L.beam_cum);
+  p.row_plant = reinterpret_cast<int*>(ws + L.row_plant);
+  p.active = reinterpret_cast<int*>(ws + L.active);
+  p.stop_depth = reinterpret_cast<int*>(ws + L.stop_depth);
+  p.root_pos = reinterpret_cast<int*>(ws + L.root_pos);
+  p.n_active = reinterpret_cast<int*>(ws + L.n_active);
+  p.dev_status = reinterpret_cast<int*>(ws + L.dev_status);
+
+  int rc = DDD_OK;
+  h->lm_kind = cfg->lm_head_kernel;
+  if (h->lm_kind == DDD_LM_HEAD_AUTO)
+    h->lm_kind = (cfg->dtype == DDD_DTYPE_BF16 && cfg->hidden % 64 == 0) ? DDD_LM_HEAD_TCGEN05 : DDD_LM_HEAD_SIMT;
+  if (h->lm_kind == DDD_LM_HEAD_TCGEN05) {
+    if (prop.major != 10) rc = DDD_ERR_UNSUPPORTED;
+    if (rc == DDD_OK) rc = tc_plan_create(p, h->sm_count, &h->tc);
+    if (rc == DDD_OK) p.lm_ctas = h->tc.ctas;
+  } else {
+    const int n_tiles = (p.V + kTile - 1) / kTile;
+    int ctas = 2 * h->sm_count;
+    if (ctas > n_tiles) ctas = n_tiles;
+    if (ctas > kMaxLmCtas) ctas = kMaxLmCtas;
+    p.lm_ctas = ctas;
+    if (prepare_simt(p) != cudaSuccess) rc = DDD_ERR_CUDA;
+  }
+  if (rc == DDD_OK && prepare_tree(p) != cudaSuccess) rc = DDD_ERR_CUDA;
+  // Zero the workspace once so that rows never written by a draft hold finite values.
+  if (rc == DDD_OK && (cudaMemset(ws, 0, L.total) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess))
+    rc = DDD_ERR_CUDA;
+  if (rc != DDD_OK) {
+    cudaGetLastError();
+    delete h;
+    return rc;
+  }
+  *out = h;
+  return DDD_OK;
+}
+
+int ddd_draft(ddd_handle* h, const void* root_hidden, const int32_t* root_token, const int32_t* root_pos,
+              const ddd_output* out, const ddd_trace* trace, void* cuda_stream) {
+  if (!h || !root_hidden || !root_token || !root_pos || !out) return DDD_ERR_INVALID_ARG;
+  if (!out->n_out || !out->stop_depth || !out->token || !out->parent || !out->depth || !out->position ||
+      !out->cum || !out->mask || !out->H_trace || !out->status)
+    return DDD_ERR_INVALID_ARG;
+  if (!aligned16(root_hidden)) return DDD_ERR_ALIGNMENT;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  DraftIO io;
+  io.out = *out;
+  if (trace) io.trace = *trace; else std::memset(&io.trace, 0, sizeof io.trace);
+
+  if (h->cfg.launch_mode == DDD_LAUNCH_GRAPH && st != nullptr) {
+    GraphKey key;
+    std::memset(&key, 0, sizeof key);
+    key.root_hidden = root_hidden; key.root_token = root_token; key.root_pos = root_pos;
+    key.out = io.out; key.trace = io.trace; key.stream = st;
+    if (!h->have_graph || std::memcmp(&key, &h->key, sizeof key) != 0) {
+      if (h->exec) { cudaGraphExecDestroy(h->exec); h->exec = nullptr; }
+      h->have_graph = false;
+      if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+        cudaGetLastError();
+        return DDD_ERR_CUDA;
+      }
+      const cudaError_t e = enqueue_draft(h, io, root_hidden, root_token, root_pos, st);
+      cudaGraph_t graph = nullptr;
+      const cudaError_t e2 = cudaStreamEndCapture(st, &graph);
+      if (e != cudaSuccess || e2 != cudaSuccess || !graph) {
+        if (graph) cudaGraphDestroy(graph);
+        cudaGetLastError();
+        return DDD_ERR_CUDA;
+      }
+      const cudaError_t e3 = cudaGraphInstantiate(&h->exec, graph, 0);
+      cudaGraphDestroy(graph);
+      if (e3 != cudaSuccess) { cudaGetLastError(); h->exec = nullptr; return DDD_ERR_CUDA; }
+      h->key = key;
+      h->have_graph = true;
+    }
+    if (cudaGraphLaunch(h->exec, st) != cudaSuccess) { cudaGetLastError(); return DDD_ERR_CUDA; }
+    return DDD_OK;
+  }
+  if (enqueue_draft(h, io, root_hidden, root_token, root_pos, st) != cudaSuccess) {
+    cudaGetLastError();
+    return DDD_ERR_CUDA;
+  }
+  return DDD_OK;
+}
+
+int ddd_draft_host(ddd_handle* h, const void* root_hidden, const int32_t* root_token, const int32_t* root_pos,
+                   const ddd_output* out, void* cuda_stream) {
+  if (!h || !root_hidden || !root_token || !root_pos || !out) return DDD_ERR_INVALID_ARG;
+  if (!out->n_out || !out->stop_depth || !out->token || !out->parent || !out->depth || !out->position ||
+      !out->cum || !out->mask || !out->H_trace || !out->status)
+    return DDD_ERR_INVALID_ARG;
+  const Layout& L = h->L;
+  const Params& p = h->p;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const size_t need = (L.in_bytes > L.out_bytes ? L.in_bytes : L.out_bytes);
+  if (!h->bounce) {
+    if (cudaMallocHost(reinterpret_cast<void**>(&h->bounce), need) != cudaSuccess) {
+      cudaGetLastError();
+      return DDD_ERR_CUDA;
+    }
+    h->bounce_bytes = need;
+  }
+  const size_t elt = p.dtype == DDD_DTYPE_FP32 ? 4 : 2;
+  const size_t B = p.B, T = p.T;
+  // pack the inputs into pinned memory: one host-to-device copy
+  std::memcpy(h->bounce, root_hidden, B * p.Hd * elt);
+  std::memcpy(h->bounce + (L.in_token - L.in_hidden), root_token, B * 4);
+  std::memcpy(h->bounce + (L.in_pos - L.in_hidden), root_pos, B * 4);
+  if (cudaMemcpyAsync(h->ws + L.in_hidden, h->bounce, L.in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+    cudaGetLastError();
+    return DDD_ERR_CUDA;
+  }
+  unsigned char* ob = h->ws + L.out_block;
+  ddd_output dev;
+  dev.n_out = reinterpret_cast<int32_t*>(ob + L.o_n_out);
+  dev.stop_depth = reinterpret_cast<int32_t*>(ob + L.o_stop);
+  dev.token = reinterpret_cast<int32_t*>(ob + L.o_token);
+  dev.parent = reinterpret_cast<int32_t*>(ob + L.o_parent);
+  dev.depth = reinterpret_cast<int32_t*>(ob + L.o_depth);
+  dev.position = reinterpret_cast<int32_t*>(ob + L.o_position);
+  dev.cum = reinterpret_cast<float*>(ob + L.o_cum);
+  dev.mask = reinterpret_cast<uint32_t*>(ob + L.o_mask);
+  dev.H_trace = reinterpret_cast<float*>(ob + L.o_H);
+  dev.status = reinterpret_cast<int32_t*>(ob + L.o_status);
+  const int rc = ddd_draft(h, h->ws + L.in_hidden, reinterpret_cast<const int32_t*>(h->ws + L.in_token),
+                           reinterpret_cast<const int32_t*>(h->ws + L.in_pos), &dev, nullptr, cuda_stream);
+  if (rc != DDD_OK) return rc;
+  // one device-to-host copy of the packed results, then scatter to the caller's arrays
+  if (cudaMemcpyAsync(h->bounce, ob, L.out_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess) {
+    cudaGetLastError();
+    return DDD_ERR_CUDA;
+  }
+  const unsigned char* hb = h->bounce;
+  std::memcpy(out->n_out, hb + L.o_n_out, B * 4);
+  std::memcpy(out->stop_depth, hb + L.o_stop, B * 4);
+  std::memcpy(out->token, hb + L.o_token, B * T * 4);
+  std::memcpy(out->parent, hb + L.o_parent, B * T * 4);
+  std::memcpy(out->depth, hb + L.o_depth, B * T * 4);
+  std::memcpy(out->position, hb + L.o_position, B * T * 4);
+  std::memcpy(out->cum, hb + L.o_cum, B * T * 4);
+  std::memcpy(out->mask, hb + L.o_mask, B * T * p.W32 * 4);
+  std::memcpy(out->H_trace, hb + L.o_H, B * p.n * 4);
+  std::memcpy(out->status, hb + L.o_status, 4);
+  return out->status[0];
+}
+
+int ddd_lm_head_pass(ddd_handle* h, void* cuda_stream) {
+  if (!h) return DDD_ERR_INVALID_ARG;
+  // Pass index 2 selects the hidden buffer written by the first draft step; all rows are forced live.
+  if (launch_lm_head(h, 2, 1, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) {
+    cudaGetLastError();
+    return DDD_ERR_CUDA;
+  }
+  return DDD_OK;
+}
+
+int ddd_launches_per_draft(const ddd_handle* h) {
+  if (!h) return DDD_ERR_INVALID_ARG;
+  return 2 + 2 * h->p.n;   // init, (LM head + select) per pass, rerank
+}
+
+int ddd_lm_head_blocks(const ddd_handle* h) {
+  if (!h) return DDD_ERR_INVALID_ARG;
+  return h->p.lm_ctas;
+}
+
+int ddd_destroy(ddd_handle* h) {
+  if (!h) return DDD_ERR_INVALID_ARG;
+  if (h->exec) cudaGraphExecDestroy(h->exec);
+  if (h->bounce) cudaFreeHost(h->bounce);
+  delete h;
+  return DDD_OK;
+}
+
+const char* ddd_strerror(int code) {
+  switch (code) {
+    case DDD_OK: return "ok";
+    case DDD_ERR_INVALID_ARG: return "invalid argument";
+    case DDD_ERR_ALIGNMENT: return "pointer not aligned as required";
+    case DDD_ERR_WORKSPACE: return "workspace too small";
+    case DDD_ERR_CUDA: return "CUDA call failed";
+    case DDD_ERR_TIMEOUT: return "a bounded wait inside a kernel ran out";
+    case DDD_ERR_UNSUPPORTED: return "not supported by this build or device";
+    default: return "unknown error code";
+  }
+}
+
+}  // extern "C"

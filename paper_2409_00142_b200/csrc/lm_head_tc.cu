@@ -1,0 +1,454 @@
+// LM-head pass on the sm_100a tensor cores.
+//
+// logits[v][r] = sum_j W[v][j] h[r][j] is computed "swap-AB": the 128 vocab rows of a W
+// tile are the M operand, the (few) beam rows are the N operand, so one tcgen05.mma of
+// M = 128, N = 16..256 keeps every vocab row in its own tensor-memory lane and every beam
+// row in its own column.  The pass is bound by streaming W from HBM once; everything else
+// hides under that stream:
+//   warp 0     TMA producer: W boxes of 32 vocab rows x 64 hidden elements (128-byte
+//              swizzle) plus the matching slice of h, into a ring of shared-memory stages
+//   warp 1     issues tcgen05.mma into one of two tensor-memory accumulators
+//   warps 2-5  epilogue: tcgen05.ld the finished accumulator, apply scale and bias, fold the
+//              tile into each beam row's online max / sum-exp and running top-k
+// Each thread block owns a contiguous range of vocab rows (a multiple of 32) and publishes
+// one partial (max, sum-exp, top-k list) per beam row; logits never reach global memory.
+// Every wait is bounded: when one runs out the block records DDD_ERR_TIMEOUT, drains what
+// it has in flight, frees its tensor memory and returns.
+#include "lm_head_tc.cuh"
+
+namespace ddd {
+
+namespace {
+
+constexpr int kTcThreads = 192;
+constexpr int kBlockM = 128;            // vocab rows per MMA tile
+constexpr int kBlockK = 64;             // hidden elements per stage: one 128-byte swizzle row
+constexpr int kUmmaK = 16;              // K of one tcgen05.mma with 16-bit operands
+constexpr int kUnitRows = 32;           // vocab rows per TMA box of W
+constexpr int kUnitBytes = kUnitRows * kBlockK * 2;   // 4096
+constexpr int kABytes = kBlockM * kBlockK * 2;        // 16384
+constexpr int kChunkCols = 16;          // accumulator columns (beam rows) per epilogue chunk
+constexpr int kSmemLimit = 232448;      // 227 KB opt-in limit per block
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+
+struct SmemPlan {
+  int a, b, zt, key, ms, plant, live, bars, tmem_ptr, abort_flag, total;
+};
+
+__host__ __device__ inline SmemPlan smem_plan(int stages, int n_pad, int R, int k) {
+  SmemPlan s;
+  int off = 0;
+  s.a = off; off += stages * kABytes;
+  s.b = off; off += stages * n_pad * kBlockK * 2;
+  s.zt = off; off += kChunkCols * kTile * 4;
+  s.key = off; off += R * k * 8;
+  s.ms = off; off += R * 8;
+  s.plant = off; off += R * 4;
+  s.live = off; off += R * 4;
+  off = (off + 7) / 8 * 8;
+  s.bars = off; off += (2 * stages + 5) * 8;
+  s.tmem_ptr = off; off += 4;
+  s.abort_flag = off; off += 4;
+  s.total = off;
+  return s;
+}
+
+// ---------------------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ unsigned long long global_timer() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false if the wait ran out of time or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                          bool heed_abort = true) {
+  unsigned long long t0 = 0;
+  for (uint32_t it = 0;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 1023u) == 1023u) {
+      if (heed_abort && *abort_flag) return false;
+      const unsigned long long now = global_timer();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > kWaitLimitNs) {
+        atomicCAS(status, DDD_OK, DDD_ERR_TIMEOUT);
+        *abort_flag = 1;
+        return false;
+      }
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y,
+                                                 unsigned long long policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%3, %4}], [%2], %5;"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "l"(policy)
+      : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, unsigned long long a_desc, unsigned long long b_desc,
+                                            uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
+      "}\n"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tc_load_16cols(uint32_t taddr, float (&v)[16]) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void epilogue_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+// Barrier over the 128 epilogue threads that also ANDs a flag, so that all four warps take
+// the same decision after a bounded wait.
+__device__ __forceinline__ bool epilogue_all(bool ok) {
+  uint32_t r;
+  asm volatile(
+      "{\n"
+      ".reg .pred p, q;\n"
+      "setp.ne.b32 p, %1, 0;\n"
+      "bar.red.and.pred q, 1, 128, p;\n"
+      "selp.u32 %0, 1, 0, q;\n"
+      "}\n"
+      : "=r"(r)
+      : "r"(ok ? 1u : 0u)
+      : "memory");
+  return r != 0;
+}
+
+// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes (64 bf16) wide
+// and 128-byte swizzled: 8-row groups are 1024 bytes apart (stride byte offset); the leading
+// byte offset is not used by swizzled K-major layouts.  Bits: [0,14) address >> 4,
+// [16,30) LBO >> 4, [32,46) SBO >> 4, [46,48) version 1, [61,64) layout 2 = SWIZZLE_128B.
+__device__ __forceinline__ unsigned long long make_smem_desc(uint32_t addr) {
+  return (unsigned long long)((addr & 0x3FFFFu) >> 4) | (1ull << 16) | ((unsigned long long)(1024 >> 4) << 32) |
+         (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor for kind::f16: D = f32 (bits [4,6) = 1), A = B = bf16 (bits [7,10)
+// and [10,13) = 1), both K-major (bits 15, 16 = 0), N >> 3 at [17,23), M >> 4 at [24,29).
+__device__ __forceinline__ uint32_t make_instr_desc(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kBlockM >> 4) << 24);
+}
+
+// ---------------------------------------------------------------------------- kernel
+__global__ void __launch_bounds__(kTcThreads, 1)
+lm_head_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_w,
+                  const __grid_constant__ CUtensorMap map_h, const int d, const int force_all,
+                  const int n_pad, const int stages, const int tmem_cols) {
+  if (!force_all && *p.n_active == 0) return;
+
+  extern __shared__ unsigned char smem_dyn[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>(
+      (reinterpret_cast<uintptr_t>(smem_dyn) + 1023u) & ~static_cast<uintptr_t>(1023u));
+  const SmemPlan sp = smem_plan(stages, n_pad, p.R, p.k);
+  float* zt = reinterpret_cast<float*>(smem + sp.zt);
+  unsigned long long* st_key = reinterpret_cast<unsigned long long*>(smem + sp.key);
+  float2* st_ms = reinterpret_cast<float2*>(smem + sp.ms);
+  int* s_plant = reinterpret_cast<int*>(smem + sp.plant);
+  int* s_live = reinterpret_cast<int*>(smem + sp.live);
+  unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + sp.bars);
+  uint32_t* tmem_ptr = reinterpret_cast<uint32_t*>(smem + sp.tmem_ptr);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + sp.abort_flag);
+
+  const uint32_t a_base = smem_u32(smem + sp.a), b_base = smem_u32(smem + sp.b);
+  const uint32_t b_bytes = (uint32_t)n_pad * kBlockK * 2;
+  const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8u * stages;
+  const uint32_t bar_tfull = bar_empty + 8u * stages, bar_tempty = bar_tfull + 16u;
+  const uint32_t bar_spare = bar_tempty + 16u;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  // this block's contiguous range of 32-row units
+  const int n_units = (p.V + kUnitRows - 1) / kUnitRows;
+  const int base_units = n_units / (int)gridDim.x, rem_units = n_units % (int)gridDim.x;
+  const int bid = blockIdx.x;
+  const int my_units = base_units + (bid < rem_units ? 1 : 0);
+  const int unit0 = bid * base_units + (bid < rem_units ? bid : rem_units);
+  const int n_tiles = (my_units + 3) / 4;
+  const int num_kb = p.Hd / kBlockK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(bar_full + 8u * s, 1);
+      mbar_init(bar_empty + 8u * s, 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(bar_tfull + 8u * a, 1);
+      mbar_init(bar_tempty + 8u * a, 4);     // one arrival per epilogue warp
+    }
+    mbar_init(bar_spare, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {   // tensor-memory allocation is a warp-wide operation
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(tmem_ptr)), "r"((uint32_t)tmem_cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  // per-row flags and running state
+  for (int r = threadIdx.x; r < p.R; r += kTcThreads) {
+    s_plant[r] = p.row_plant[r];
+    s_live[r] = row_live(p, r, d, force_all) ? 1 : 0;
+    st_ms[r] = make_float2(neg_inf(), 0.f);
+  }
+  for (int i = threadIdx.x; i < p.R * p.k; i += kTcThreads) st_key[i] = 0ull;
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_ptr;
+
+  if (warp == 0) {
+    // ======================================================================= TMA producer
+    if (lane == 0) {
+      unsigned long long evict_first;
+      asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(evict_first));
+      int stage = 0, issued = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int t = 0; t < n_tiles && ok; ++t) {
+        const int units = min(4, my_units - 4 * t);
+        const int row0 = (unit0 + 4 * t) * kUnitRows;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(bar_empty + 8u * stage, phase ^ 1u, abort_flag, p.dev_status)) { ok = false; break; }
+          const uint32_t full = bar_full + 8u * stage;
+          mbar_expect_tx(full, (uint32_t)units * kUnitBytes + b_bytes);
+          const uint32_t a_dst = a_base + (uint32_t)stage * kABytes;
+          for (int u = 0; u < units; ++u)
+            tma_load_2d_hint(a_dst + (uint32_t)u * kUnitBytes, &map_w, full, kb * kBlockK, row0 + u * kUnitRows,
+                             evict_first);
+          tma_load_2d(b_base + (uint32_t)stage * b_bytes, &map_h, full, kb * kBlockK, 0);
+          ++issued;
+          if (++stage == stages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {
+        // gave up: wait (bounded) until every copy already issued has landed
+        for (int s = 0; s < stages; ++s) {
+          const int fills = (issued + stages - 1 - s) / stages;
+          if (fills > 0)
+            mbar_wait(bar_full + 8u * s, (uint32_t)((fills - 1) & 1), abort_flag, p.dev_status, false);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ======================================================================= MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc = make_instr_desc(n_pad);
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int t = 0; t < n_tiles && ok; ++t) {
+        const int acc = t & 1;
+        const uint32_t acc_phase = (uint32_t)(t >> 1) & 1u;
+        if (!mbar_wait(bar_tempty + 8u * acc, acc_phase ^ 1u, abort_flag, p.dev_status)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * n_pad);
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(bar_full + 8u * stage, phase, abort_flag, p.dev_status)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t a_addr = a_base + (uint32_t)stage * kABytes;
+          const uint32_t b_addr = b_base + (uint32_t)stage * b_bytes;
+#pragma unroll
+          for (int k4 = 0; k4 < kBlockK / kUmmaK; ++k4) {
+            tc_mma_bf16(d_tmem, make_smem_desc(a_addr + k4 * kUmmaK * 2), make_smem_desc(b_addr + k4 * kUmmaK * 2),
+                        idesc, (kb | k4) != 0 ? 1u : 0u);
+          }
+          tc_commit(bar_empty + 8u * stage);     // frees the stage once these MMAs have read it
+          if (++stage == stages) { stage = 0; phase ^= 1u; }
+        }
+        if (ok) tc_commit(bar_tfull + 8u * acc);   // accumulator complete
+      }
+      if (!ok) {
+        // make sure no MMA is still running before tensor memory is released
+        tc_commit(bar_spare);
+        mbar_wait(bar_spare, 0u, abort_flag, p.dev_status, false);
+      }
+    }
+  } else {
+    // ======================================================================= epilogue
+    const int quarter = warp & 3;            // tensor-memory lanes this warp may read
+    const int ew = warp - 2;                 // owner of beam rows r with r % 4 == ew
+    const int n_chunks = (p.R + kChunkCols - 1) / kChunkCols;
+    bool ok = true;
+    for (int t = 0; t < n_tiles && ok; ++t) {
+      const int acc = t & 1;
+      const uint32_t acc_phase = (uint32_t)(t >> 1) & 1u;
+      const int rows = min(4, my_units - 4 * t) * kUnitRows;
+      const int row0 = (unit0 + 4 * t) * kUnitRows;
+      // The four warps must leave this wait together (they share named barrier 1 below).
+      ok = epilogue_all(mbar_wait(bar_tfull + 8u * acc, acc_phase, abort_flag, p.dev_status, false));
+      if (!ok) break;
+      tc_fence_after();
+      const int vrow = quarter * 32 + lane;
+      const int v = row0 + vrow;
+      const bool v_ok = vrow < rows && v < p.V;
+      const float bias = (v_ok && p.bias) ? p.bias[v] : 0.f;
+      for (int ch = 0; ch < n_chunks; ++ch) {
+        const int c0 = ch * kChunkCols;
+        float accv[16];
+        tc_load_16cols(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * n_pad + c0), accv);
+        if (ch == n_chunks - 1) {
+          // accumulator fully read by this warp: hand it back to the MMA warp
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_tempty + 8u * acc);
+        }
+#pragma unroll
+        for (int c = 0; c < kChunkCols; ++c) {
+          const int r = c0 + c;
+          float z = neg_inf();
+          if (v_ok && r < p.R && s_plant[r] != v) z = fmaf(accv[c], p.s, bias);
+          zt[c * kTile + vrow] = z;
+        }
+        epilogue_barrier();
+        for (int rr = ew; rr < kChunkCols; rr += 4) {
+          const int r = c0 + rr;
+          if (r >= p.R || !s_live[r]) continue;
+          float2 ms = st_ms[r];
+          unsigned long long key = lane < p.k ? st_key[r * p.k + lane] : 0ull;
+          row_tile_update(zt + rr * kTile, row0, p.k, ms.x, ms.y, key);
+          if (lane < p.k) st_key[r * p.k + lane] = key;
+          if (lane == 0) st_ms[r] = ms;
+        }
+        epilogue_barrier();
+      }
+    }
+    // publish this block's partial results (each row by its owning warp)
+    if (ok) {
+      for (int r = ew; r < p.R; r += 4) {
+        if (!s_live[r]) continue;
+        const size_t slot = (size_t)bid * p.R + r;
+        if (lane < p.k) p.part_key[slot * p.k + lane] = st_key[r * p.k + lane];
+        if (lane == 0) p.part_ms[slot] = st_ms[r];
+      }
+    }
+  }
+
+  // ---- teardown: everyone meets, then the allocating warp frees tensor memory
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (warp == 1) {
+    __syncwarp();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)tmem_cols)
+                 : "memory");
+  }
+}
+
+// ---------------------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn) return fn;
+  void* ptr = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess || !ptr)
+    return nullptr;
+  fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  return fn;
+}
+
+// 2-D bf16 tensor [rows][cols] (cols contiguous), box box_rows x 64 columns, 128-byte swizzle,
+// out-of-range elements read as zero.
+bool encode_2d(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {cols * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)kBlockK, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+int tc_plan_create(const Params& p, int sm_count, TcPlan* plan) {
+  if (p.dtype != DDD_DTYPE_BF16 || p.Hd % kBlockK != 0) return DDD_ERR_UNSUPPORTED;
+  const int n_pad = (p.R + 15) / 16 * 16;
+  if (n_pad > 256) return DDD_ERR_UNSUPPORTED;
+  int cols = 32;
+  while (cols < 2 * n_pad) cols *= 2;
+  if (cols > 512) return DDD_ERR_UNSUPPORTED;
+  const int n_units = (p.V + kUnitRows - 1) / kUnitRows;
+  int ctas = sm_count < n_units ? sm_count : n_units;
+  if (ctas > kMaxLmCtas) ctas = kMaxLmCtas;
+  int stages = 0;
+  for (int s = 16; s >= 2; --s) {
+    if (smem_plan(s, n_pad, p.R, p.k).total + 1024 <= kSmemLimit) { stages = s; break; }
+  }
+  if (stages == 0) return DDD_ERR_UNSUPPORTED;
+  plan->ctas = ctas;
+  plan->n_pad = n_pad;
+  plan->stages = stages;
+  plan->tmem_cols = cols;
+  plan->smem = (size_t)smem_plan(stages, n_pad, p.R, p.k).total + 1024;
+  if (!encode_2d(&plan->map_w, p.W, (uint64_t)p.V, (uint64_t)p.Hd, kUnitRows)) return DDD_ERR_CUDA;
+  for (int i = 0; i < 2; ++i)
+    if (!encode_2d(&plan->map_h[i], p.hbuf[i], (uint64_t)p.R, (uint64_t)p.Hd, (uint32_t)n_pad)) return DDD_ERR_CUDA;
+  if (cudaFuncSetAttribute(lm_head_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan->smem) !=
+      cudaSuccess)
+    return DDD_ERR_CUDA;
+  return DDD_OK;
+}
+
+cudaError_t launch_lm_head_tc(const Params& p, const TcPlan& plan, int d, int force_all, cudaStream_t st) {
+  lm_head_tc_kernel<<<plan.ctas, kTcThreads, plan.smem, st>>>(p, plan.map_w, plan.map_h[(d - 1) & 1], d, force_all,
+                                                              plan.n_pad, plan.stages, plan.tmem_cols);
+  return cudaGetLastError();
+}
+
+}  // namespace ddd
