@@ -168,8 +168,10 @@ int ddd_create(const ddd_config *cfg /* HOST */, const void *W, const void *E, c
  *   root_pos    DEVICE [B] int32: its position id
  *   out         HOST struct of DEVICE pointers, all required
  *   trace       HOST struct of DEVICE pointers or NULL
- * In DDD_LAUNCH_GRAPH mode the captured graph is reused while these pointers and the stream
- * stay the same, and re-captured when they change.
+ * In DDD_LAUNCH_GRAPH mode everything after the first kernel is replayed from a captured CUDA
+ * graph, which is reused while the out / trace pointers and the stream stay the same and is
+ * re-captured when they change (the root_* pointers may change freely).  Graph mode needs a
+ * non-default stream; with NULL the kernels are enqueued one by one.
  * Errors: INVALID_ARG, ALIGNMENT, CUDA.
  */
 int ddd_draft(ddd_handle *h, const void *root_hidden, const int32_t *root_token,

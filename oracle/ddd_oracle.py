@@ -257,10 +257,19 @@ def first_node_of_pass(d: int, k: int) -> int:
     return 1 if d == 1 else 1 + k + (d - 2) * k * k
 
 
-def _margin_note(scores: np.ndarray, k: int, tol: float) -> Optional[str]:
+def _margin_note(scores: np.ndarray, k: int, tol: float, ordered: bool = True) -> Optional[str]:
+    """Describes a near-tie that makes more than one answer acceptable, or None.
+
+    For an ordered top-k any two neighbours among the best k+1 scores closer than tol may
+    legally swap; for an unordered selection only the k-th / (k+1)-th boundary matters.
+    """
     s = np.sort(np.asarray(scores, dtype=np.float64))[::-1]
     if len(s) > k and s[k - 1] - s[k] < tol:
         return f"k-th and (k+1)-th differ by {s[k - 1] - s[k]:.3e}"
+    if ordered:
+        gaps = -np.diff(s[:k])
+        if len(gaps) and gaps.min() < tol:
+            return f"two of the best k differ by {gaps.min():.3e}"
     return None
 
 
@@ -410,7 +419,7 @@ def draft(cfg, weights: Dict, root_hidden, root_token, root_pos,
             chosen = ids if not r.violations else rerank(cum, m)
         else:
             chosen = rerank(cum, m)
-        note = _margin_note(cum, min(m, N), tol)
+        note = _margin_note(cum, min(m, N), tol, ordered=False)
         if note:
             r.ambiguities.append(f"rerank: {note}")
         node_id = np.concatenate([[0], chosen]).astype(np.int64)

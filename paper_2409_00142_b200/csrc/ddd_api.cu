@@ -100,9 +100,6 @@ Layout make_layout(const ddd_config* c) {
 }
 
 struct GraphKey {
-  const void* root_hidden;
-  const int32_t* root_token;
-  const int32_t* root_pos;
   ddd_output out;
   ddd_trace trace;
   cudaStream_t stream;
@@ -134,9 +131,10 @@ cudaError_t launch_lm_head(const ddd_handle* h, int d, int force_all, cudaStream
   return launch_lm_head_simt(h->p, d, force_all, h->p.lm_ctas, st);
 }
 
-cudaError_t enqueue_draft(const ddd_handle* h, const DraftIO& io, const void* root_hidden,
-                          const int32_t* root_token, const int32_t* root_pos, cudaStream_t st) {
-  cudaError_t e = launch_init(h->p, io, root_hidden, root_token, root_pos, st);
+// Everything after the init kernel: it depends on the output pointers only, so a captured
+// graph of it can be replayed for any root.
+cudaError_t enqueue_passes(const ddd_handle* h, const DraftIO& io, cudaStream_t st) {
+  cudaError_t e = cudaSuccess;
   for (int d = 1; d <= h->p.n && e == cudaSuccess; ++d) {
     e = launch_lm_head(h, d, 0, st);
     if (e == cudaSuccess) e = launch_select(h->p, io, d, st);
@@ -255,7 +253,6 @@ int ddd_draft(ddd_handle* h, const void* root_hidden, const int32_t* root_token,
   if (h->cfg.launch_mode == DDD_LAUNCH_GRAPH && st != nullptr) {
     GraphKey key;
     std::memset(&key, 0, sizeof key);
-    key.root_hidden = root_hidden; key.root_token = root_token; key.root_pos = root_pos;
     key.out = io.out; key.trace = io.trace; key.stream = st;
     if (!h->have_graph || std::memcmp(&key, &h->key, sizeof key) != 0) {
       if (h->exec) { cudaGraphExecDestroy(h->exec); h->exec = nullptr; }
@@ -264,7 +261,7 @@ int ddd_draft(ddd_handle* h, const void* root_hidden, const int32_t* root_token,
         cudaGetLastError();
         return DDD_ERR_CUDA;
       }
-      const cudaError_t e = enqueue_draft(h, io, root_hidden, root_token, root_pos, st);
+      const cudaError_t e = enqueue_passes(h, io, st);
       cudaGraph_t graph = nullptr;
       const cudaError_t e2 = cudaStreamEndCapture(st, &graph);
       if (e != cudaSuccess || e2 != cudaSuccess || !graph) {
@@ -278,10 +275,15 @@ int ddd_draft(ddd_handle* h, const void* root_hidden, const int32_t* root_token,
       h->key = key;
       h->have_graph = true;
     }
-    if (cudaGraphLaunch(h->exec, st) != cudaSuccess) { cudaGetLastError(); return DDD_ERR_CUDA; }
+    if (launch_init(h->p, io, root_hidden, root_token, root_pos, st) != cudaSuccess ||
+        cudaGraphLaunch(h->exec, st) != cudaSuccess) {
+      cudaGetLastError();
+      return DDD_ERR_CUDA;
+    }
     return DDD_OK;
   }
-  if (enqueue_draft(h, io, root_hidden, root_token, root_pos, st) != cudaSuccess) {
+  if (launch_init(h->p, io, root_hidden, root_token, root_pos, st) != cudaSuccess ||
+      enqueue_passes(h, io, st) != cudaSuccess) {
     cudaGetLastError();
     return DDD_ERR_CUDA;
   }

@@ -1,0 +1,190 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle on the same seeded
+inputs.  Small cases are compared element by element with both LM-head kernels; full-size
+configurations run in the launch configuration the benchmark times (tensor-core kernel,
+CUDA graph)."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import ddd_synth as S
+import paper_2409_00142_b200 as P
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+NEG = -1e30
+
+_weights_cache = {}
+
+
+def weights_for(cfg):
+    key = (cfg.seed, cfg.hidden, cfg.vocab, cfg.dtype, cfg.sigma_w, cfg.bias_kind, cfg.plant_frac)
+    if key not in _weights_cache:
+        if len(_weights_cache) > 2:
+            _weights_cache.clear()
+        _weights_cache[key] = S.make_weights(cfg)
+    return _weights_cache[key]
+
+
+def engine_for(cfg, kernel, mode=P.DDD_LAUNCH_STREAM):
+    return P.DraftEngine(cfg, weights_for(cfg), lm_head_kernel=kernel, launch_mode=mode)
+
+
+SIMT, TC = P.DDD_LM_HEAD_SIMT, P.DDD_LM_HEAD_TCGEN05
+
+
+# ----------------------------------------------------------------------------- tiny (fp32)
+@pytest.mark.parametrize("threshold", [-2.0, -8.0, NEG])
+def test_tiny_fp32(threshold):
+    cfg = S.CONFIGS["tiny"].replace(threshold=threshold)
+    eng = engine_for(cfg, P.DDD_LM_HEAD_AUTO)
+    for i in range(4):
+        roots = S.make_roots(cfg, i)
+        g = parity.run_gpu(eng, roots)
+        parity.compare_with_oracle(cfg, weights_for(cfg), roots, g)
+    assert parity.strict_equal_when_unambiguous(cfg, weights_for(cfg), roots, g) >= 0
+    eng.close()
+
+
+def test_uniform_logits_closed_form_on_gpu():
+    # W = 0: every logprob is -ln V, ties resolve to the lowest token / candidate index,
+    # H_d = ln k - d ln V exactly as the closed form says.
+    cfg = S.CONFIGS["tiny"].replace(threshold=NEG)
+    w = dict(weights_for(cfg))
+    w["W"] = torch.zeros_like(w["W"])
+    eng = P.DraftEngine(cfg, w)
+    roots = S.make_roots(cfg, 0)
+    g = parity.run_gpu(eng, roots)
+    k, V = cfg.k, cfg.vocab
+    assert int(g["stop_depth"][0]) == cfg.max_depth
+    for d in range(1, cfg.max_depth + 1):
+        assert abs(g["H_trace"][0, d - 1] - (math.log(k) - d * math.log(V))) < 1e-4
+        assert g["beam_sel"][0, d - 1].tolist() == list(range(k))
+    assert g["tree_token"][0, 1:k + 1].tolist() == list(range(k))
+    parity.compare_with_oracle(cfg, w, roots, g, strict=True)
+    eng.close()
+
+
+# ----------------------------------------------------------------------------- scaled-down shapes
+def small_cases():
+    c = S.CONFIGS
+    return {
+        # several 128-row tiles per block plus a ragged tail (vocab not a multiple of 32)
+        "7b": S.scaled_down(c["llama2_7b"], 512, 8200 - 12, threshold=-4.0),
+        "13b_plant": S.scaled_down(c["vicuna_13b"], 640, 6000, threshold=-2.0, plant_frac=0.3),
+        "70b_batch": S.scaled_down(c["llama2_70b_b16"], 512, 4096 + 40, threshold=-3.0),
+        "128k_zipf": S.scaled_down(c["llama3_8b_128k"], 256, 20000 + 8, threshold=-3.0),
+        "full_depth": S.scaled_down(c["llama2_7b"], 256, 3000, threshold=NEG),
+    }
+
+
+@pytest.mark.parametrize("kernel", [SIMT, TC], ids=["simt", "tcgen05"])
+@pytest.mark.parametrize("case", list(small_cases()))
+def test_small_shapes_match_oracle(case, kernel):
+    cfg = small_cases()[case]
+    eng = engine_for(cfg, kernel)
+    depths = []
+    for i in range(3):
+        roots = S.make_roots(cfg, i)
+        g = parity.run_gpu(eng, roots)
+        parity.compare_with_oracle(cfg, weights_for(cfg), roots, g)
+        depths += g["stop_depth"].tolist()
+    if case == "70b_batch":
+        assert len(set(depths)) > 1, "batched sequences should stop at different depths"
+    if case == "13b_plant":
+        assert max(depths) > 2, "planted tokens should keep some drafts going"
+    eng.close()
+
+
+def test_strict_oracle_agrees_when_no_near_ties():
+    cfg = small_cases()["7b"]
+    eng = engine_for(cfg, TC)
+    checked = 0
+    for i in range(3):
+        roots = S.make_roots(cfg, 10 + i)
+        g = parity.run_gpu(eng, roots)
+        checked += parity.strict_equal_when_unambiguous(cfg, weights_for(cfg), roots, g)
+    eng.close()
+    assert checked >= 1
+
+
+def test_check_schedule_and_paper_parameters():
+    # S = {5, 7, 9}, n = 11, w = 10 (Section 3.2): stops can only happen at checked steps.
+    mask = sum(1 << (s - 1) for s in (5, 7, 9))
+    cfg = S.scaled_down(S.CONFIGS["llama2_7b"], 256, 4000, threshold=-0.3, max_depth=11, check_mask=mask)
+    eng = engine_for(cfg, TC)
+    roots = S.make_roots(cfg, 0)
+    g = parity.run_gpu(eng, roots)
+    assert int(g["stop_depth"][0]) in (5, 7, 9, 11)
+    parity.compare_with_oracle(cfg, weights_for(cfg), roots, g)
+    eng.close()
+
+
+def test_k1_greedy_chain_and_k_equal_to_limit():
+    base = S.scaled_down(S.CONFIGS["llama2_7b"], 256, 2048, threshold=NEG)
+    for k, depth, m in ((1, 6, 4), (32, 3, 200)):
+        cfg = base.replace(k=k, max_depth=depth, total_tokens=m)
+        for kernel in (SIMT, TC):
+            eng = engine_for(cfg, kernel)
+            roots = S.make_roots(cfg, 0)
+            g = parity.run_gpu(eng, roots)
+            parity.compare_with_oracle(cfg, weights_for(cfg), roots, g)
+            eng.close()
+
+
+# ----------------------------------------------------------------------------- launch modes
+def test_graph_mode_host_variant_and_determinism():
+    cfg = small_cases()["7b"]
+    roots = S.make_roots(cfg, 1)
+    eng_s = engine_for(cfg, TC, P.DDD_LAUNCH_STREAM)
+    a = parity.run_gpu(eng_s, roots)
+    a2 = parity.run_gpu(eng_s, roots)
+    eng_g = engine_for(cfg, TC, P.DDD_LAUNCH_GRAPH)
+    with torch.cuda.stream(torch.cuda.Stream()):
+        b = parity.run_gpu(eng_g, roots)
+        b2 = parity.run_gpu(eng_g, roots)           # second launch replays the captured graph
+        other = S.make_roots(cfg, 2)
+        c = parity.run_gpu(eng_g, other)            # new input pointers: re-captured
+    for name in a:
+        np.testing.assert_array_equal(a[name], a2[name], err_msg=name)    # run-to-run identical
+        np.testing.assert_array_equal(a[name], b[name], err_msg=name)     # graph == stream
+        np.testing.assert_array_equal(b[name], b2[name], err_msg=name)
+    parity.compare_with_oracle(cfg, weights_for(cfg), other, c)
+    # host-buffer entry point
+    host_out = eng_s.make_host_out()
+    eng_s.draft_host(roots["root_hidden"].pin_memory(), roots["root_token"].pin_memory(),
+                     roots["root_pos"].pin_memory(), host_out)
+    for name in host_out:
+        np.testing.assert_array_equal(host_out[name].numpy(), a[name], err_msg=name)
+    assert P.ddd_launches_per_draft(eng_s.handle) == 2 + 2 * cfg.max_depth
+    assert 1 <= P.ddd_lm_head_blocks(eng_s.handle) <= 512
+    eng_s.close()
+    eng_g.close()
+
+
+def test_simt_and_tensor_core_kernels_agree():
+    cfg = small_cases()["70b_batch"]
+    roots = S.make_roots(cfg, 5)
+    e1, e2 = engine_for(cfg, SIMT), engine_for(cfg, TC)
+    a, b = parity.run_gpu(e1, roots), parity.run_gpu(e2, roots)
+    np.testing.assert_array_equal(a["stop_depth"], b["stop_depth"])
+    np.testing.assert_allclose(a["H_trace"], b["H_trace"], atol=2e-3)
+    e1.close()
+    e2.close()
+
+
+# ----------------------------------------------------------------------------- full-size configurations
+@pytest.mark.parametrize("name,n_drafts,threshold", [
+    ("llama2_7b", 2, -4.0), ("llama2_7b", 1, NEG), ("vicuna_13b", 1, -2.0),
+    ("llama2_70b_b16", 1, -2.0), ("llama3_8b_128k", 1, -3.0)])
+def test_full_size_configs_in_bench_launch_configuration(name, n_drafts, threshold):
+    cfg = S.CONFIGS[name].replace(threshold=threshold)
+    eng = engine_for(cfg, P.DDD_LM_HEAD_AUTO, P.DDD_LAUNCH_GRAPH)
+    with torch.cuda.stream(torch.cuda.Stream()):
+        for i in range(n_drafts):
+            roots = S.make_roots(cfg, i)
+            g = parity.run_gpu(eng, roots)
+            parity.compare_with_oracle(cfg, weights_for(cfg), roots, g)
+    eng.close()
+    _weights_cache.clear()
