@@ -1,0 +1,361 @@
+#!/usr/bin/env python
+"""Benchmark of the draft-tree hot path.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One step = one batch of `--drafts-per-step` whole drafts (every expansion pass, the gate,
+the draft step, the rerank and the mask) of the 7B-shaped workload, each from its own seeded
+root.  `value` is drafts per second with inputs resident in HBM; `e2e` is the same metric
+through ddd_draft_host with pinned host buffers.  With N > 1 (torchrun) every rank runs the
+same number of drafts on its own GPU on a disjoint block of draft indices (replicas: no
+data-path collective), and the time is the maximum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+import ddd_synth as S  # noqa: E402
+
+METRIC = "drafts_per_sec"
+UNIT = "drafts/s"
+NEG = -1e30
+FALLBACK_HBM_GBS = 6650.0
+CLOCK_QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+               "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama2_7b", choices=list(S.CONFIGS))
+    ap.add_argument("--threshold", type=float, default=None, help="override the workload's threshold x")
+    ap.add_argument("--drafts-per-step", type=int, default=32)
+    ap.add_argument("--lm-head-reps", type=int, default=200)
+    ap.add_argument("--cpu-sample", type=int, default=None, help="drafts the CPU baseline times")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sweep", action="store_true")
+    return ap.parse_args()
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.file = None
+
+    def start(self):
+        try:
+            self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={CLOCK_QUERY}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=self.file, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.file.flush()
+        self.file.seek(0)
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.file.read().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1]))
+                smax.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.file.close()
+        os.unlink(self.file.name)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def dist_setup(n_gpus: int):
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    return rank, world, local
+
+
+def barrier(world):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+def max_over_ranks(value: float, world: int, device) -> float:
+    if world == 1:
+        return value
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def sum_over_ranks(value: float, world: int, device) -> float:
+    if world == 1:
+        return value
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return float(t.item())
+
+
+def timed_drafts(eng, roots_dev, steps: int, warmup: int, world: int, device):
+    """Returns (ms per step as max over ranks, mean stop depth)."""
+    stream = torch.cuda.current_stream(device)
+
+    def one_step():
+        for r in roots_dev:
+            eng.draft(r["root_hidden"], r["root_token"], r["root_pos"])
+
+    for _ in range(warmup):
+        one_step()
+    torch.cuda.synchronize(device)
+    barrier(world)
+    torch.cuda.synchronize(device)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        one_step()
+    e1.record(stream)
+    torch.cuda.synchronize(device)
+    barrier(world)
+    ms = e0.elapsed_time(e1) / steps
+    return max_over_ranks(ms, world, device), ms
+
+
+def mean_stop_depth(eng, roots_dev, device):
+    depths = []
+    for r in roots_dev:
+        eng.draft(r["root_hidden"], r["root_token"], r["root_pos"])
+        torch.cuda.synchronize(device)
+        assert int(eng.out["status"].item()) == 0, "device reported an error status"
+        depths += eng.out["stop_depth"].cpu().tolist()
+    return sum(depths) / len(depths)
+
+
+def run_reference(args):
+    """The CPU oracle, as it stands, timed on the host cores on a bounded sample."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import ddd_oracle as O
+    cfg = S.CONFIGS[args.workload]
+    if args.threshold is not None:
+        cfg = cfg.replace(threshold=args.threshold)
+    w = S.make_weights(cfg)
+    sample = args.cpu_sample or 1
+    times, depths = [], []
+    idx = 0
+    for step in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        for _ in range(sample):
+            res = O.draft(cfg, w, **S.make_roots(cfg, idx))
+            depths += [r.stop_depth for r in res]
+            idx += 1
+        dt = time.perf_counter() - t0
+        if step >= args.warmup:
+            times.append(dt)
+    ms = 1e3 * sum(times) / len(times)
+    value = sample * cfg.batch / (ms / 1e3)
+    cores = O.num_threads()
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "threshold": cfg.threshold, "drafts_per_step": sample,
+                   "batch": cfg.batch, "mean_stop_depth": sum(depths) / len(depths)},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": f"{sample} draft(s) of {cfg.name} per step, x={cfg.threshold}"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+    import paper_2409_00142_b200 as P
+
+    rank, world, local = dist_setup(args.gpus)
+    device = torch.device("cuda", local)
+    torch.cuda.set_device(device)
+    cfg = S.CONFIGS[args.workload]
+    if args.threshold is not None:
+        cfg = cfg.replace(threshold=args.threshold)
+    weights = S.make_weights(cfg)
+    n_per_rank = args.drafts_per_step
+    my_indices = S.shard_draft_indices(n_per_rank * world, rank, world)
+    roots_host = [S.make_roots(cfg, i) for i in my_indices]
+    stream = torch.cuda.Stream(device)
+
+    with torch.cuda.stream(stream):
+        eng = P.DraftEngine(cfg, weights, device=local, launch_mode=P.DDD_LAUNCH_GRAPH, with_trace=False)
+        roots_dev = [{k: v.to(device) for k, v in r.items()} for r in roots_host]
+        torch.cuda.synchronize(device)
+        depth_mean = mean_stop_depth(eng, roots_dev, device)
+
+        sampler = ClockSampler(local)
+        sampler.start()
+        ms_step, _ = timed_drafts(eng, roots_dev, args.steps, args.warmup, world, device)
+        clocks = sampler.stop()
+        drafts_total = n_per_rank * world * cfg.batch
+        value = drafts_total / (ms_step / 1e3)
+
+        # ---- the LM-head kernel alone: CUDA events on the launching stream, W (> L2) streamed each launch
+        for _ in range(5):
+            eng.lm_head_pass()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(args.lm_head_reps):
+            eng.lm_head_pass()
+        e1.record(stream)
+        torch.cuda.synchronize(device)
+        lm_us = 1e3 * e0.elapsed_time(e1) / args.lm_head_reps
+        elt = 4 if cfg.dtype == "fp32" else 2
+        w_bytes = cfg.vocab * cfg.hidden * elt
+        achieved = w_bytes / (lm_us * 1e-6) / 1e9
+        peak, peak_kind = measured_peak()
+
+        # ---- fixed full depth (x = -inf): per-expansion-step time independent of where drafts stop
+        extra = {}
+        if not args.no_sweep:
+            full_cfg = cfg.replace(threshold=NEG)
+            eng_full = P.DraftEngine(full_cfg, {"W": eng.W, "E": eng.E, "bias": eng.bias,
+                                                "plant_next": eng.plant_next}, device=local,
+                                     launch_mode=P.DDD_LAUNCH_GRAPH, with_trace=False)
+            ms_full, _ = timed_drafts(eng_full, roots_dev, max(3, args.steps // 4), args.warmup, world, device)
+            per_draft_us = 1e3 * ms_full / n_per_rank
+            extra["full_depth"] = {"drafts_per_sec": drafts_total / (ms_full / 1e3),
+                                   "us_per_draft": per_draft_us,
+                                   "us_per_expansion_step": per_draft_us / cfg.max_depth,
+                                   "passes": cfg.max_depth}
+            eng_full.close()
+            if cfg.name == "llama2_7b" and args.threshold is None:
+                sweep = {}
+                for x in S.LLAMA2_7B_THRESHOLDS:
+                    cx = cfg.replace(threshold=x)
+                    ex = P.DraftEngine(cx, {"W": eng.W, "E": eng.E, "bias": eng.bias,
+                                            "plant_next": eng.plant_next}, device=local,
+                                       launch_mode=P.DDD_LAUNCH_GRAPH, with_trace=False)
+                    dm = mean_stop_depth(ex, roots_dev, device)
+                    msx, _ = timed_drafts(ex, roots_dev, max(3, args.steps // 4), args.warmup, world, device)
+                    sweep[str(x)] = {"drafts_per_sec": drafts_total / (msx / 1e3), "mean_stop_depth": dm}
+                    ex.close()
+                extra["threshold_sweep"] = sweep
+
+        # ---- end to end through the host-buffer entry point (pinned host memory, copies inside)
+        host_out = eng.make_host_out(pinned=True)
+        pinned = [{k: v.pin_memory() for k, v in r.items()} for r in roots_host]
+        for r in pinned[:4]:
+            eng.draft_host(r["root_hidden"], r["root_token"], r["root_pos"], host_out)
+        torch.cuda.synchronize(device)
+        barrier(world)
+        t0 = time.perf_counter()
+        e2e_steps = max(2, args.steps // 4)
+        for _ in range(e2e_steps):
+            for r in pinned:
+                eng.draft_host(r["root_hidden"], r["root_token"], r["root_pos"], host_out)
+        torch.cuda.synchronize(device)
+        e2e_ms = 1e3 * (time.perf_counter() - t0) / e2e_steps
+        e2e_ms = max_over_ranks(e2e_ms, world, device)
+        h2d = sum(v.numel() * v.element_size() for v in pinned[0].values()) * n_per_rank
+        d2h = sum(v.numel() * v.element_size() for v in host_out.values()) * n_per_rank
+        launches = P.ddd_launches_per_draft(eng.handle) * n_per_rank * args.steps
+        blocks = P.ddd_lm_head_blocks(eng.handle)
+        eng.close()
+
+    if rank != 0:
+        if world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+        return
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": cfg.dtype if cfg.dtype != "fp32" else "f32", "data": "synthetic",
+        "config": {"workload": cfg.name, "batch": cfg.batch, "hidden": cfg.hidden, "vocab": cfg.vocab,
+                   "k": cfg.k, "max_depth": cfg.max_depth, "total_tokens": cfg.total_tokens,
+                   "threshold": cfg.threshold, "drafts_per_step": n_per_rank * world,
+                   "mean_stop_depth": depth_mean, "parallelism": f"replicas{world}",
+                   "l2": "inputs larger than L2: every pass streams W (%.0f MB) from HBM" % (w_bytes / 1e6),
+                   "launch": "cuda_graph"},
+        "clocks": clocks,
+        "e2e": {"value": n_per_rank * world * cfg.batch / (e2e_ms / 1e3), "unit": UNIT,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": launches,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "traffic": None, "peak_kind": f"of {peak_kind}",
+                     "kernel": "lm_head", "us_per_launch": lm_us, "algorithmic_bytes_per_launch": w_bytes,
+                     "frac_of_8TBs_nominal": achieved / 8000.0, "blocks": blocks},
+    }
+    line.update(extra)
+    if not args.no_cpu_baseline and world == 1:
+        from oracle import ddd_oracle as O
+        sample = args.cpu_sample or 2
+        t0 = time.perf_counter()
+        for i in range(sample):
+            O.draft(cfg, weights, **roots_host[i % len(roots_host)])
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": sample * cfg.batch / dt, "unit": UNIT, "cores": O.num_threads(),
+                                "kind": "oracle",
+                                "sample": f"{sample} draft(s) of {cfg.name}, x={cfg.threshold}, {dt:.1f} s"}
+    print(json.dumps(line))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -39,6 +39,23 @@ __global__ void init_kernel(const Params p, const T* __restrict__ root_hidden,
 }
 
 // ---------------------------------------------------------------------------- select / gate / step
+__device__ __forceinline__ double warp_sum_f64(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFullMask, v, o);
+  return v;
+}
+
+// fp64 -> bf16 bit pattern with one round-to-nearest-even step (normal range): keep the top
+// 7 explicit mantissa bits of the double, then the narrowing conversions are exact.
+__device__ __forceinline__ uint32_t f64_to_bf16_bits(double y) {
+  unsigned long long bits = (unsigned long long)__double_as_longlong(y);
+  const unsigned long long lsb = (bits >> 45) & 1ull;
+  bits += ((1ull << 44) - 1ull) + lsb;
+  bits &= ~((1ull << 45) - 1ull);
+  const float f = (float)__longlong_as_double((long long)bits);
+  return __float_as_uint(f) >> 16;
+}
+
 // Dynamic shared memory: first-entry keys of every LM-head block for each of the k rows.
 __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Params p, const DraftIO io,
                                                                        const int d) {
@@ -190,6 +207,10 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
 
   // ---- phase 3: synthetic draft step, one warp per new beam row:
   //      h_child = round( u / sqrt(mean(u^2) + eps) ),  u = h_parent + E[token]
+  // The rounding to the storage type is a quantisation decision, so everything before it is
+  // done in fp64 and the result is rounded once, directly from fp64: an fp32 evaluation
+  // would flip about one element in 10^5 to the neighbouring bf16 value, and one such flip
+  // moves a logit by up to a few 1e-3.
   if (warp < k) {
     const int i = warp;
     const int parent_slot = sel_flat[i] / k;
@@ -201,21 +222,22 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
       const __nv_bfloat16* hp = static_cast<const __nv_bfloat16*>(p.hbuf[(d - 1) & 1]) + src_row;
       const __nv_bfloat16* e = static_cast<const __nv_bfloat16*>(p.E) + e_row;
       __nv_bfloat16* out = static_cast<__nv_bfloat16*>(p.hbuf[d & 1]) + dst_row;
-      float ss = 0.f;
+      double ss = 0.0;
       for (int j = lane * 8; j < p.Hd; j += 256) {
         const uint4 a = *reinterpret_cast<const uint4*>(hp + j);
         const uint4 c = *reinterpret_cast<const uint4*>(e + j);
         const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, cw[4] = {c.x, c.y, c.z, c.w};
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-          const float u0 = __uint_as_float(aw[q] << 16) + __uint_as_float(cw[q] << 16);
-          const float u1 = __uint_as_float(aw[q] & 0xFFFF0000u) + __uint_as_float(cw[q] & 0xFFFF0000u);
-          ss = fmaf(u0, u0, ss);
-          ss = fmaf(u1, u1, ss);
+          const double u0 = (double)__uint_as_float(aw[q] << 16) + (double)__uint_as_float(cw[q] << 16);
+          const double u1 = (double)__uint_as_float(aw[q] & 0xFFFF0000u) +
+                            (double)__uint_as_float(cw[q] & 0xFFFF0000u);
+          ss = fma(u0, u0, ss);
+          ss = fma(u1, u1, ss);
         }
       }
-      ss = warp_sum(ss);
-      const float inv = 1.0f / sqrtf(ss / (float)p.Hd + p.eps);
+      ss = warp_sum_f64(ss);
+      const double inv = 1.0 / sqrt(ss / (double)p.Hd + (double)p.eps);
       for (int j = lane * 8; j < p.Hd; j += 256) {
         const uint4 a = *reinterpret_cast<const uint4*>(hp + j);
         const uint4 c = *reinterpret_cast<const uint4*>(e + j);
@@ -223,10 +245,10 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
         uint32_t ow[4];
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-          const float u0 = __uint_as_float(aw[q] << 16) + __uint_as_float(cw[q] << 16);
-          const float u1 = __uint_as_float(aw[q] & 0xFFFF0000u) + __uint_as_float(cw[q] & 0xFFFF0000u);
-          const __nv_bfloat162 y = __floats2bfloat162_rn(u0 * inv, u1 * inv);
-          ow[q] = *reinterpret_cast<const uint32_t*>(&y);
+          const double u0 = (double)__uint_as_float(aw[q] << 16) + (double)__uint_as_float(cw[q] << 16);
+          const double u1 = (double)__uint_as_float(aw[q] & 0xFFFF0000u) +
+                            (double)__uint_as_float(cw[q] & 0xFFFF0000u);
+          ow[q] = f64_to_bf16_bits(u0 * inv) | (f64_to_bf16_bits(u1 * inv) << 16);
         }
         *reinterpret_cast<uint4*>(out + j) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
       }
@@ -234,14 +256,14 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
       const float* hp = static_cast<const float*>(p.hbuf[(d - 1) & 1]) + src_row;
       const float* e = static_cast<const float*>(p.E) + e_row;
       float* out = static_cast<float*>(p.hbuf[d & 1]) + dst_row;
-      float ss = 0.f;
+      double ss = 0.0;
       for (int j = lane; j < p.Hd; j += 32) {
-        const float u = hp[j] + e[j];
-        ss = fmaf(u, u, ss);
+        const double u = (double)hp[j] + (double)e[j];
+        ss = fma(u, u, ss);
       }
-      ss = warp_sum(ss);
-      const float inv = 1.0f / sqrtf(ss / (float)p.Hd + p.eps);
-      for (int j = lane; j < p.Hd; j += 32) out[j] = (hp[j] + e[j]) * inv;
+      ss = warp_sum_f64(ss);
+      const double inv = 1.0 / sqrt(ss / (double)p.Hd + (double)p.eps);
+      for (int j = lane; j < p.Hd; j += 32) out[j] = __double2float_rn(((double)hp[j] + (double)e[j]) * inv);
     }
   }
 }

@@ -98,10 +98,11 @@ def test_small_shapes_match_oracle(case, kernel):
 
 
 def test_strict_oracle_agrees_when_no_near_ties():
-    cfg = small_cases()["7b"]
+    # a narrow beam leaves few neighbouring scores, so most drafts have no near-tie at all
+    cfg = small_cases()["7b"].replace(k=3, max_depth=5, total_tokens=20)
     eng = engine_for(cfg, TC)
     checked = 0
-    for i in range(3):
+    for i in range(8):
         roots = S.make_roots(cfg, 10 + i)
         g = parity.run_gpu(eng, roots)
         checked += parity.strict_equal_when_unambiguous(cfg, weights_for(cfg), roots, g)
