@@ -205,6 +205,38 @@ int ddd_lm_head_pass(ddd_handle *h, void *cuda_stream);
 int ddd_launches_per_draft(const ddd_handle *h);
 int ddd_lm_head_blocks(const ddd_handle *h);
 
+/*
+ * One LM-head pass that allocates nothing.  (The paper has no counterpart: this exists for
+ * integration, not for the method.)  For `rows` hidden rows it computes
+ * logits = logit_scale * h W^T + bias, the log-softmax of every row, and the row's k best
+ * tokens with their log-probabilities - the same arithmetic as one pass of ddd_draft - but it
+ * needs no handle and no caller workspace.  It is meant for callers that cannot obtain device
+ * memory at call time: code living inside another library's callback or plug-in interface
+ * that is handed fixed buffers only, a process whose device memory belongs to a framework pool
+ * it must not call into, or a latency-critical loop where cudaMalloc (which may synchronise
+ * the device) is unacceptable.  Its scratch space, the per-block partial results, is a fixed
+ * array of 2,162,688 bytes inside the library's device image; every GPU that loads the
+ * library holds it until the process exits.
+ *   W            DEVICE [vocab][hidden], dtype DDD_DTYPE_*, 16-byte aligned
+ *   bias         DEVICE [vocab] fp32 or NULL
+ *   hidden_rows  DEVICE [rows][hidden], same dtype, 16-byte aligned
+ *   out_token    DEVICE [rows][k] int32, best first (ties: lower token id)
+ *   out_logprob  DEVICE [rows][k] fp32, clamped to <= 0
+ *   out_lse      DEVICE [rows] fp32 logsumexp of the row's logits
+ * Limits: 1 <= rows <= 32, 1 <= k <= DDD_MAX_K, hidden a multiple of 8, vocab > k.  Sizes
+ * beyond these do not fit the fixed scratch and return DDD_ERR_INVALID_ARG; misaligned W or
+ * hidden_rows return DDD_ERR_ALIGNMENT.  Works on the device that is current in the calling
+ * thread and only enqueues two kernels on `cuda_stream`; it calls no allocating routine.
+ * The first call on each device looks up the scratch array's device address (a one-time
+ * set-up under a lock); make that first call before starting any stream capture.
+ * All calls share the one scratch array: it keeps whatever the previous call left, which is
+ * harmless because every slot that is read is rewritten first, but two calls whose kernels
+ * overlap on the GPU (different streams, or different threads) race.  Serialise them.
+ */
+int ddd_lm_head_topk_noalloc(const void *W, const float *bias, const void *hidden_rows, int32_t dtype,
+                             int32_t rows, int32_t hidden, int32_t vocab, int32_t k, float logit_scale,
+                             int32_t *out_token, float *out_logprob, float *out_lse, void *cuda_stream);
+
 /* Releases host state (and the captured graph).  Device memory stays with the caller. */
 int ddd_destroy(ddd_handle *h);
 

@@ -72,6 +72,9 @@ def load_library():
     lib.ddd_launches_per_draft.argtypes = [vp]
     lib.ddd_lm_head_blocks.restype = ctypes.c_int
     lib.ddd_lm_head_blocks.argtypes = [vp]
+    lib.ddd_lm_head_topk_noalloc.restype = ctypes.c_int
+    lib.ddd_lm_head_topk_noalloc.argtypes = [vp, vp, vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
+                                             ctypes.c_int32, ctypes.c_int32, ctypes.c_float, vp, vp, vp, vp]
     lib.ddd_destroy.restype = ctypes.c_int
     lib.ddd_destroy.argtypes = [vp]
     lib.ddd_strerror.restype = ctypes.c_char_p
@@ -83,7 +86,8 @@ def load_library():
 def exported_symbols():
     """Names this binding expects the library to export (all of include/ddd.h)."""
     return ["ddd_workspace_bytes", "ddd_create", "ddd_draft", "ddd_draft_host", "ddd_lm_head_pass",
-            "ddd_launches_per_draft", "ddd_lm_head_blocks", "ddd_destroy", "ddd_strerror"]
+            "ddd_launches_per_draft", "ddd_lm_head_blocks", "ddd_lm_head_topk_noalloc", "ddd_destroy",
+            "ddd_strerror"]
 
 
 # ----------------------------------------------------------------------------- same-name wrappers
@@ -133,6 +137,17 @@ def ddd_launches_per_draft(handle: int) -> int:
 
 def ddd_lm_head_blocks(handle: int) -> int:
     return int(load_library().ddd_lm_head_blocks(handle))
+
+
+def ddd_lm_head_topk_noalloc(W: int, bias: Optional[int], hidden_rows: int, dtype: int, rows: int, hidden: int,
+                             vocab: int, k: int, logit_scale: float, out_token: int, out_logprob: int,
+                             out_lse: int, stream: int) -> None:
+    """LM-head pass with top-k for callers that cannot allocate device memory: the scratch is a
+    fixed array inside the library (see include/ddd.h).  All pointers are device addresses."""
+    rc = load_library().ddd_lm_head_topk_noalloc(W, bias, hidden_rows, dtype, rows, hidden, vocab, k,
+                                                 logit_scale, out_token, out_logprob, out_lse, stream)
+    if rc != 0:
+        raise DddError(rc, "ddd_lm_head_topk_noalloc")
 
 
 def ddd_destroy(handle: int) -> None:
