@@ -18,7 +18,7 @@ size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
   size_t hbuf[2], part_key, part_ms, tree_token, tree_parent, tree_cum, beam_node, beam_tok, beam_cum,
-      row_plant, active, stop_depth, root_pos, n_active, dev_status;
+      row_plant, active, stop_depth, root_pos, n_active, dev_status, w_packed;
   // staging for ddd_draft_host: inputs, then the packed output block
   size_t in_hidden, in_token, in_pos, out_block;
   size_t o_n_out, o_stop, o_token, o_parent, o_depth, o_position, o_cum, o_mask, o_H, o_status, out_bytes;
@@ -70,6 +70,10 @@ Layout make_layout(const ddd_config* c) {
   L.root_pos = take(B * 4);
   L.n_active = take(4);
   L.dev_status = take(4);
+  // packed copy of W for the tensor-core kernel (kept 1024-byte aligned relative to the base)
+  off = (off + 1023) / 1024 * 1024;
+  const bool tc_possible = c->dtype == DDD_DTYPE_BF16 && c->hidden % 64 == 0 && c->lm_head_kernel != DDD_LM_HEAD_SIMT;
+  L.w_packed = take(tc_possible ? tc_packed_bytes(c->vocab, c->hidden) : 0);
   // host-variant staging: inputs packed back to back (each 16-byte aligned), one output block
   L.in_hidden = take(0);
   size_t in = 0;
@@ -210,14 +214,16 @@ int ddd_create(const ddd_config* cfg, const void* W, const void* E, const float*
   p.dev_status = reinterpret_cast<int*>(ws + L.dev_status);
 
   int rc = DDD_OK;
+  // Zero the workspace once so that rows never written by a draft hold finite values.
+  if (cudaMemset(ws, 0, L.total) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) rc = DDD_ERR_CUDA;
   h->lm_kind = cfg->lm_head_kernel;
   if (h->lm_kind == DDD_LM_HEAD_AUTO)
     h->lm_kind = (cfg->dtype == DDD_DTYPE_BF16 && cfg->hidden % 64 == 0) ? DDD_LM_HEAD_TCGEN05 : DDD_LM_HEAD_SIMT;
-  if (h->lm_kind == DDD_LM_HEAD_TCGEN05) {
+  if (rc == DDD_OK && h->lm_kind == DDD_LM_HEAD_TCGEN05) {
     if (prop.major != 10) rc = DDD_ERR_UNSUPPORTED;
-    if (rc == DDD_OK) rc = tc_plan_create(p, h->sm_count, &h->tc);
+    if (rc == DDD_OK) rc = tc_plan_create(p, h->sm_count, ws + L.w_packed, &h->tc);
     if (rc == DDD_OK) p.lm_ctas = h->tc.ctas;
-  } else {
+  } else if (rc == DDD_OK) {
     const int n_tiles = (p.V + kTile - 1) / kTile;
     int ctas = 2 * h->sm_count;
     if (ctas > n_tiles) ctas = n_tiles;
@@ -226,9 +232,6 @@ int ddd_create(const ddd_config* cfg, const void* W, const void* E, const float*
     if (prepare_simt(p) != cudaSuccess) rc = DDD_ERR_CUDA;
   }
   if (rc == DDD_OK && prepare_tree(p) != cudaSuccess) rc = DDD_ERR_CUDA;
-  // Zero the workspace once so that rows never written by a draft hold finite values.
-  if (rc == DDD_OK && (cudaMemset(ws, 0, L.total) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess))
-    rc = DDD_ERR_CUDA;
   if (rc != DDD_OK) {
     cudaGetLastError();
     delete h;

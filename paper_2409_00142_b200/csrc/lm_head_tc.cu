@@ -5,8 +5,13 @@
 // M = 128, N = 16..256 keeps every vocab row in its own tensor-memory lane and every beam
 // row in its own column.  The pass is bound by streaming W from HBM once; everything else
 // hides under that stream:
-//   warp 0     TMA producer: W boxes of 32 vocab rows x 64 hidden elements (128-byte
-//              swizzle) plus the matching slice of h, into a ring of shared-memory stages
+//   warp 0     TMA producer: W comes from a copy that ddd_create packs once into the exact
+//              shared-memory image the MMA wants - pre-swizzled 4 KB chunks of 32 vocab rows x
+//              64 hidden elements, ordered [K-block][32-row unit] - so the rows of one MMA tile
+//              and one K-block are a single contiguous run fetched by one plain bulk copy
+//              (cp.async.bulk); the matching slice of h comes through a 3-D tensor map; both
+//              land in a ring of shared-memory stages.  Issuing a copy costs the thread a few
+//              hundred cycles, so stages are made of few, large copies
 //   warp 1     issues tcgen05.mma into one of two tensor-memory accumulators
 //   warps 2-5  epilogue: tcgen05.ld the finished accumulator, apply scale and bias, fold the
 //              tile into each beam row's online max / sum-exp and running top-k
@@ -14,6 +19,8 @@
 // one partial (max, sum-exp, top-k list) per beam row; logits never reach global memory.
 // Every wait is bounded: when one runs out the block records DDD_ERR_TIMEOUT, drains what
 // it has in flight, frees its tensor memory and returns.
+#include <cstdlib>
+
 #include "lm_head_tc.cuh"
 
 namespace ddd {
@@ -35,11 +42,11 @@ struct SmemPlan {
   int a, b, zt, key, ms, plant, live, bars, tmem_ptr, abort_flag, total;
 };
 
-__host__ __device__ inline SmemPlan smem_plan(int stages, int n_pad, int R, int k) {
+__host__ __device__ inline SmemPlan smem_plan(int stages, int ksub, int n_pad, int R, int k) {
   SmemPlan s;
   int off = 0;
-  s.a = off; off += stages * kABytes;
-  s.b = off; off += stages * n_pad * kBlockK * 2;
+  s.a = off; off += stages * ksub * kABytes;
+  s.b = off; off += stages * ksub * n_pad * kBlockK * 2;
   s.zt = off; off += kChunkCols * kTile * 4;
   s.key = off; off += R * k * 8;
   s.ms = off; off += R * 8;
@@ -102,18 +109,18 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
   }
 }
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y, int z) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y)
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z)
       : "memory");
 }
-__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y,
-                                                 unsigned long long policy) {
+// Plain (untiled) bulk copy global -> shared; addresses and size are multiples of 16 bytes.
+__device__ __forceinline__ void bulk_load_hint(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar,
+                                               unsigned long long policy) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
-      " [%0], [%1, {%3, %4}], [%2], %5;"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "l"(policy)
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+      ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(policy)
       : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -179,15 +186,15 @@ __device__ __forceinline__ uint32_t make_instr_desc(int n) {
 
 // ---------------------------------------------------------------------------- kernel
 __global__ void __launch_bounds__(kTcThreads, 1)
-lm_head_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_w,
+lm_head_tc_kernel(const Params p, const unsigned char* __restrict__ w_packed,
                   const __grid_constant__ CUtensorMap map_h, const int d, const int force_all,
-                  const int n_pad, const int stages, const int tmem_cols) {
+                  const int n_pad, const int stages, const int tmem_cols, const int ksub) {
   if (!force_all && *p.n_active == 0) return;
 
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(
       (reinterpret_cast<uintptr_t>(smem_dyn) + 1023u) & ~static_cast<uintptr_t>(1023u));
-  const SmemPlan sp = smem_plan(stages, n_pad, p.R, p.k);
+  const SmemPlan sp = smem_plan(stages, ksub, n_pad, p.R, p.k);
   float* zt = reinterpret_cast<float*>(smem + sp.zt);
   unsigned long long* st_key = reinterpret_cast<unsigned long long*>(smem + sp.key);
   float2* st_ms = reinterpret_cast<float2*>(smem + sp.ms);
@@ -211,8 +218,29 @@ lm_head_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_w,
   const int bid = blockIdx.x;
   const int my_units = base_units + (bid < rem_units ? 1 : 0);
   const int unit0 = bid * base_units + (bid < rem_units ? bid : rem_units);
+  // MMA tiles: up to four consecutive units, counted from the start of the block's range.
   const int n_tiles = (my_units + 3) / 4;
-  const int num_kb = p.Hd / kBlockK;
+  const int num_kb = p.Hd / (kBlockK * ksub);      // stages per tile; each holds ksub K-blocks of 64
+  const uint32_t a_stage = (uint32_t)ksub * kABytes, b_stage = (uint32_t)ksub * b_bytes;
+
+  // One (tile, K-group) step of the pipeline: which packed chunk it reads and where it lands.
+  const int total_iters = n_tiles * num_kb;
+  const int prefill = total_iters < stages ? total_iters : stages;
+  unsigned long long evict_first = 0ull;
+  auto issue = [&](int it, int stage) {
+    const int t = it / num_kb, kb = it - t * num_kb;
+    const int nu = min(4, my_units - 4 * t);
+    const uint32_t full = bar_full + 8u * stage;
+    mbar_expect_tx(full, (uint32_t)ksub * ((uint32_t)nu * kUnitBytes + b_bytes));
+    // W: for each 64-element K-block the tile's units are one contiguous run of the packed copy
+    const unsigned char* src = w_packed + ((size_t)(kb * ksub) * n_units + (size_t)(unit0 + 4 * t)) * kUnitBytes;
+    const uint32_t dst = a_base + (uint32_t)stage * a_stage;
+    for (int kk = 0; kk < ksub; ++kk)
+      bulk_load_hint(dst + (uint32_t)kk * kABytes, src + (size_t)kk * n_units * kUnitBytes, (uint32_t)nu * kUnitBytes,
+                     full, evict_first);
+    // h: ksub K-blocks of all beam rows in one tensor copy
+    tma_load_3d(b_base + (uint32_t)stage * b_stage, &map_h, full, 0, 0, kb * ksub);
+  };
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < stages; ++s) {
@@ -227,6 +255,9 @@ lm_head_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_w,
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    // Start streaming right away, while the other warps are still setting up.
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(evict_first));
+    for (int it = 0; it < prefill; ++it) issue(it, it);
   }
   if (warp == 1) {   // tensor-memory allocation is a warp-wide operation
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
@@ -248,26 +279,14 @@ lm_head_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_w,
   if (warp == 0) {
     // ======================================================================= TMA producer
     if (lane == 0) {
-      unsigned long long evict_first;
-      asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(evict_first));
-      int stage = 0, issued = 0;
-      uint32_t phase = 0;
+      int stage = prefill % stages, issued = prefill;
+      uint32_t phase = (prefill == stages) ? 1u : 0u;
       bool ok = true;
-      for (int t = 0; t < n_tiles && ok; ++t) {
-        const int units = min(4, my_units - 4 * t);
-        const int row0 = (unit0 + 4 * t) * kUnitRows;
-        for (int kb = 0; kb < num_kb; ++kb) {
-          if (!mbar_wait(bar_empty + 8u * stage, phase ^ 1u, abort_flag, p.dev_status)) { ok = false; break; }
-          const uint32_t full = bar_full + 8u * stage;
-          mbar_expect_tx(full, (uint32_t)units * kUnitBytes + b_bytes);
-          const uint32_t a_dst = a_base + (uint32_t)stage * kABytes;
-          for (int u = 0; u < units; ++u)
-            tma_load_2d_hint(a_dst + (uint32_t)u * kUnitBytes, &map_w, full, kb * kBlockK, row0 + u * kUnitRows,
-                             evict_first);
-          tma_load_2d(b_base + (uint32_t)stage * b_bytes, &map_h, full, kb * kBlockK, 0);
-          ++issued;
-          if (++stage == stages) { stage = 0; phase ^= 1u; }
-        }
+      for (int it = prefill; it < total_iters; ++it) {
+        if (!mbar_wait(bar_empty + 8u * stage, phase ^ 1u, abort_flag, p.dev_status)) { ok = false; break; }
+        issue(it, stage);
+        ++issued;
+        if (++stage == stages) { stage = 0; phase ^= 1u; }
       }
       if (!ok) {
         // gave up: wait (bounded) until every copy already issued has landed
@@ -294,12 +313,14 @@ lm_head_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_w,
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(bar_full + 8u * stage, phase, abort_flag, p.dev_status)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t a_addr = a_base + (uint32_t)stage * kABytes;
-          const uint32_t b_addr = b_base + (uint32_t)stage * b_bytes;
+          for (int kk = 0; kk < ksub; ++kk) {
+            const uint32_t a_addr = a_base + (uint32_t)stage * a_stage + (uint32_t)kk * kABytes;
+            const uint32_t b_addr = b_base + (uint32_t)stage * b_stage + (uint32_t)kk * b_bytes;
 #pragma unroll
-          for (int k4 = 0; k4 < kBlockK / kUmmaK; ++k4) {
-            tc_mma_bf16(d_tmem, make_smem_desc(a_addr + k4 * kUmmaK * 2), make_smem_desc(b_addr + k4 * kUmmaK * 2),
-                        idesc, (kb | k4) != 0 ? 1u : 0u);
+            for (int k4 = 0; k4 < kBlockK / kUmmaK; ++k4) {
+              tc_mma_bf16(d_tmem, make_smem_desc(a_addr + k4 * kUmmaK * 2),
+                          make_smem_desc(b_addr + k4 * kUmmaK * 2), idesc, (kb | kk | k4) != 0 ? 1u : 0u);
+            }
           }
           tc_commit(bar_empty + 8u * stage);     // frees the stage once these MMAs have read it
           if (++stage == stages) { stage = 0; phase ^= 1u; }
@@ -383,6 +404,25 @@ lm_head_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_w,
   }
 }
 
+// ---------------------------------------------------------------------------- one-time repack of W
+// Packed layout: 4 KB chunks, chunk number kb * n_units + u holds rows 32u .. 32u+31 of K-block
+// kb (hidden elements 64 kb .. 64 kb + 63), 128 bytes per row, with the 16-byte pieces of each
+// row permuted by the 128-byte swizzle (piece c of row r sits at piece c ^ (r & 7)).  A run of
+// consecutive chunks is byte for byte the shared-memory image of a K-major SWIZZLE_128B
+// operand, so the LM-head kernel fetches any run of units with one plain bulk copy.  Rows past
+// V are zero.
+__global__ void __launch_bounds__(256) pack_w_kernel(const __nv_bfloat16* __restrict__ W, unsigned char* __restrict__ out,
+                                                     int V, int Hd, int n_units) {
+  const size_t chunk = blockIdx.x;                 // kb * n_units + u
+  const int kb = (int)(chunk / n_units), u = (int)(chunk % n_units);
+  uint4* dst = reinterpret_cast<uint4*>(out + chunk * kUnitBytes);
+  const int r = threadIdx.x >> 3, c = threadIdx.x & 7;     // 32 rows x 8 pieces of 16 bytes
+  const int v = u * kUnitRows + r;
+  uint4 val = make_uint4(0u, 0u, 0u, 0u);
+  if (v < V) val = *reinterpret_cast<const uint4*>(W + (size_t)v * Hd + kb * kBlockK + c * 8);
+  dst[r * 8 + (c ^ (r & 7))] = val;
+}
+
 // ---------------------------------------------------------------------------- host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -400,23 +440,30 @@ EncodeTiledFn get_encode_fn() {
   return fn;
 }
 
-// 2-D bf16 tensor [rows][cols] (cols contiguous), box box_rows x 64 columns, 128-byte swizzle,
-// out-of-range elements read as zero.
-bool encode_2d(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+// The hidden rows [rows][cols] bf16 (cols contiguous) seen as a 3-D tensor {64 columns, rows,
+// cols / 64 K-blocks}: one box of 64 x box_rows x box_kb lands as box_kb consecutive K-major,
+// 128-byte-swizzled operand tiles.  Out-of-range rows read as zero.
+bool encode_hidden_3d(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows,
+                      uint32_t box_kb) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return false;
-  const cuuint64_t dims[2] = {cols, rows};
-  const cuuint64_t strides[1] = {cols * 2};
-  const cuuint32_t box[2] = {(cuuint32_t)kBlockK, box_rows};
-  const cuuint32_t estr[2] = {1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+  const cuuint64_t dims[3] = {(cuuint64_t)kBlockK, rows, cols / kBlockK};
+  const cuuint64_t strides[2] = {cols * 2, (cuuint64_t)kBlockK * 2};
+  const cuuint32_t box[3] = {(cuuint32_t)kBlockK, box_rows, box_kb};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 }  // namespace
 
-int tc_plan_create(const Params& p, int sm_count, TcPlan* plan) {
+size_t tc_packed_bytes(int vocab, int hidden) {
+  const size_t units = ((size_t)vocab + kUnitRows - 1) / kUnitRows;
+  return units * kUnitRows * (size_t)hidden * 2;
+}
+
+int tc_plan_create(const Params& p, int sm_count, void* w_packed, TcPlan* plan) {
   if (p.dtype != DDD_DTYPE_BF16 || p.Hd % kBlockK != 0) return DDD_ERR_UNSUPPORTED;
   const int n_pad = (p.R + 15) / 16 * 16;
   if (n_pad > 256) return DDD_ERR_UNSUPPORTED;
@@ -426,19 +473,34 @@ int tc_plan_create(const Params& p, int sm_count, TcPlan* plan) {
   const int n_units = (p.V + kUnitRows - 1) / kUnitRows;
   int ctas = sm_count < n_units ? sm_count : n_units;
   if (ctas > kMaxLmCtas) ctas = kMaxLmCtas;
+  int ksub = 2;
+  if (const char* e = getenv("DDD_TC_KSUB")) ksub = atoi(e);
+  while (ksub > 1 && (p.Hd % (kBlockK * ksub) != 0 || smem_plan(2, ksub, n_pad, p.R, p.k).total + 1024 > kSmemLimit))
+    ksub /= 2;
+  if (ksub < 1) ksub = 1;
+  int max_stages = 16;
+  if (const char* e = getenv("DDD_TC_STAGES")) max_stages = atoi(e);
   int stages = 0;
-  for (int s = 16; s >= 2; --s) {
-    if (smem_plan(s, n_pad, p.R, p.k).total + 1024 <= kSmemLimit) { stages = s; break; }
+  for (int s = max_stages; s >= 2; --s) {
+    if (smem_plan(s, ksub, n_pad, p.R, p.k).total + 1024 <= kSmemLimit) { stages = s; break; }
   }
   if (stages == 0) return DDD_ERR_UNSUPPORTED;
+  plan->ksub = ksub;
   plan->ctas = ctas;
   plan->n_pad = n_pad;
   plan->stages = stages;
   plan->tmem_cols = cols;
-  plan->smem = (size_t)smem_plan(stages, n_pad, p.R, p.k).total + 1024;
-  if (!encode_2d(&plan->map_w, p.W, (uint64_t)p.V, (uint64_t)p.Hd, kUnitRows)) return DDD_ERR_CUDA;
+  plan->smem = (size_t)smem_plan(stages, ksub, n_pad, p.R, p.k).total + 1024;
+  plan->w_packed = static_cast<unsigned char*>(w_packed);
+  {
+    const size_t chunks = tc_packed_bytes(p.V, p.Hd) / kUnitBytes;
+    pack_w_kernel<<<(unsigned)chunks, 256>>>(static_cast<const __nv_bfloat16*>(p.W), plan->w_packed, p.V, p.Hd,
+                                             n_units);
+    if (cudaGetLastError() != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) return DDD_ERR_CUDA;
+  }
   for (int i = 0; i < 2; ++i)
-    if (!encode_2d(&plan->map_h[i], p.hbuf[i], (uint64_t)p.R, (uint64_t)p.Hd, (uint32_t)n_pad)) return DDD_ERR_CUDA;
+    if (!encode_hidden_3d(&plan->map_h[i], p.hbuf[i], (uint64_t)p.R, (uint64_t)p.Hd, (uint32_t)n_pad, (uint32_t)ksub))
+      return DDD_ERR_CUDA;
   if (cudaFuncSetAttribute(lm_head_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan->smem) !=
       cudaSuccess)
     return DDD_ERR_CUDA;
@@ -446,8 +508,8 @@ int tc_plan_create(const Params& p, int sm_count, TcPlan* plan) {
 }
 
 cudaError_t launch_lm_head_tc(const Params& p, const TcPlan& plan, int d, int force_all, cudaStream_t st) {
-  lm_head_tc_kernel<<<plan.ctas, kTcThreads, plan.smem, st>>>(p, plan.map_w, plan.map_h[(d - 1) & 1], d, force_all,
-                                                              plan.n_pad, plan.stages, plan.tmem_cols);
+  lm_head_tc_kernel<<<plan.ctas, kTcThreads, plan.smem, st>>>(p, plan.w_packed, plan.map_h[(d - 1) & 1], d, force_all,
+                                                              plan.n_pad, plan.stages, plan.tmem_cols, plan.ksub);
   return cudaGetLastError();
 }
 

@@ -8,17 +8,21 @@
 namespace ddd {
 
 struct TcPlan {
-  CUtensorMap map_w;      // W [V][Hd] bf16: box of 64 hidden elements x 32 vocab rows, 128-byte swizzle
+  unsigned char* w_packed; // W re-laid out as pre-swizzled 16 KB chunks [tile of 128 rows][K-block of 64]
   CUtensorMap map_h[2];   // hidden rows [R][Hd] bf16 of each pass parity: box 64 x n_pad
   int ctas;               // persistent thread blocks, one per SM at most
   int n_pad;              // MMA N: beam rows rounded up to a multiple of 16
   int stages;             // depth of the shared-memory ring
+  int ksub;               // 64-element K-blocks per stage
   int tmem_cols;          // allocated tensor-memory columns (power of two)
   size_t smem;            // dynamic shared memory per block
 };
 
-// Encodes the tensor maps and sizes the pipeline.  Returns a DDD_* code.
-int tc_plan_create(const Params& p, int sm_count, TcPlan* plan);
+// Bytes of the packed copy of W (vocab rounded up to whole 128-row tiles).
+size_t tc_packed_bytes(int vocab, int hidden);
+// Packs W into `w_packed` (device, 1024-byte aligned, tc_packed_bytes), encodes the tensor maps of
+// the hidden buffers and sizes the pipeline.  Synchronises the device.  Returns a DDD_* code.
+int tc_plan_create(const Params& p, int sm_count, void* w_packed, TcPlan* plan);
 cudaError_t launch_lm_head_tc(const Params& p, const TcPlan& plan, int d, int force_all, cudaStream_t st);
 
 }  // namespace ddd
