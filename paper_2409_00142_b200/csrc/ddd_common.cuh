@@ -102,6 +102,9 @@ __device__ __forceinline__ bool row_live(const Params& p, int r, int d, int forc
 // the column does not exist or is excluded) into that row's running state:
 //   (m, s)    online max and sum exp(z - m), identical in all lanes
 //   list_key  lane j < k holds the j-th best (logit, token) key seen so far, 0 = empty
+// Tiles must be fed in ascending token order: on equal logits an entry already in the list
+// (lower token) beats any entry of the new tile, and inside the tile lane / slot order is
+// token order, so ties resolve to the lower token with 32-bit compares only.
 __device__ __forceinline__ void row_tile_update(const float* zrow, int tok0, int k, float& m, float& s,
                                                 unsigned long long& list_key) {
   const int lane = threadIdx.x & 31;
@@ -122,35 +125,45 @@ __device__ __forceinline__ void row_tile_update(const float* zrow, int tok0, int
     s += st * __expf(mt - m);
   }
 
-  unsigned long long keys[4];
+  // ordered 32-bit scores; 0 marks "no entry" (a real score is never 0: even -inf maps above it)
+  uint32_t o[4];
 #pragma unroll
-  for (int i = 0; i < 4; ++i)
-    keys[i] = (z[i] == neg_inf()) ? 0ull : make_key(z[i], (uint32_t)(tok0 + 4 * lane + i));
+  for (int i = 0; i < 4; ++i) o[i] = (z[i] == neg_inf()) ? 0u : float_to_ordered(z[i]);
+  uint32_t carry_o = (uint32_t)(list_key >> 32);
+  uint32_t carry_tok = key_index(list_key);
   // Nothing to do unless some entry beats the current k-th best (0 while the list is not full).
-  const unsigned long long kth = __shfl_sync(kFullMask, list_key, k - 1);
-  const bool beats = keys[0] > kth || keys[1] > kth || keys[2] > kth || keys[3] > kth;
-  if (!__any_sync(kFullMask, beats)) return;
+  const uint32_t kth = __shfl_sync(kFullMask, carry_o, k - 1);
+  const uint32_t tile_best = max(max(o[0], o[1]), max(o[2], o[3]));
+  if (!__any_sync(kFullMask, tile_best > kth)) return;
 
-  unsigned long long carry = list_key;
-  unsigned long long best = carry;
-#pragma unroll
-  for (int i = 0; i < 4; ++i) best = keys[i] > best ? keys[i] : best;
-  unsigned long long new_list = 0ull;
+  uint32_t new_o = 0u, new_tok = 0u;
   for (int j = 0; j < k; ++j) {
-    const unsigned long long wk = warp_max_key(best);
-    if (wk == 0ull) break;               // pool exhausted (uniform)
-    if (lane == j) new_list = wk;
-    if (best == wk) {                    // keys are unique (distinct tokens): exactly one owner
-      if (carry == wk) carry = 0ull;
+    const uint32_t best = max(carry_o, max(max(o[0], o[1]), max(o[2], o[3])));
+    const uint32_t top = __reduce_max_sync(kFullMask, best);
+    if (top == 0u) break;                       // pool exhausted (uniform)
+    uint32_t win_tok;
+    const unsigned in_list = __ballot_sync(kFullMask, carry_o == top);
+    if (in_list) {                              // uniform: an old entry wins ties
+      const int src = __ffs(in_list) - 1;
+      win_tok = __shfl_sync(kFullMask, carry_tok, src);
+      if (lane == src) carry_o = 0u;
+    } else {
+      const unsigned in_tile = __ballot_sync(kFullMask, best == top);
+      const int src = __ffs(in_tile) - 1;
+      int slot = 3;
+      if (o[2] == top) slot = 2;
+      if (o[1] == top) slot = 1;
+      if (o[0] == top) slot = 0;
+      win_tok = __shfl_sync(kFullMask, (uint32_t)(tok0 + 4 * lane + slot), src);
+      if (lane == src) {
 #pragma unroll
-      for (int i = 0; i < 4; ++i)
-        if (keys[i] == wk) keys[i] = 0ull;
-      best = carry;
-#pragma unroll
-      for (int i = 0; i < 4; ++i) best = keys[i] > best ? keys[i] : best;
+        for (int i = 0; i < 4; ++i)
+          if (i == slot) o[i] = 0u;
+      }
     }
+    if (lane == j) { new_o = top; new_tok = win_tok; }
   }
-  list_key = new_list;
+  list_key = new_o ? (((unsigned long long)new_o << 32) | (unsigned long long)(0xFFFFFFFFu - new_tok)) : 0ull;
 }
 
 // ---------------------------------------------------------------------------- launchers (host)

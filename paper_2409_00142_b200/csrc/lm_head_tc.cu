@@ -13,21 +13,22 @@
 //              land in a ring of shared-memory stages.  Issuing a copy costs the thread a few
 //              hundred cycles, so stages are made of few, large copies
 //   warp 1     issues tcgen05.mma into one of two tensor-memory accumulators
-//   warps 2-5  epilogue: tcgen05.ld the finished accumulator, apply scale and bias, fold the
-//              tile into each beam row's online max / sum-exp and running top-k
+//   warps 2-17 epilogue: four of them tcgen05.ld the finished accumulator, apply scale and bias
+//              and transpose it through shared memory; then every warp folds one beam row's
+//              128 values into that row's online max / sum-exp and running top-k
 // Each thread block owns a contiguous range of vocab rows (a multiple of 32) and publishes
 // one partial (max, sum-exp, top-k list) per beam row; logits never reach global memory.
 // Every wait is bounded: when one runs out the block records DDD_ERR_TIMEOUT, drains what
 // it has in flight, frees its tensor memory and returns.
-#include <cstdlib>
-
 #include "lm_head_tc.cuh"
 
 namespace ddd {
 
 namespace {
 
-constexpr int kTcThreads = 192;
+constexpr int kEpiWarps = 16;           // warps 2..17: four of them read tensor memory, all fold rows
+constexpr int kEpiThreads = 32 * kEpiWarps;
+constexpr int kTcThreads = 64 + kEpiThreads;
 constexpr int kBlockM = 128;            // vocab rows per MMA tile
 constexpr int kBlockK = 64;             // hidden elements per stage: one 128-byte swizzle row
 constexpr int kUmmaK = 16;              // K of one tcgen05.mma with 16-bit operands
@@ -152,20 +153,22 @@ __device__ __forceinline__ void tc_load_16cols(uint32_t taddr, float (&v)[16]) {
 #pragma unroll
   for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
-__device__ __forceinline__ void epilogue_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
-// Barrier over the 128 epilogue threads that also ANDs a flag, so that all four warps take
-// the same decision after a bounded wait.
+__device__ __forceinline__ void epilogue_barrier() {
+  asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+}
+// Barrier over the epilogue threads that also ANDs a flag, so that all their warps take the
+// same decision after a bounded wait.
 __device__ __forceinline__ bool epilogue_all(bool ok) {
   uint32_t r;
   asm volatile(
       "{\n"
       ".reg .pred p, q;\n"
       "setp.ne.b32 p, %1, 0;\n"
-      "bar.red.and.pred q, 1, 128, p;\n"
+      "bar.red.and.pred q, 1, %2, p;\n"
       "selp.u32 %0, 1, 0, q;\n"
       "}\n"
       : "=r"(r)
-      : "r"(ok ? 1u : 0u)
+      : "r"(ok ? 1u : 0u), "n"(kEpiThreads)
       : "memory");
   return r != 0;
 }
@@ -257,8 +260,9 @@ lm_head_tc_kernel(const Params p, const unsigned char* __restrict__ w_packed,
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     // Start streaming right away, while the other warps are still setting up.
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(evict_first));
-    for (int it = 0; it < prefill; ++it) issue(it, it);
+    issue(0, 0);
   }
+  __syncwarp();
   if (warp == 1) {   // tensor-memory allocation is a warp-wide operation
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                  ::"r"(smem_u32(tmem_ptr)), "r"((uint32_t)tmem_cols) : "memory");
@@ -276,43 +280,50 @@ lm_head_tc_kernel(const Params p, const unsigned char* __restrict__ w_packed,
   tc_fence_after();
   const uint32_t tmem_base = *tmem_ptr;
 
+  // Warps 0 and 1 run their loops with all 32 lanes (every lane waits, lane 0 issues), so that
+  // each warp stays converged for the block-wide barriers and the warp-wide tcgen05 calls.
   if (warp == 0) {
     // ======================================================================= TMA producer
-    if (lane == 0) {
-      int stage = prefill % stages, issued = prefill;
-      uint32_t phase = (prefill == stages) ? 1u : 0u;
-      bool ok = true;
-      for (int it = prefill; it < total_iters; ++it) {
-        if (!mbar_wait(bar_empty + 8u * stage, phase ^ 1u, abort_flag, p.dev_status)) { ok = false; break; }
-        issue(it, stage);
-        ++issued;
-        if (++stage == stages) { stage = 0; phase ^= 1u; }
+    if (lane == 0)
+      for (int it = 1; it < prefill; ++it) issue(it, it);
+    __syncwarp();
+    int stage = prefill % stages, issued = prefill;
+    uint32_t phase = (prefill == stages) ? 1u : 0u;
+    bool ok = true;
+    for (int it = prefill; it < total_iters; ++it) {
+      ok = __all_sync(kFullMask, mbar_wait(bar_empty + 8u * stage, phase ^ 1u, abort_flag, p.dev_status));
+      if (!ok) break;
+      if (lane == 0) issue(it, stage);
+      __syncwarp();
+      ++issued;
+      if (++stage == stages) { stage = 0; phase ^= 1u; }
+    }
+    if (!ok) {
+      // gave up: wait (bounded) until every copy already issued has landed
+      for (int s = 0; s < stages; ++s) {
+        const int fills = (issued + stages - 1 - s) / stages;
+        if (fills > 0) mbar_wait(bar_full + 8u * s, (uint32_t)((fills - 1) & 1), abort_flag, p.dev_status, false);
       }
-      if (!ok) {
-        // gave up: wait (bounded) until every copy already issued has landed
-        for (int s = 0; s < stages; ++s) {
-          const int fills = (issued + stages - 1 - s) / stages;
-          if (fills > 0)
-            mbar_wait(bar_full + 8u * s, (uint32_t)((fills - 1) & 1), abort_flag, p.dev_status, false);
-        }
-      }
+      __syncwarp();
     }
   } else if (warp == 1) {
     // ======================================================================= MMA issuer
-    if (lane == 0) {
-      const uint32_t idesc = make_instr_desc(n_pad);
-      int stage = 0;
-      uint32_t phase = 0;
-      bool ok = true;
-      for (int t = 0; t < n_tiles && ok; ++t) {
-        const int acc = t & 1;
-        const uint32_t acc_phase = (uint32_t)(t >> 1) & 1u;
-        if (!mbar_wait(bar_tempty + 8u * acc, acc_phase ^ 1u, abort_flag, p.dev_status)) { ok = false; break; }
+    const uint32_t idesc = make_instr_desc(n_pad);
+    int stage = 0;
+    uint32_t phase = 0;
+    bool ok = true;
+    for (int t = 0; t < n_tiles && ok; ++t) {
+      const int acc = t & 1;
+      const uint32_t acc_phase = (uint32_t)(t >> 1) & 1u;
+      ok = __all_sync(kFullMask, mbar_wait(bar_tempty + 8u * acc, acc_phase ^ 1u, abort_flag, p.dev_status));
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t d_tmem = tmem_base + (uint32_t)(acc * n_pad);
+      for (int kb = 0; kb < num_kb; ++kb) {
+        ok = __all_sync(kFullMask, mbar_wait(bar_full + 8u * stage, phase, abort_flag, p.dev_status));
+        if (!ok) break;
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * n_pad);
-        for (int kb = 0; kb < num_kb; ++kb) {
-          if (!mbar_wait(bar_full + 8u * stage, phase, abort_flag, p.dev_status)) { ok = false; break; }
-          tc_fence_after();
+        if (lane == 0) {
           for (int kk = 0; kk < ksub; ++kk) {
             const uint32_t a_addr = a_base + (uint32_t)stage * a_stage + (uint32_t)kk * kABytes;
             const uint32_t b_addr = b_base + (uint32_t)stage * b_stage + (uint32_t)kk * b_bytes;
@@ -323,20 +334,25 @@ lm_head_tc_kernel(const Params p, const unsigned char* __restrict__ w_packed,
             }
           }
           tc_commit(bar_empty + 8u * stage);     // frees the stage once these MMAs have read it
-          if (++stage == stages) { stage = 0; phase ^= 1u; }
         }
-        if (ok) tc_commit(bar_tfull + 8u * acc);   // accumulator complete
+        __syncwarp();
+        if (++stage == stages) { stage = 0; phase ^= 1u; }
       }
-      if (!ok) {
-        // make sure no MMA is still running before tensor memory is released
-        tc_commit(bar_spare);
-        mbar_wait(bar_spare, 0u, abort_flag, p.dev_status, false);
-      }
+      if (ok && lane == 0) tc_commit(bar_tfull + 8u * acc);   // accumulator complete
+      __syncwarp();
+    }
+    if (!ok) {
+      // make sure no MMA is still running before tensor memory is released
+      if (lane == 0) tc_commit(bar_spare);
+      __syncwarp();
+      mbar_wait(bar_spare, 0u, abort_flag, p.dev_status, false);
+      __syncwarp();
     }
   } else {
     // ======================================================================= epilogue
-    const int quarter = warp & 3;            // tensor-memory lanes this warp may read
-    const int ew = warp - 2;                 // owner of beam rows r with r % 4 == ew
+    const int quarter = warp & 3;            // tensor-memory lanes this warp may read (loader warps)
+    const int ew = warp - 2;                 // owner of beam rows r with r % kEpiWarps == ew
+    const bool loader = ew < 4;              // warps 2..5 cover the four lane quarters
     const int n_chunks = (p.R + kChunkCols - 1) / kChunkCols;
     bool ok = true;
     for (int t = 0; t < n_tiles && ok; ++t) {
@@ -354,23 +370,25 @@ lm_head_tc_kernel(const Params p, const unsigned char* __restrict__ w_packed,
       const float bias = (v_ok && p.bias) ? p.bias[v] : 0.f;
       for (int ch = 0; ch < n_chunks; ++ch) {
         const int c0 = ch * kChunkCols;
-        float accv[16];
-        tc_load_16cols(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * n_pad + c0), accv);
-        if (ch == n_chunks - 1) {
-          // accumulator fully read by this warp: hand it back to the MMA warp
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(bar_tempty + 8u * acc);
-        }
+        if (loader) {
+          float accv[16];
+          tc_load_16cols(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * n_pad + c0), accv);
+          if (ch == n_chunks - 1) {
+            // accumulator fully read by this warp: hand it back to the MMA warp
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_tempty + 8u * acc);
+          }
 #pragma unroll
-        for (int c = 0; c < kChunkCols; ++c) {
-          const int r = c0 + c;
-          float z = neg_inf();
-          if (v_ok && r < p.R && s_plant[r] != v) z = fmaf(accv[c], p.s, bias);
-          zt[c * kTile + vrow] = z;
+          for (int c = 0; c < kChunkCols; ++c) {
+            const int r = c0 + c;
+            float z = neg_inf();
+            if (v_ok && r < p.R && s_plant[r] != v) z = fmaf(accv[c], p.s, bias);
+            zt[c * kTile + vrow] = z;
+          }
         }
         epilogue_barrier();
-        for (int rr = ew; rr < kChunkCols; rr += 4) {
+        for (int rr = ew; rr < kChunkCols; rr += kEpiWarps) {
           const int r = c0 + rr;
           if (r >= p.R || !s_live[r]) continue;
           float2 ms = st_ms[r];
@@ -384,7 +402,7 @@ lm_head_tc_kernel(const Params p, const unsigned char* __restrict__ w_packed,
     }
     // publish this block's partial results (each row by its owning warp)
     if (ok) {
-      for (int r = ew; r < p.R; r += 4) {
+      for (int r = ew; r < p.R; r += kEpiWarps) {
         if (!s_live[r]) continue;
         const size_t slot = (size_t)bid * p.R + r;
         if (lane < p.k) p.part_key[slot * p.k + lane] = st_key[r * p.k + lane];
@@ -393,7 +411,9 @@ lm_head_tc_kernel(const Params p, const unsigned char* __restrict__ w_packed,
     }
   }
 
-  // ---- teardown: everyone meets, then the allocating warp frees tensor memory
+  // ---- teardown: everyone meets, then the allocating warp frees tensor memory.  Warps 0 and 1
+  // ran single-lane loops: reconverge them first, the block barrier counts whole warps.
+  __syncwarp();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -473,15 +493,13 @@ int tc_plan_create(const Params& p, int sm_count, void* w_packed, TcPlan* plan) 
   const int n_units = (p.V + kUnitRows - 1) / kUnitRows;
   int ctas = sm_count < n_units ? sm_count : n_units;
   if (ctas > kMaxLmCtas) ctas = kMaxLmCtas;
-  int ksub = 2;
-  if (const char* e = getenv("DDD_TC_KSUB")) ksub = atoi(e);
-  while (ksub > 1 && (p.Hd % (kBlockK * ksub) != 0 || smem_plan(2, ksub, n_pad, p.R, p.k).total + 1024 > kSmemLimit))
+  // K-blocks per stage: as many as still leave a ring of three stages (the producer thread
+  // pays a fixed few hundred cycles per copy it issues, so few large copies win), at most 4.
+  int ksub = 4;
+  while (ksub > 1 && (p.Hd % (kBlockK * ksub) != 0 || smem_plan(3, ksub, n_pad, p.R, p.k).total + 1024 > kSmemLimit))
     ksub /= 2;
-  if (ksub < 1) ksub = 1;
-  int max_stages = 16;
-  if (const char* e = getenv("DDD_TC_STAGES")) max_stages = atoi(e);
   int stages = 0;
-  for (int s = max_stages; s >= 2; --s) {
+  for (int s = 8; s >= 2; --s) {
     if (smem_plan(s, ksub, n_pad, p.R, p.k).total + 1024 <= kSmemLimit) { stages = s; break; }
   }
   if (stages == 0) return DDD_ERR_UNSUPPORTED;
