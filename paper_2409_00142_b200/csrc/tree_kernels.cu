@@ -56,35 +56,324 @@ __device__ __forceinline__ uint32_t f64_to_bf16_bits(double y) {
   return __float_as_uint(f) >> 16;
 }
 
-// Dynamic shared memory: first-entry keys of every LM-head block for each of the k rows.
+// Loads issued by one thread are batched (a few independent loads, then their use): a single
+// block runs this kernel between two LM-head passes, so its time is made of memory round
+// trips, and a loop that loads and uses one value per iteration pays one trip per iteration.
+constexpr int kSelCandCap = 256;   // candidates kept per row by the pruned merge (k <= 16: k*k)
+
+// Merge of one beam row's per-block partial lists, k <= 16.  first_s holds every block's best
+// key.  The k-th largest of those, T, is a lower bound of the row's k-th best key, and only
+// the k blocks whose best key reaches T can hold anything >= T: their lists are fetched, the
+// entries >= T (at most k*k, usually about 2k) are collected and the k best of them are the
+// answer.  Lane j returns the j-th best key (0 if there is none).
+__device__ __forceinline__ unsigned long long merge_row_pruned(const Params& p, int r, int k, int nc,
+                                                               const unsigned long long* first_s,
+                                                               unsigned long long* cand_s, int* cand_n) {
+  const int lane = threadIdx.x & 31;
+  unsigned long long prev = ~0ull, T = 1ull;
+  for (int j = 0; j < k; ++j) {
+    unsigned long long best = 0ull;
+    for (int c = lane; c < nc; c += 32) {
+      const unsigned long long key = first_s[c];
+      if (key < prev && key > best) best = key;
+    }
+    const unsigned long long wk = warp_max_key(best);
+    if (wk == 0ull) { T = 1ull; break; }      // fewer than k blocks have anything: keep all
+    prev = wk;
+    T = wk;
+  }
+  if (lane == 0) *cand_n = 0;
+  __syncwarp();
+  for (int c = lane; c < nc; c += 32) {
+    if (first_s[c] < T) continue;
+    const unsigned long long* list = p.part_key + ((size_t)c * p.R + r) * k;
+    unsigned long long e[16];
+#pragma unroll
+    for (int q = 0; q < 16; ++q) e[q] = q < k ? list[q] : 0ull;
+#pragma unroll
+    for (int q = 0; q < 16; ++q)
+      if (e[q] >= T) {
+        const int pos = atomicAdd(cand_n, 1);
+        if (pos < kSelCandCap) cand_s[pos] = e[q];
+      }
+  }
+  __syncwarp();
+  const int C = min(*cand_n, kSelCandCap);
+  unsigned long long res = 0ull;
+  prev = ~0ull;
+  for (int j = 0; j < k; ++j) {
+    unsigned long long best = 0ull;
+    for (int c = lane; c < C; c += 32) {
+      const unsigned long long key = cand_s[c];
+      if (key < prev && key > best) best = key;
+    }
+    const unsigned long long wk = warp_max_key(best);
+    if (wk == 0ull) break;
+    if (lane == j) res = wk;
+    prev = wk;
+  }
+  return res;
+}
+
+// Same result for any k: pick the k blocks with the best first keys, then walk their sorted
+// lists in a k-way merge straight from global memory (lane j owns one list).
+__device__ __forceinline__ unsigned long long merge_row_kway(const Params& p, int r, int k, int nc,
+                                                             const unsigned long long* first_s) {
+  const int lane = threadIdx.x & 31;
+  unsigned long long prev = ~0ull, cur = 0ull, nxt = 0ull;
+  int my_cta = -1;
+  for (int j = 0; j < k; ++j) {
+    unsigned long long best = 0ull;
+    int best_c = -1;
+    for (int c = lane; c < nc; c += 32) {
+      const unsigned long long key = first_s[c];
+      if (key < prev && key > best) { best = key; best_c = c; }
+    }
+    const unsigned long long wk = warp_max_key(best);
+    if (wk == 0ull) break;
+    const unsigned owner = __ballot_sync(kFullMask, best == wk);
+    const int win_c = __shfl_sync(kFullMask, best_c, __ffs(owner) - 1);
+    if (lane == j) { cur = wk; my_cta = win_c; }
+    prev = wk;
+  }
+  const unsigned long long* my_list = my_cta >= 0 ? p.part_key + ((size_t)my_cta * p.R + r) * k : nullptr;
+  int pos = 1;
+  if (my_list && pos < k) nxt = my_list[pos];
+  unsigned long long res = 0ull;
+  for (int j = 0; j < k; ++j) {
+    const unsigned long long wk = warp_max_key(cur);
+    if (wk == 0ull) break;
+    if (lane == j) res = wk;
+    if (cur == wk) {
+      cur = nxt;
+      ++pos;
+      nxt = (my_list && pos < k) ? my_list[pos] : 0ull;
+    }
+  }
+  return res;
+}
+
+// 8 (bf16) or 4 (fp32) consecutive elements of h_parent + E[token], formed in fp64.
+template <typename T>
+struct Chunk;
+template <>
+struct Chunk<__nv_bfloat16> {
+  static constexpr int N = 8;
+  typedef uint4 Raw;
+  __device__ static void sum(const uint4& a, const uint4& c, double (&u)[8]) {
+    const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, cw[4] = {c.x, c.y, c.z, c.w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      u[2 * q] = (double)__uint_as_float(aw[q] << 16) + (double)__uint_as_float(cw[q] << 16);
+      u[2 * q + 1] = (double)__uint_as_float(aw[q] & 0xFFFF0000u) + (double)__uint_as_float(cw[q] & 0xFFFF0000u);
+    }
+  }
+  __device__ static uint4 round(const double (&y)[8]) {
+    uint32_t w[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) w[q] = f64_to_bf16_bits(y[2 * q]) | (f64_to_bf16_bits(y[2 * q + 1]) << 16);
+    return make_uint4(w[0], w[1], w[2], w[3]);
+  }
+};
+template <>
+struct Chunk<float> {
+  static constexpr int N = 4;
+  typedef uint4 Raw;
+  __device__ static void sum(const uint4& a, const uint4& c, double (&u)[4]) {
+    u[0] = (double)__uint_as_float(a.x) + (double)__uint_as_float(c.x);
+    u[1] = (double)__uint_as_float(a.y) + (double)__uint_as_float(c.y);
+    u[2] = (double)__uint_as_float(a.z) + (double)__uint_as_float(c.z);
+    u[3] = (double)__uint_as_float(a.w) + (double)__uint_as_float(c.w);
+  }
+  __device__ static uint4 round(const double (&y)[4]) {
+    return make_uint4(__float_as_uint(__double2float_rn(y[0])), __float_as_uint(__double2float_rn(y[1])),
+                      __float_as_uint(__double2float_rn(y[2])), __float_as_uint(__double2float_rn(y[3])));
+  }
+};
+
+// Synthetic draft step for the k new beam rows of one sequence, by the whole block:
+//   h_child = round( u / sqrt(mean(u^2) + eps) ),  u = h_parent + E[token]
+// The rounding to the storage type is a quantisation decision, so everything before it is done
+// in fp64 and the result is rounded once, directly from fp64: an fp32 evaluation would flip
+// about one element in 10^5 to the neighbouring bf16 value, and one such flip moves a logit by
+// up to a few 1e-3.  Work is cut into 16-byte chunks; a warp's 32 chunks lie in one row
+// (the caller checks that a row has a multiple of 32 chunks), and per-row sums are combined
+// in a fixed order.
+template <typename T>
+__device__ void draft_step_block(const Params& p, int b, int d, const int* sel_flat, const int* sel_tok,
+                                 double* row_part /* [k][slots] */, double* row_inv /* [k] */) {
+  constexpr int N = Chunk<T>::N;
+  constexpr int kBatch = 4;
+  const int k = p.k, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int cpr = p.Hd / N;            // chunks per row
+  const int slots = cpr / 32;          // warp-sized groups of chunks per row
+  const int total = k * cpr;
+  const uint4* Hsrc = reinterpret_cast<const uint4*>(p.hbuf[(d - 1) & 1]);
+  const uint4* Esrc = reinterpret_cast<const uint4*>(p.E);
+  uint4* Hdst = reinterpret_cast<uint4*>(p.hbuf[d & 1]);
+  auto locate = [&](int q, size_t& hs, size_t& es, size_t& hd, int& row) {
+    row = q / cpr;
+    const int col = q - row * cpr;
+    const int tok = sel_tok[row];
+    hs = (size_t)(b * k + sel_flat[row] / k) * cpr + col;
+    es = (size_t)(tok >= 0 && tok < p.V ? tok : 0) * cpr + col;
+    hd = (size_t)(b * k + row) * cpr + col;
+  };
+  // pass 1: sum of squares per row
+  for (int q0 = threadIdx.x; q0 < total; q0 += kBatch * blockDim.x) {
+    uint4 hv[kBatch], ev[kBatch];
+    int rows[kBatch];
+#pragma unroll
+    for (int i = 0; i < kBatch; ++i) {
+      const int q = q0 + i * blockDim.x;
+      rows[i] = -1;
+      if (q < total) {
+        size_t hs, es, hd;
+        locate(q, hs, es, hd, rows[i]);
+        hv[i] = Hsrc[hs];
+        ev[i] = Esrc[es];
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < kBatch; ++i) {
+      const int q = q0 + i * blockDim.x;
+      if (q0 - lane + i * (int)blockDim.x >= total) continue;   // whole warp past the end (uniform)
+      double ss = 0.0;
+      if (rows[i] >= 0) {
+        double u[N];
+        Chunk<T>::sum(hv[i], ev[i], u);
+#pragma unroll
+        for (int e = 0; e < N; ++e) ss = fma(u[e], u[e], ss);
+      }
+      ss = warp_sum_f64(ss);
+      if (lane == 0) {
+        const int row = q / cpr;
+        row_part[row * slots + (q - row * cpr) / 32] = ss;
+      }
+    }
+  }
+  __syncthreads();
+  if (warp < k && lane == 0) {
+    double ss = 0.0;
+    for (int j = 0; j < slots; ++j) ss += row_part[warp * slots + j];
+    row_inv[warp] = 1.0 / sqrt(ss / (double)p.Hd + (double)p.eps);
+  }
+  __syncthreads();
+  // pass 2: scale, round once, store (the inputs come back from the L1 / L2 caches)
+  for (int q0 = threadIdx.x; q0 < total; q0 += kBatch * blockDim.x) {
+    uint4 hv[kBatch], ev[kBatch];
+    size_t dst[kBatch];
+    int rows[kBatch];
+#pragma unroll
+    for (int i = 0; i < kBatch; ++i) {
+      const int q = q0 + i * blockDim.x;
+      rows[i] = -1;
+      if (q < total) {
+        size_t hs, es;
+        locate(q, hs, es, dst[i], rows[i]);
+        hv[i] = Hsrc[hs];
+        ev[i] = Esrc[es];
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < kBatch; ++i) {
+      if (rows[i] < 0) continue;
+      double u[N];
+      Chunk<T>::sum(hv[i], ev[i], u);
+      const double inv = row_inv[rows[i]];
+#pragma unroll
+      for (int e = 0; e < N; ++e) u[e] *= inv;
+      Hdst[dst[i]] = Chunk<T>::round(u);
+    }
+  }
+}
+
+// The same step with one warp per row, for hidden sizes whose rows are not a whole number of
+// 32-chunk groups.
+template <typename T>
+__device__ void draft_step_warp(const Params& p, int b, int d, const int* sel_flat, const int* sel_tok) {
+  constexpr int N = Chunk<T>::N;
+  const int k = p.k, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (warp >= k) return;
+  const int cpr = p.Hd / N;
+  const int tok = sel_tok[warp];
+  const uint4* hp = reinterpret_cast<const uint4*>(p.hbuf[(d - 1) & 1]) + (size_t)(b * k + sel_flat[warp] / k) * cpr;
+  const uint4* e = reinterpret_cast<const uint4*>(p.E) + (size_t)(tok >= 0 && tok < p.V ? tok : 0) * cpr;
+  uint4* out = reinterpret_cast<uint4*>(p.hbuf[d & 1]) + (size_t)(b * k + warp) * cpr;
+  double ss = 0.0;
+  for (int c = lane; c < cpr; c += 32) {
+    double u[N];
+    Chunk<T>::sum(hp[c], e[c], u);
+#pragma unroll
+    for (int i = 0; i < N; ++i) ss = fma(u[i], u[i], ss);
+  }
+  ss = warp_sum_f64(ss);
+  const double inv = 1.0 / sqrt(ss / (double)p.Hd + (double)p.eps);
+  for (int c = lane; c < cpr; c += 32) {
+    double u[N];
+    Chunk<T>::sum(hp[c], e[c], u);
+#pragma unroll
+    for (int i = 0; i < N; ++i) u[i] *= inv;
+    out[c] = Chunk<T>::round(u);
+  }
+}
+
+template <typename T>
+__device__ void draft_step(const Params& p, int b, int d, const int* sel_flat, const int* sel_tok, double* row_part,
+                           double* row_inv) {
+  const int cpr = p.Hd / Chunk<T>::N;
+  if (cpr % 32 == 0 && cpr / 32 <= 64)
+    draft_step_block<T>(p, b, d, sel_flat, sel_tok, row_part, row_inv);
+  else
+    draft_step_warp<T>(p, b, d, sel_flat, sel_tok);
+}
+
+// Dynamic shared memory: per beam row of this sequence, every LM-head block's best key and
+// its (max, sum-exp); then the candidate lists of the pruned merge.
 __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Params p, const DraftIO io,
                                                                        const int d) {
   const int b = blockIdx.x;
   if (p.active[b] == 0) return;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int k = p.k, nc = p.lm_ctas, R = p.R;
+  const int P = (d == 1) ? 1 : k;                            // beam rows of this sequence in pass d
+  const int base = (d == 1) ? 1 : 1 + k + (d - 2) * k * k;   // node id of candidate (0, 0)
+  const bool pruned = k <= 16;
+
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  unsigned long long* firsts = reinterpret_cast<unsigned long long*>(smem_raw);   // [k][lm_ctas]
+  unsigned long long* firsts = reinterpret_cast<unsigned long long*>(smem_raw);                // [k][nc]
+  float2* ms_s = reinterpret_cast<float2*>(firsts + (size_t)k * nc);                            // [k][nc]
+  unsigned long long* cand_list = reinterpret_cast<unsigned long long*>(ms_s + (size_t)k * nc);  // [k][cap]
   __shared__ unsigned long long cand_key[DDD_MAX_K * DDD_MAX_K];
   __shared__ float cand_val[DDD_MAX_K * DDD_MAX_K];
   __shared__ int cand_tok[DDD_MAX_K * DDD_MAX_K];
   __shared__ int sel_flat[DDD_MAX_K];
   __shared__ int sel_tok[DDD_MAX_K];
+  __shared__ int cand_count[DDD_MAX_K];
+  __shared__ double row_part[DDD_MAX_K * 64];
+  __shared__ double row_inv[DDD_MAX_K];
   __shared__ int s_stop;
 
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int k = p.k, nc = p.lm_ctas, R = p.R;
-  const int P = (d == 1) ? 1 : k;                            // beam rows of this sequence in pass d
-  const int base = (d == 1) ? 1 : 1 + k + (d - 2) * k * k;   // node id of candidate (0, 0)
+  // ---- phase 0: the whole block fetches what phase 1 needs in one round trip
+  for (int i = threadIdx.x; i < P * nc; i += blockDim.x) {
+    const int pr = i / nc, c = i - pr * nc;
+    const size_t slot = (size_t)c * R + (b * k + pr);
+    firsts[pr * nc + c] = p.part_key[slot * k];
+    ms_s[pr * nc + c] = p.part_ms[slot];
+  }
+  __syncthreads();
 
   // ---- phase 1: one warp per beam row merges the per-block partials of the LM-head pass
   if (warp < P) {
     const int pr = warp, r = b * k + pr;
+    const float2* my_ms = ms_s + (size_t)pr * nc;
     // log-sum-exp over all blocks (fixed lane-strided order, then a butterfly: deterministic)
     float M = neg_inf();
-    for (int c = lane; c < nc; c += 32) M = fmaxf(M, p.part_ms[(size_t)c * R + r].x);
+    for (int c = lane; c < nc; c += 32) M = fmaxf(M, my_ms[c].x);
     M = ordered_to_float(__reduce_max_sync(kFullMask, float_to_ordered(M)));
     float S = 0.f;
     for (int c = lane; c < nc; c += 32) {
-      const float2 ms = p.part_ms[(size_t)c * R + r];
+      const float2 ms = my_ms[c];
       if (ms.y > 0.f) S += ms.y * expf(ms.x - M);
     }
     S = warp_sum(S);
@@ -100,42 +389,10 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
     }
     const float lse = M + logf(S);
 
-    // the k blocks with the best first entries are the only ones that can hold a top-k entry
-    unsigned long long* my_first = firsts + (size_t)pr * nc;
-    for (int c = lane; c < nc; c += 32) my_first[c] = p.part_key[((size_t)c * R + r) * k];
-    __syncwarp();
-    unsigned long long prev = ~0ull, cur = 0ull, nxt = 0ull;
-    int my_cta = -1;
-    for (int j = 0; j < k; ++j) {
-      unsigned long long best = 0ull;
-      int best_c = -1;
-      for (int c = lane; c < nc; c += 32) {
-        const unsigned long long key = my_first[c];
-        if (key < prev && key > best) { best = key; best_c = c; }
-      }
-      const unsigned long long wk = warp_max_key(best);
-      if (wk == 0ull) break;
-      const unsigned owner = __ballot_sync(kFullMask, best == wk);
-      const int win_c = __shfl_sync(kFullMask, best_c, __ffs(owner) - 1);
-      if (lane == j) { cur = wk; my_cta = win_c; }
-      prev = wk;
-    }
-    // k-way merge of those blocks' sorted lists; lane j walks the list of block my_cta
-    const unsigned long long* my_list =
-        my_cta >= 0 ? p.part_key + ((size_t)my_cta * R + r) * k : nullptr;
-    int pos = 1;
-    if (my_list && pos < k) nxt = my_list[pos];
-    unsigned long long res = 0ull;
-    for (int j = 0; j < k; ++j) {
-      const unsigned long long wk = warp_max_key(cur);
-      if (wk == 0ull) break;
-      if (lane == j) res = wk;
-      if (cur == wk) {
-        cur = nxt;
-        ++pos;
-        nxt = (my_list && pos < k) ? my_list[pos] : 0ull;
-      }
-    }
+    unsigned long long res =
+        pruned ? merge_row_pruned(p, r, k, nc, firsts + (size_t)pr * nc, cand_list + (size_t)pr * kSelCandCap,
+                                  &cand_count[pr])
+               : merge_row_kway(p, r, k, nc, firsts + (size_t)pr * nc);
     // insert the planted candidate into the sorted result
     if (pc >= 0) {
       const int ins = __popc(__ballot_sync(kFullMask, lane < k && res > plant_key));
@@ -205,67 +462,11 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
   __syncthreads();
   if (s_stop) return;
 
-  // ---- phase 3: synthetic draft step, one warp per new beam row:
-  //      h_child = round( u / sqrt(mean(u^2) + eps) ),  u = h_parent + E[token]
-  // The rounding to the storage type is a quantisation decision, so everything before it is
-  // done in fp64 and the result is rounded once, directly from fp64: an fp32 evaluation
-  // would flip about one element in 10^5 to the neighbouring bf16 value, and one such flip
-  // moves a logit by up to a few 1e-3.
-  if (warp < k) {
-    const int i = warp;
-    const int parent_slot = sel_flat[i] / k;
-    const int tok = sel_tok[i];
-    const size_t src_row = (size_t)(b * k + parent_slot) * p.Hd;
-    const size_t dst_row = (size_t)(b * k + i) * p.Hd;
-    const size_t e_row = (size_t)(tok >= 0 && tok < p.V ? tok : 0) * p.Hd;
-    if (p.dtype == DDD_DTYPE_BF16) {
-      const __nv_bfloat16* hp = static_cast<const __nv_bfloat16*>(p.hbuf[(d - 1) & 1]) + src_row;
-      const __nv_bfloat16* e = static_cast<const __nv_bfloat16*>(p.E) + e_row;
-      __nv_bfloat16* out = static_cast<__nv_bfloat16*>(p.hbuf[d & 1]) + dst_row;
-      double ss = 0.0;
-      for (int j = lane * 8; j < p.Hd; j += 256) {
-        const uint4 a = *reinterpret_cast<const uint4*>(hp + j);
-        const uint4 c = *reinterpret_cast<const uint4*>(e + j);
-        const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, cw[4] = {c.x, c.y, c.z, c.w};
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const double u0 = (double)__uint_as_float(aw[q] << 16) + (double)__uint_as_float(cw[q] << 16);
-          const double u1 = (double)__uint_as_float(aw[q] & 0xFFFF0000u) +
-                            (double)__uint_as_float(cw[q] & 0xFFFF0000u);
-          ss = fma(u0, u0, ss);
-          ss = fma(u1, u1, ss);
-        }
-      }
-      ss = warp_sum_f64(ss);
-      const double inv = 1.0 / sqrt(ss / (double)p.Hd + (double)p.eps);
-      for (int j = lane * 8; j < p.Hd; j += 256) {
-        const uint4 a = *reinterpret_cast<const uint4*>(hp + j);
-        const uint4 c = *reinterpret_cast<const uint4*>(e + j);
-        const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, cw[4] = {c.x, c.y, c.z, c.w};
-        uint32_t ow[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const double u0 = (double)__uint_as_float(aw[q] << 16) + (double)__uint_as_float(cw[q] << 16);
-          const double u1 = (double)__uint_as_float(aw[q] & 0xFFFF0000u) +
-                            (double)__uint_as_float(cw[q] & 0xFFFF0000u);
-          ow[q] = f64_to_bf16_bits(u0 * inv) | (f64_to_bf16_bits(u1 * inv) << 16);
-        }
-        *reinterpret_cast<uint4*>(out + j) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
-      }
-    } else {
-      const float* hp = static_cast<const float*>(p.hbuf[(d - 1) & 1]) + src_row;
-      const float* e = static_cast<const float*>(p.E) + e_row;
-      float* out = static_cast<float*>(p.hbuf[d & 1]) + dst_row;
-      double ss = 0.0;
-      for (int j = lane; j < p.Hd; j += 32) {
-        const double u = (double)hp[j] + (double)e[j];
-        ss = fma(u, u, ss);
-      }
-      ss = warp_sum_f64(ss);
-      const double inv = 1.0 / sqrt(ss / (double)p.Hd + (double)p.eps);
-      for (int j = lane; j < p.Hd; j += 32) out[j] = __double2float_rn(((double)hp[j] + (double)e[j]) * inv);
-    }
-  }
+  // ---- phase 3: synthetic draft step for the k new beam rows
+  if (p.dtype == DDD_DTYPE_BF16)
+    draft_step<__nv_bfloat16>(p, b, d, sel_flat, sel_tok, row_part, row_inv);
+  else
+    draft_step<float>(p, b, d, sel_flat, sel_tok, row_part, row_inv);
 }
 
 // ---------------------------------------------------------------------------- rerank + mask
@@ -433,7 +634,10 @@ __global__ void __launch_bounds__(kRerankThreads) rerank_mask_kernel(const Param
   }
 }
 
-size_t select_smem(const Params& p) { return (size_t)p.k * p.lm_ctas * sizeof(unsigned long long); }
+size_t select_smem(const Params& p) {
+  return (size_t)p.k * p.lm_ctas * (sizeof(unsigned long long) + sizeof(float2)) +
+         (p.k <= 16 ? (size_t)p.k * kSelCandCap * sizeof(unsigned long long) : 0);
+}
 size_t rerank_smem(const Params& p) { return (size_t)p.Nn * (sizeof(uint32_t) + sizeof(int)); }
 
 }  // namespace
