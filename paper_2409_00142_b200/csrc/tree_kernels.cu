@@ -1,12 +1,17 @@
 // Kernels around the LM head: draft initialisation, the per-pass select / gate / draft
 // step, and the final rerank with the bit-packed tree mask.  One thread block per sequence.
+#include <cooperative_groups.h>
+
 #include "ddd_common.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace ddd {
 
 namespace {
 
 constexpr int kSelThreads = 1024;
+constexpr int kSelCluster = 8;      // thread blocks (one cluster) working on one sequence
 constexpr int kRerankThreads = 1024;
 
 // ---------------------------------------------------------------------------- init
@@ -59,22 +64,20 @@ __device__ __forceinline__ uint32_t f64_to_bf16_bits(double y) {
 // Loads issued by one thread are batched (a few independent loads, then their use): a single
 // block runs this kernel between two LM-head passes, so its time is made of memory round
 // trips, and a loop that loads and uses one value per iteration pays one trip per iteration.
-constexpr int kSelCandCap = 256;   // candidates kept per row by the pruned merge (k <= 16: k*k)
-
-// Merge of one beam row's per-block partial lists, k <= 16.  first_s holds every block's best
-// key.  The k-th largest of those, T, is a lower bound of the row's k-th best key, and only
-// the k blocks whose best key reaches T can hold anything >= T: their lists are fetched, the
-// entries >= T (at most k*k, usually about 2k) are collected and the k best of them are the
-// answer.  Lane j returns the j-th best key (0 if there is none).
-__device__ __forceinline__ unsigned long long merge_row_pruned(const Params& p, int r, int k, int nc,
-                                                               const unsigned long long* first_s,
+// Merge of one beam row's per-block partial lists when all of them are in shared memory
+// (keys_s[c * k + q] = q-th best key of block c, descending, 0 = empty).  The k-th largest of
+// the blocks' best keys, T, is a lower bound of the row's k-th best key, and only the k blocks
+// whose best key reaches T can hold anything >= T: their entries >= T (at most k*k, usually
+// about 2k) are collected and the k best of them are the answer.  Lane j returns the j-th
+// best key (0 if there is none).
+__device__ __forceinline__ unsigned long long merge_row_pruned(int k, int nc, const unsigned long long* keys_s,
                                                                unsigned long long* cand_s, int* cand_n) {
   const int lane = threadIdx.x & 31;
   unsigned long long prev = ~0ull, T = 1ull;
   for (int j = 0; j < k; ++j) {
     unsigned long long best = 0ull;
     for (int c = lane; c < nc; c += 32) {
-      const unsigned long long key = first_s[c];
+      const unsigned long long key = keys_s[(size_t)c * k];
       if (key < prev && key > best) best = key;
     }
     const unsigned long long wk = warp_max_key(best);
@@ -84,21 +87,18 @@ __device__ __forceinline__ unsigned long long merge_row_pruned(const Params& p, 
   }
   if (lane == 0) *cand_n = 0;
   __syncwarp();
+  const int cap = k * k;
   for (int c = lane; c < nc; c += 32) {
-    if (first_s[c] < T) continue;
-    const unsigned long long* list = p.part_key + ((size_t)c * p.R + r) * k;
-    unsigned long long e[16];
-#pragma unroll
-    for (int q = 0; q < 16; ++q) e[q] = q < k ? list[q] : 0ull;
-#pragma unroll
-    for (int q = 0; q < 16; ++q)
-      if (e[q] >= T) {
-        const int pos = atomicAdd(cand_n, 1);
-        if (pos < kSelCandCap) cand_s[pos] = e[q];
-      }
+    const unsigned long long* list = keys_s + (size_t)c * k;
+    for (int q = 0; q < k; ++q) {
+      const unsigned long long key = list[q];
+      if (key < T) break;                      // lists are sorted: nothing further qualifies
+      const int pos = atomicAdd(cand_n, 1);
+      if (pos < cap) cand_s[pos] = key;
+    }
   }
   __syncwarp();
-  const int C = min(*cand_n, kSelCandCap);
+  const int C = min(*cand_n, cap);
   unsigned long long res = 0ull;
   prev = ~0ull;
   for (int j = 0; j < k; ++j) {
@@ -115,8 +115,9 @@ __device__ __forceinline__ unsigned long long merge_row_pruned(const Params& p, 
   return res;
 }
 
-// Same result for any k: pick the k blocks with the best first keys, then walk their sorted
-// lists in a k-way merge straight from global memory (lane j owns one list).
+// Same result when the lists do not fit in shared memory: pick the k blocks with the best
+// first keys, then walk their sorted lists in a k-way merge straight from global memory
+// (lane j owns one list).
 __device__ __forceinline__ unsigned long long merge_row_kway(const Params& p, int r, int k, int nc,
                                                              const unsigned long long* first_s) {
   const int lane = threadIdx.x & 31;
@@ -191,23 +192,27 @@ struct Chunk<float> {
   }
 };
 
-// Synthetic draft step for the k new beam rows of one sequence, by the whole block:
+// Synthetic draft step for the k new beam rows of one sequence, by all blocks of the cluster:
 //   h_child = round( u / sqrt(mean(u^2) + eps) ),  u = h_parent + E[token]
 // The rounding to the storage type is a quantisation decision, so everything before it is done
 // in fp64 and the result is rounded once, directly from fp64: an fp32 evaluation would flip
 // about one element in 10^5 to the neighbouring bf16 value, and one such flip moves a logit by
-// up to a few 1e-3.  Work is cut into 16-byte chunks; a warp's 32 chunks lie in one row
-// (the caller checks that a row has a multiple of 32 chunks), and per-row sums are combined
-// in a fixed order.
+// up to a few 1e-3.  Work is cut into 16-byte chunks dealt round-robin to the cluster's
+// threads; a warp's 32 chunks lie in one row (the caller checks that a row has a multiple of
+// 32 chunks).  Every warp sends its partial sum of squares to all blocks through distributed
+// shared memory, and each block adds a row's partials in the same fixed order.
 template <typename T>
-__device__ void draft_step_block(const Params& p, int b, int d, const int* sel_flat, const int* sel_tok,
-                                 double* row_part /* [k][slots] */, double* row_inv /* [k] */) {
+__device__ void draft_step_cluster(const Params& p, int b, int d, const int* sel_flat, const int* sel_tok,
+                                   double* row_part /* [k][slots] */, double* row_inv /* [k] */) {
+  cg::cluster_group cluster = cg::this_cluster();
   constexpr int N = Chunk<T>::N;
   constexpr int kBatch = 4;
   const int k = p.k, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int cpr = p.Hd / N;            // chunks per row
   const int slots = cpr / 32;          // warp-sized groups of chunks per row
   const int total = k * cpr;
+  const int first = (int)cluster.block_rank() * (int)blockDim.x + (int)threadIdx.x;
+  const int stride = kSelCluster * (int)blockDim.x;
   const uint4* Hsrc = reinterpret_cast<const uint4*>(p.hbuf[(d - 1) & 1]);
   const uint4* Esrc = reinterpret_cast<const uint4*>(p.E);
   uint4* Hdst = reinterpret_cast<uint4*>(p.hbuf[d & 1]);
@@ -220,39 +225,35 @@ __device__ void draft_step_block(const Params& p, int b, int d, const int* sel_f
     hd = (size_t)(b * k + row) * cpr + col;
   };
   // pass 1: sum of squares per row
-  for (int q0 = threadIdx.x; q0 < total; q0 += kBatch * blockDim.x) {
+  for (int q0 = first; q0 - lane < total; q0 += kBatch * stride) {
     uint4 hv[kBatch], ev[kBatch];
-    int rows[kBatch];
 #pragma unroll
     for (int i = 0; i < kBatch; ++i) {
-      const int q = q0 + i * blockDim.x;
-      rows[i] = -1;
+      const int q = q0 + i * stride;
       if (q < total) {
         size_t hs, es, hd;
-        locate(q, hs, es, hd, rows[i]);
+        int row;
+        locate(q, hs, es, hd, row);
         hv[i] = Hsrc[hs];
         ev[i] = Esrc[es];
       }
     }
 #pragma unroll
     for (int i = 0; i < kBatch; ++i) {
-      const int q = q0 + i * blockDim.x;
-      if (q0 - lane + i * (int)blockDim.x >= total) continue;   // whole warp past the end (uniform)
+      const int q = q0 + i * stride;
+      if (q - lane >= total) continue;          // whole warp past the end (total is a multiple of 32)
+      double u[N];
+      Chunk<T>::sum(hv[i], ev[i], u);
       double ss = 0.0;
-      if (rows[i] >= 0) {
-        double u[N];
-        Chunk<T>::sum(hv[i], ev[i], u);
 #pragma unroll
-        for (int e = 0; e < N; ++e) ss = fma(u[e], u[e], ss);
-      }
+      for (int e = 0; e < N; ++e) ss = fma(u[e], u[e], ss);
       ss = warp_sum_f64(ss);
-      if (lane == 0) {
-        const int row = q / cpr;
-        row_part[row * slots + (q - row * cpr) / 32] = ss;
-      }
+      const int row = q / cpr;
+      const int slot = row * slots + (q - row * cpr) / 32;
+      if (lane < kSelCluster) cluster.map_shared_rank(row_part, lane)[slot] = ss;
     }
   }
-  __syncthreads();
+  cluster.sync();
   if (warp < k && lane == 0) {
     double ss = 0.0;
     for (int j = 0; j < slots; ++j) ss += row_part[warp * slots + j];
@@ -260,13 +261,13 @@ __device__ void draft_step_block(const Params& p, int b, int d, const int* sel_f
   }
   __syncthreads();
   // pass 2: scale, round once, store (the inputs come back from the L1 / L2 caches)
-  for (int q0 = threadIdx.x; q0 < total; q0 += kBatch * blockDim.x) {
+  for (int q0 = first; q0 - lane < total; q0 += kBatch * stride) {
     uint4 hv[kBatch], ev[kBatch];
     size_t dst[kBatch];
     int rows[kBatch];
 #pragma unroll
     for (int i = 0; i < kBatch; ++i) {
-      const int q = q0 + i * blockDim.x;
+      const int q = q0 + i * stride;
       rows[i] = -1;
       if (q < total) {
         size_t hs, es;
@@ -288,8 +289,8 @@ __device__ void draft_step_block(const Params& p, int b, int d, const int* sel_f
   }
 }
 
-// The same step with one warp per row, for hidden sizes whose rows are not a whole number of
-// 32-chunk groups.
+// The same step with one warp per row (run by one block), for hidden sizes whose rows are not
+// a whole number of 32-chunk groups.
 template <typename T>
 __device__ void draft_step_warp(const Params& p, int b, int d, const int* sel_flat, const int* sel_tok) {
   constexpr int N = Chunk<T>::N;
@@ -318,55 +319,70 @@ __device__ void draft_step_warp(const Params& p, int b, int d, const int* sel_fl
   }
 }
 
+// Called by every block of the cluster (the choice below is the same in all of them).
 template <typename T>
 __device__ void draft_step(const Params& p, int b, int d, const int* sel_flat, const int* sel_tok, double* row_part,
                            double* row_inv) {
   const int cpr = p.Hd / Chunk<T>::N;
   if (cpr % 32 == 0 && cpr / 32 <= 64)
-    draft_step_block<T>(p, b, d, sel_flat, sel_tok, row_part, row_inv);
-  else
+    draft_step_cluster<T>(p, b, d, sel_flat, sel_tok, row_part, row_inv);
+  else if (cg::this_cluster().block_rank() == 0)
     draft_step_warp<T>(p, b, d, sel_flat, sel_tok);
 }
 
-// Dynamic shared memory: per beam row of this sequence, every LM-head block's best key and
-// its (max, sum-exp); then the candidate lists of the pruned merge.
+// One cluster of kSelCluster blocks per sequence.  Beam row pr is merged by block pr % 8
+// (warp pr / 8), which first copies that row's partial lists into its shared memory; the
+// candidates go to block 0 through distributed shared memory, block 0 picks the new beam and
+// takes the stop decision, and all blocks share the draft step.
+// Dynamic shared memory per block, for its rows_max = ceil(k / 8) rows: the blocks' key lists
+// [rows_max][nc][k] (or only their first keys [rows_max][nc] when the lists do not fit),
+// their (max, sum-exp) [rows_max][nc], and the candidate lists [rows_max][k*k].
 __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Params p, const DraftIO io,
-                                                                       const int d) {
-  const int b = blockIdx.x;
-  if (p.active[b] == 0) return;
+                                                                       const int d, const int lists_in_smem) {
+  cg::cluster_group cluster = cg::this_cluster();
+  const int crank = (int)cluster.block_rank();
+  const int b = blockIdx.x / kSelCluster;
+  if (p.active[b] == 0) return;                               // same decision in the whole cluster
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int k = p.k, nc = p.lm_ctas, R = p.R;
   const int P = (d == 1) ? 1 : k;                            // beam rows of this sequence in pass d
   const int base = (d == 1) ? 1 : 1 + k + (d - 2) * k * k;   // node id of candidate (0, 0)
-  const bool pruned = k <= 16;
+  const int rows_max = (k + kSelCluster - 1) / kSelCluster;
+  const int n_mine = P > crank ? (P - crank + kSelCluster - 1) / kSelCluster : 0;   // rows of this block
+  const int kl = lists_in_smem ? k : 1;                       // keys kept per (row, LM-head block)
 
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  unsigned long long* firsts = reinterpret_cast<unsigned long long*>(smem_raw);                // [k][nc]
-  float2* ms_s = reinterpret_cast<float2*>(firsts + (size_t)k * nc);                            // [k][nc]
-  unsigned long long* cand_list = reinterpret_cast<unsigned long long*>(ms_s + (size_t)k * nc);  // [k][cap]
-  __shared__ unsigned long long cand_key[DDD_MAX_K * DDD_MAX_K];
-  __shared__ float cand_val[DDD_MAX_K * DDD_MAX_K];
-  __shared__ int cand_tok[DDD_MAX_K * DDD_MAX_K];
+  unsigned long long* keys_s = reinterpret_cast<unsigned long long*>(smem_raw);              // [rows_max][nc][kl]
+  float2* ms_s = reinterpret_cast<float2*>(keys_s + (size_t)rows_max * nc * kl);              // [rows_max][nc]
+  unsigned long long* cand_list = reinterpret_cast<unsigned long long*>(ms_s + (size_t)rows_max * nc);
+  __shared__ unsigned long long cand_key[DDD_MAX_K * DDD_MAX_K];   // used in block 0
+  __shared__ float cand_val[DDD_MAX_K * DDD_MAX_K];                // used in block 0
+  __shared__ int cand_tok[DDD_MAX_K * DDD_MAX_K];                  // used in block 0
   __shared__ int sel_flat[DDD_MAX_K];
   __shared__ int sel_tok[DDD_MAX_K];
-  __shared__ int cand_count[DDD_MAX_K];
+  __shared__ int cand_count[DDD_MAX_K / kSelCluster];
   __shared__ double row_part[DDD_MAX_K * 64];
   __shared__ double row_inv[DDD_MAX_K];
   __shared__ int s_stop;
 
-  // ---- phase 0: the whole block fetches what phase 1 needs in one round trip
-  for (int i = threadIdx.x; i < P * nc; i += blockDim.x) {
-    const int pr = i / nc, c = i - pr * nc;
-    const size_t slot = (size_t)c * R + (b * k + pr);
-    firsts[pr * nc + c] = p.part_key[slot * k];
-    ms_s[pr * nc + c] = p.part_ms[slot];
+  // ---- phase 0: the block fetches everything phase 1 needs for its rows in one round trip
+  for (int i = threadIdx.x; i < n_mine * nc * kl; i += blockDim.x) {
+    const int j = i / (nc * kl), rem = i - j * nc * kl, c = rem / kl, q = rem - c * kl;
+    const int r = b * k + crank + kSelCluster * j;
+    keys_s[i] = p.part_key[((size_t)c * R + r) * k + q];
+  }
+  for (int i = threadIdx.x; i < n_mine * nc; i += blockDim.x) {
+    const int j = i / nc, c = i - j * nc;
+    const int r = b * k + crank + kSelCluster * j;
+    ms_s[i] = p.part_ms[(size_t)c * R + r];
   }
   __syncthreads();
 
   // ---- phase 1: one warp per beam row merges the per-block partials of the LM-head pass
-  if (warp < P) {
-    const int pr = warp, r = b * k + pr;
-    const float2* my_ms = ms_s + (size_t)pr * nc;
+  if (warp < n_mine) {
+    const int pr = crank + kSelCluster * warp, r = b * k + pr;
+    const float2* my_ms = ms_s + (size_t)warp * nc;
+    const unsigned long long* my_keys = keys_s + (size_t)warp * nc * kl;
     // log-sum-exp over all blocks (fixed lane-strided order, then a butterfly: deterministic)
     float M = neg_inf();
     for (int c = lane; c < nc; c += 32) M = fmaxf(M, my_ms[c].x);
@@ -389,10 +405,9 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
     }
     const float lse = M + logf(S);
 
-    unsigned long long res =
-        pruned ? merge_row_pruned(p, r, k, nc, firsts + (size_t)pr * nc, cand_list + (size_t)pr * kSelCandCap,
-                                  &cand_count[pr])
-               : merge_row_kway(p, r, k, nc, firsts + (size_t)pr * nc);
+    unsigned long long res = lists_in_smem
+                                 ? merge_row_pruned(k, nc, my_keys, cand_list + (size_t)warp * k * k, &cand_count[warp])
+                                 : merge_row_kway(p, r, k, nc, my_keys);
     // insert the planted candidate into the sorted result
     if (pc >= 0) {
       const int ins = __popc(__ballot_sync(kFullMask, lane < k && res > plant_key));
@@ -409,16 +424,17 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
       p.tree_token[node] = tok;
       p.tree_parent[node] = p.beam_node[b * k + pr];
       p.tree_cum[node] = cand;
-      cand_key[flat] = (res != 0ull) ? make_key(cand, (uint32_t)flat) : 0ull;
-      cand_val[flat] = cand;
-      cand_tok[flat] = tok;
+      // the candidates of all rows meet in block 0
+      cluster.map_shared_rank(cand_key, 0)[flat] = (res != 0ull) ? make_key(cand, (uint32_t)flat) : 0ull;
+      cluster.map_shared_rank(cand_val, 0)[flat] = cand;
+      cluster.map_shared_rank(cand_tok, 0)[flat] = tok;
     }
     if (lane == 0 && io.trace.row_lse) io.trace.row_lse[((size_t)b * p.n + (d - 1)) * k + pr] = lse;
   }
-  __syncthreads();
+  cluster.sync();
 
-  // ---- phase 2: warp 0 picks the new beam, evaluates Eq. 1 and takes the stop decision
-  if (warp == 0) {
+  // ---- phase 2: warp 0 of block 0 picks the new beam, evaluates Eq. 1 and takes the stop decision
+  if (crank == 0 && warp == 0) {
     const int n_cand = P * k;
     unsigned long long prev = ~0ull, mine = 0ull;
     for (int j = 0; j < k; ++j) {
@@ -439,10 +455,16 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
     const float H = M + logf(sum);
     bool stop = (d == p.n);
     if (!stop && ((p.check_mask >> (d - 1)) & 1u)) stop = H < p.x;
+    const int tok = lane < k ? cand_tok[flat] : -1;
+    // every block needs the selection and the decision for the draft step
+    for (int rk = 0; rk < kSelCluster; ++rk) {
+      if (lane < k) {
+        cluster.map_shared_rank(sel_flat, rk)[lane] = flat;
+        cluster.map_shared_rank(sel_tok, rk)[lane] = tok;
+      }
+      if (lane == 0) *cluster.map_shared_rank(&s_stop, rk) = stop ? 1 : 0;
+    }
     if (lane < k) {
-      const int tok = cand_tok[flat];
-      sel_flat[lane] = flat;
-      sel_tok[lane] = tok;
       p.beam_node[b * k + lane] = base + flat;
       p.beam_tok[b * k + lane] = tok;
       p.beam_cum[b * k + lane] = cum;
@@ -451,7 +473,6 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
     }
     if (lane == 0) {
       io.out.H_trace[(size_t)b * p.n + (d - 1)] = H;
-      s_stop = stop ? 1 : 0;
       if (stop) {
         p.stop_depth[b] = d;
         p.active[b] = 0;
@@ -459,8 +480,8 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
       }
     }
   }
-  __syncthreads();
-  if (s_stop) return;
+  cluster.sync();
+  if (s_stop) return;       // no block touches another block's shared memory after this point
 
   // ---- phase 3: synthetic draft step for the k new beam rows
   if (p.dtype == DDD_DTYPE_BF16)
@@ -634,10 +655,16 @@ __global__ void __launch_bounds__(kRerankThreads) rerank_mask_kernel(const Param
   }
 }
 
-size_t select_smem(const Params& p) {
-  return (size_t)p.k * p.lm_ctas * (sizeof(unsigned long long) + sizeof(float2)) +
-         (p.k <= 16 ? (size_t)p.k * kSelCandCap * sizeof(unsigned long long) : 0);
+// Can the partial lists of a block's rows live in its shared memory?  (Host and device agree
+// through the kernel argument.)
+size_t select_smem_bytes(const Params& p, bool lists) {
+  const size_t rows_max = (p.k + kSelCluster - 1) / kSelCluster;
+  const size_t kl = lists ? p.k : 1;
+  return rows_max * p.lm_ctas * (kl * sizeof(unsigned long long) + sizeof(float2)) +
+         rows_max * (size_t)p.k * p.k * sizeof(unsigned long long);
 }
+bool select_lists_in_smem(const Params& p) { return select_smem_bytes(p, true) <= 160 * 1024; }
+size_t select_smem(const Params& p) { return select_smem_bytes(p, select_lists_in_smem(p)); }
 size_t rerank_smem(const Params& p) { return (size_t)p.Nn * (sizeof(uint32_t) + sizeof(int)); }
 
 }  // namespace
@@ -662,8 +689,19 @@ cudaError_t launch_init(const Params& p, const DraftIO&, const void* root_hidden
 }
 
 cudaError_t launch_select(const Params& p, const DraftIO& io, int d, cudaStream_t st) {
-  select_gate_step_kernel<<<p.B, kSelThreads, select_smem(p), st>>>(p, io, d);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(p.B * kSelCluster), 1, 1);
+  cfg.blockDim = dim3(kSelThreads, 1, 1);
+  cfg.dynamicSmemBytes = select_smem(p);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = kSelCluster;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, select_gate_step_kernel, p, io, d, select_lists_in_smem(p) ? 1 : 0);
 }
 
 cudaError_t launch_rerank(const Params& p, const DraftIO& io, cudaStream_t st) {
