@@ -33,6 +33,10 @@ METRIC = "drafts_per_sec"
 UNIT = "drafts/s"
 NEG = -1e30
 FALLBACK_HBM_GBS = 6650.0
+# DRAM bytes (read + write) of one LM-head launch from the ncu capture summarised under
+# profiles/, valid only while the kernel source is the one that was profiled.
+NCU_TRAFFIC = {"llama2_7b": {"bytes": 266.0e6, "source_sha256_16": "6c75161731a55103",
+                             "profile": "profiles/lm_head_tc_llama2_7b.md"}}
 CLOCK_QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
                "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
                "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
@@ -52,6 +56,21 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true")
     return ap.parse_args()
+
+
+def ncu_traffic(workload: str):
+    import hashlib
+    ent = NCU_TRAFFIC.get(workload)
+    if not ent:
+        return None
+    src = os.path.join(ROOT, "paper_2409_00142_b200", "csrc", "lm_head_tc.cu")
+    try:
+        with open(src, "rb") as f:
+            if hashlib.sha256(f.read()).hexdigest()[:16] != ent["source_sha256_16"]:
+                return None          # kernel changed since the counters were taken
+    except OSError:
+        return None
+    return ent["bytes"]
 
 
 def measured_peak():
@@ -336,18 +355,21 @@ def main():
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": launches,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak, "traffic": None, "peak_kind": f"of {peak_kind}",
+                     "frac": achieved / peak, "traffic": ncu_traffic(cfg.name), "peak_kind": f"of {peak_kind}",
                      "kernel": "lm_head", "us_per_launch": lm_us, "algorithmic_bytes_per_launch": w_bytes,
                      "frac_of_8TBs_nominal": achieved / 8000.0, "blocks": blocks},
     }
     line.update(extra)
     if not args.no_cpu_baseline and world == 1:
         from oracle import ddd_oracle as O
-        sample = args.cpu_sample or 2
-        t0 = time.perf_counter()
-        for i in range(sample):
-            O.draft(cfg, weights, **roots_host[i % len(roots_host)])
-        dt = time.perf_counter() - t0
+        # a bounded sample of the same workload: drafts until about 12 s of CPU work (or --cpu-sample drafts)
+        sample, t0 = 0, time.perf_counter()
+        while True:
+            O.draft(cfg, weights, **roots_host[sample % len(roots_host)])
+            sample += 1
+            dt = time.perf_counter() - t0
+            if (args.cpu_sample and sample >= args.cpu_sample) or (not args.cpu_sample and (dt > 12.0 or sample >= 400)):
+                break
         line["cpu_baseline"] = {"value": sample * cfg.batch / dt, "unit": UNIT, "cores": O.num_threads(),
                                 "kind": "oracle",
                                 "sample": f"{sample} draft(s) of {cfg.name}, x={cfg.threshold}, {dt:.1f} s"}
