@@ -65,52 +65,38 @@ __device__ __forceinline__ uint32_t f64_to_bf16_bits(double y) {
 // block runs this kernel between two LM-head passes, so its time is made of memory round
 // trips, and a loop that loads and uses one value per iteration pays one trip per iteration.
 // Merge of one beam row's per-block partial lists when all of them are in shared memory
-// (keys_s[c * k + q] = q-th best key of block c, descending, 0 = empty).  The k-th largest of
-// the blocks' best keys, T, is a lower bound of the row's k-th best key, and only the k blocks
-// whose best key reaches T can hold anything >= T: their entries >= T (at most k*k, usually
-// about 2k) are collected and the k best of them are the answer.  Lane j returns the j-th
-// best key (0 if there is none).
-__device__ __forceinline__ unsigned long long merge_row_pruned(int k, int nc, const unsigned long long* keys_s,
-                                                               unsigned long long* cand_s, int* cand_n) {
+// (keys_s[c * k + q] = q-th best key of block c, descending, 0 = empty): a k-way merge in
+// which every lane keeps the heads of its NL lists (blocks lane, lane + 32, ...) in registers.
+// One round = best head of the lane, maximum over the warp, the owning lane steps that list.
+// Lane j returns the j-th best key (0 if there is none).
+template <int NL>
+__device__ __forceinline__ unsigned long long merge_row_heads(int k, int nc, const unsigned long long* keys_s) {
   const int lane = threadIdx.x & 31;
-  unsigned long long prev = ~0ull, T = 1ull;
-  for (int j = 0; j < k; ++j) {
-    unsigned long long best = 0ull;
-    for (int c = lane; c < nc; c += 32) {
-      const unsigned long long key = keys_s[(size_t)c * k];
-      if (key < prev && key > best) best = key;
-    }
-    const unsigned long long wk = warp_max_key(best);
-    if (wk == 0ull) { T = 1ull; break; }      // fewer than k blocks have anything: keep all
-    prev = wk;
-    T = wk;
+  unsigned long long head[NL];
+  int pos[NL];
+#pragma unroll
+  for (int i = 0; i < NL; ++i) {
+    const int c = lane + 32 * i;
+    head[i] = c < nc ? keys_s[(size_t)c * k] : 0ull;
+    pos[i] = 0;
   }
-  if (lane == 0) *cand_n = 0;
-  __syncwarp();
-  const int cap = k * k;
-  for (int c = lane; c < nc; c += 32) {
-    const unsigned long long* list = keys_s + (size_t)c * k;
-    for (int q = 0; q < k; ++q) {
-      const unsigned long long key = list[q];
-      if (key < T) break;                      // lists are sorted: nothing further qualifies
-      const int pos = atomicAdd(cand_n, 1);
-      if (pos < cap) cand_s[pos] = key;
-    }
-  }
-  __syncwarp();
-  const int C = min(*cand_n, cap);
   unsigned long long res = 0ull;
-  prev = ~0ull;
   for (int j = 0; j < k; ++j) {
-    unsigned long long best = 0ull;
-    for (int c = lane; c < C; c += 32) {
-      const unsigned long long key = cand_s[c];
-      if (key < prev && key > best) best = key;
-    }
+    unsigned long long best = head[0];
+#pragma unroll
+    for (int i = 1; i < NL; ++i) best = head[i] > best ? head[i] : best;
     const unsigned long long wk = warp_max_key(best);
     if (wk == 0ull) break;
     if (lane == j) res = wk;
-    prev = wk;
+    if (best == wk) {                      // keys are unique: one lane, one list
+#pragma unroll
+      for (int i = 0; i < NL; ++i) {
+        if (head[i] == wk) {
+          ++pos[i];
+          head[i] = pos[i] < k ? keys_s[(size_t)(lane + 32 * i) * k + pos[i]] : 0ull;
+        }
+      }
+    }
   }
   return res;
 }
@@ -336,7 +322,7 @@ __device__ void draft_step(const Params& p, int b, int d, const int* sel_flat, c
 // takes the stop decision, and all blocks share the draft step.
 // Dynamic shared memory per block, for its rows_max = ceil(k / 8) rows: the blocks' key lists
 // [rows_max][nc][k] (or only their first keys [rows_max][nc] when the lists do not fit),
-// their (max, sum-exp) [rows_max][nc], and the candidate lists [rows_max][k*k].
+// their (max, sum-exp) [rows_max][nc], and the rows' planted columns [rows_max].
 __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Params p, const DraftIO io,
                                                                        const int d, const int lists_in_smem) {
   cg::cluster_group cluster = cg::this_cluster();
@@ -354,27 +340,26 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
   extern __shared__ __align__(16) unsigned char smem_raw[];
   unsigned long long* keys_s = reinterpret_cast<unsigned long long*>(smem_raw);              // [rows_max][nc][kl]
   float2* ms_s = reinterpret_cast<float2*>(keys_s + (size_t)rows_max * nc * kl);              // [rows_max][nc]
-  unsigned long long* cand_list = reinterpret_cast<unsigned long long*>(ms_s + (size_t)rows_max * nc);
+  int* plant_s = reinterpret_cast<int*>(ms_s + (size_t)rows_max * nc);                        // [rows_max]
   __shared__ unsigned long long cand_key[DDD_MAX_K * DDD_MAX_K];   // used in block 0
   __shared__ float cand_val[DDD_MAX_K * DDD_MAX_K];                // used in block 0
   __shared__ int cand_tok[DDD_MAX_K * DDD_MAX_K];                  // used in block 0
   __shared__ int sel_flat[DDD_MAX_K];
   __shared__ int sel_tok[DDD_MAX_K];
-  __shared__ int cand_count[DDD_MAX_K / kSelCluster];
   __shared__ double row_part[DDD_MAX_K * 64];
   __shared__ double row_inv[DDD_MAX_K];
   __shared__ int s_stop;
 
   // ---- phase 0: the block fetches everything phase 1 needs for its rows in one round trip
-  for (int i = threadIdx.x; i < n_mine * nc * kl; i += blockDim.x) {
-    const int j = i / (nc * kl), rem = i - j * nc * kl, c = rem / kl, q = rem - c * kl;
+  // (a warp copies one LM-head block's list per step: lane q takes the q-th key)
+  for (int j = 0; j < n_mine; ++j) {
     const int r = b * k + crank + kSelCluster * j;
-    keys_s[i] = p.part_key[((size_t)c * R + r) * k + q];
-  }
-  for (int i = threadIdx.x; i < n_mine * nc; i += blockDim.x) {
-    const int j = i / nc, c = i - j * nc;
-    const int r = b * k + crank + kSelCluster * j;
-    ms_s[i] = p.part_ms[(size_t)c * R + r];
+    for (int c = warp; c < nc; c += kSelThreads / 32) {
+      const size_t slot = (size_t)c * R + r;
+      if (lane < kl) keys_s[((size_t)j * nc + c) * kl + lane] = p.part_key[slot * k + lane];
+      if (lane == 31) ms_s[(size_t)j * nc + c] = p.part_ms[slot];
+    }
+    if (threadIdx.x == 0) plant_s[j] = p.row_plant[r];
   }
   __syncthreads();
 
@@ -394,7 +379,7 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
     }
     S = warp_sum(S);
     // planted column: its logit is (max of the others) + delta and it was left out of the partials
-    const int pc = p.row_plant[r];
+    const int pc = plant_s[warp];
     unsigned long long plant_key = 0ull;
     if (pc >= 0) {
       const float zc = M + p.plant_delta;
@@ -405,9 +390,10 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
     }
     const float lse = M + logf(S);
 
-    unsigned long long res = lists_in_smem
-                                 ? merge_row_pruned(k, nc, my_keys, cand_list + (size_t)warp * k * k, &cand_count[warp])
-                                 : merge_row_kway(p, r, k, nc, my_keys);
+    unsigned long long res;
+    if (!lists_in_smem) res = merge_row_kway(p, r, k, nc, my_keys);
+    else if (nc <= 160) res = merge_row_heads<5>(k, nc, my_keys);
+    else res = merge_row_heads<16>(k, nc, my_keys);
     // insert the planted candidate into the sorted result
     if (pc >= 0) {
       const int ins = __popc(__ballot_sync(kFullMask, lane < k && res > plant_key));
@@ -434,53 +420,77 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
   cluster.sync();
 
   // ---- phase 2: warp 0 of block 0 picks the new beam, evaluates Eq. 1 and takes the stop decision
+  int bk_flat = 0, bk_tok = -1;     // kept by warp 0 of block 0 for the bookkeeping after the barrier
+  float bk_cum = 0.f, bk_H = 0.f;
+  bool bk_stop = false;
   if (crank == 0 && warp == 0) {
     const int n_cand = P * k;
-    unsigned long long prev = ~0ull, mine = 0ull;
-    for (int j = 0; j < k; ++j) {
-      unsigned long long best = 0ull;
-      for (int c = lane; c < n_cand; c += 32) {
-        const unsigned long long key = cand_key[c];
-        if (key < prev && key > best) best = key;
+    unsigned long long mine = 0ull;
+    if (n_cand <= 128) {
+      unsigned long long ck[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) ck[i] = lane + 32 * i < n_cand ? cand_key[lane + 32 * i] : 0ull;
+      for (int j = 0; j < k; ++j) {
+        unsigned long long best = ck[0];
+#pragma unroll
+        for (int i = 1; i < 4; ++i) best = ck[i] > best ? ck[i] : best;
+        const unsigned long long wk = warp_max_key(best);
+        if (lane == j) mine = wk;
+        if (wk == 0ull) break;
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          if (ck[i] == wk) ck[i] = 0ull;
       }
-      const unsigned long long wk = warp_max_key(best);
-      if (lane == j) mine = wk;
-      prev = wk;
+    } else {
+      unsigned long long prev = ~0ull;
+      for (int j = 0; j < k; ++j) {
+        unsigned long long best = 0ull;
+        for (int c = lane; c < n_cand; c += 32) {
+          const unsigned long long key = cand_key[c];
+          if (key < prev && key > best) best = key;
+        }
+        const unsigned long long wk = warp_max_key(best);
+        if (lane == j) mine = wk;
+        prev = wk;
+      }
     }
     const bool have = lane < k && mine != 0ull;
-    const int flat = have ? (int)key_index(mine) : 0;
-    const float cum = have ? cand_val[flat] : neg_inf();
-    const float M = __shfl_sync(kFullMask, cum, 0);           // sorted descending: entry 0 is the max
-    const float sum = warp_sum(have ? expf(cum - M) : 0.f);
-    const float H = M + logf(sum);
-    bool stop = (d == p.n);
-    if (!stop && ((p.check_mask >> (d - 1)) & 1u)) stop = H < p.x;
-    const int tok = lane < k ? cand_tok[flat] : -1;
+    bk_flat = have ? (int)key_index(mine) : 0;
+    bk_cum = have ? cand_val[bk_flat] : neg_inf();
+    const float M = __shfl_sync(kFullMask, bk_cum, 0);        // sorted descending: entry 0 is the max
+    const float sum = warp_sum(have ? expf(bk_cum - M) : 0.f);
+    bk_H = M + logf(sum);
+    bk_stop = (d == p.n);
+    if (!bk_stop && ((p.check_mask >> (d - 1)) & 1u)) bk_stop = bk_H < p.x;
+    bk_tok = lane < k ? cand_tok[bk_flat] : -1;
     // every block needs the selection and the decision for the draft step
     for (int rk = 0; rk < kSelCluster; ++rk) {
       if (lane < k) {
-        cluster.map_shared_rank(sel_flat, rk)[lane] = flat;
-        cluster.map_shared_rank(sel_tok, rk)[lane] = tok;
+        cluster.map_shared_rank(sel_flat, rk)[lane] = bk_flat;
+        cluster.map_shared_rank(sel_tok, rk)[lane] = bk_tok;
       }
-      if (lane == 0) *cluster.map_shared_rank(&s_stop, rk) = stop ? 1 : 0;
+      if (lane == 0) *cluster.map_shared_rank(&s_stop, rk) = bk_stop ? 1 : 0;
     }
+  }
+  cluster.sync();
+  // the bookkeeping in global memory is off the other warps' critical path
+  if (crank == 0 && warp == 0) {
     if (lane < k) {
-      p.beam_node[b * k + lane] = base + flat;
-      p.beam_tok[b * k + lane] = tok;
-      p.beam_cum[b * k + lane] = cum;
-      p.row_plant[b * k + lane] = (p.plant_next && tok >= 0 && tok < p.V) ? p.plant_next[tok] : -1;
-      if (io.trace.beam_sel) io.trace.beam_sel[((size_t)b * p.n + (d - 1)) * k + lane] = flat;
+      p.beam_node[b * k + lane] = base + bk_flat;
+      p.beam_tok[b * k + lane] = bk_tok;
+      p.beam_cum[b * k + lane] = bk_cum;
+      p.row_plant[b * k + lane] = (p.plant_next && bk_tok >= 0 && bk_tok < p.V) ? p.plant_next[bk_tok] : -1;
+      if (io.trace.beam_sel) io.trace.beam_sel[((size_t)b * p.n + (d - 1)) * k + lane] = bk_flat;
     }
     if (lane == 0) {
-      io.out.H_trace[(size_t)b * p.n + (d - 1)] = H;
-      if (stop) {
+      io.out.H_trace[(size_t)b * p.n + (d - 1)] = bk_H;
+      if (bk_stop) {
         p.stop_depth[b] = d;
         p.active[b] = 0;
         atomicSub(p.n_active, 1);
       }
     }
   }
-  cluster.sync();
   if (s_stop) return;       // no block touches another block's shared memory after this point
 
   // ---- phase 3: synthetic draft step for the k new beam rows
@@ -660,8 +670,7 @@ __global__ void __launch_bounds__(kRerankThreads) rerank_mask_kernel(const Param
 size_t select_smem_bytes(const Params& p, bool lists) {
   const size_t rows_max = (p.k + kSelCluster - 1) / kSelCluster;
   const size_t kl = lists ? p.k : 1;
-  return rows_max * p.lm_ctas * (kl * sizeof(unsigned long long) + sizeof(float2)) +
-         rows_max * (size_t)p.k * p.k * sizeof(unsigned long long);
+  return rows_max * p.lm_ctas * (kl * sizeof(unsigned long long) + sizeof(float2)) + rows_max * sizeof(int);
 }
 bool select_lists_in_smem(const Params& p) { return select_smem_bytes(p, true) <= 160 * 1024; }
 size_t select_smem(const Params& p) { return select_smem_bytes(p, select_lists_in_smem(p)); }
