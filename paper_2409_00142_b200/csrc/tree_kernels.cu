@@ -393,7 +393,7 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
     unsigned long long res;
     if (!lists_in_smem) res = merge_row_kway(p, r, k, nc, my_keys);
     else if (nc <= 160) res = merge_row_heads<5>(k, nc, my_keys);
-    else res = merge_row_heads<16>(k, nc, my_keys);
+    else res = merge_row_heads<10>(k, nc, my_keys);      // the host keeps nc <= 320 on this path
     // insert the planted candidate into the sorted result
     if (pc >= 0) {
       const int ins = __popc(__ballot_sync(kFullMask, lane < k && res > plant_key));
@@ -672,7 +672,9 @@ size_t select_smem_bytes(const Params& p, bool lists) {
   const size_t kl = lists ? p.k : 1;
   return rows_max * p.lm_ctas * (kl * sizeof(unsigned long long) + sizeof(float2)) + rows_max * sizeof(int);
 }
-bool select_lists_in_smem(const Params& p) { return select_smem_bytes(p, true) <= 160 * 1024; }
+bool select_lists_in_smem(const Params& p) {
+  return p.lm_ctas <= 320 && select_smem_bytes(p, true) <= 160 * 1024;
+}
 size_t select_smem(const Params& p) { return select_smem_bytes(p, select_lists_in_smem(p)); }
 size_t rerank_smem(const Params& p) { return (size_t)p.Nn * (sizeof(uint32_t) + sizeof(int)); }
 
