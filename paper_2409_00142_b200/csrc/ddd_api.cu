@@ -18,7 +18,7 @@ size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
   size_t hbuf[2], part_key, part_ms, tree_token, tree_parent, tree_cum, beam_node, beam_tok, beam_cum,
-      row_plant, active, stop_depth, root_pos, n_active, dev_status, w_packed;
+      row_plant, active, stop_depth, root_pos, n_active, dev_status, lm_ticket, w_packed;
   // staging for ddd_draft_host: inputs, then the packed output block
   size_t in_hidden, in_token, in_pos, out_block;
   size_t o_n_out, o_stop, o_token, o_parent, o_depth, o_position, o_cum, o_mask, o_H, o_status, out_bytes;
@@ -70,6 +70,7 @@ Layout make_layout(const ddd_config* c) {
   L.root_pos = take(B * 4);
   L.n_active = take(4);
   L.dev_status = take(4);
+  L.lm_ticket = take(8);
   // packed copy of W for the tensor-core kernel (kept 1024-byte aligned relative to the base)
   off = (off + 1023) / 1024 * 1024;
   const bool tc_possible = c->dtype == DDD_DTYPE_BF16 && c->hidden % 64 == 0 && c->lm_head_kernel != DDD_LM_HEAD_SIMT;
@@ -123,6 +124,8 @@ struct ddd_handle {
   cudaGraphExec_t exec;
   GraphKey key;
   bool have_graph;
+  bool use_pdl;    // programmatic dependent launch between the kernels of a draft
+  bool graph_pdl;  // whether the captured graph uses it
   // pinned host bounce buffer for ddd_draft_host
   unsigned char* bounce;
   size_t bounce_bytes;
@@ -130,21 +133,50 @@ struct ddd_handle {
 
 namespace {
 
-cudaError_t launch_lm_head(const ddd_handle* h, int d, int force_all, cudaStream_t st) {
-  if (h->lm_kind == DDD_LM_HEAD_TCGEN05) return launch_lm_head_tc(h->p, h->tc, d, force_all, st);
+cudaError_t launch_lm_head(const ddd_handle* h, int d, int force_all, bool pdl, cudaStream_t st) {
+  if (h->lm_kind == DDD_LM_HEAD_TCGEN05) return launch_lm_head_tc(h->p, h->tc, d, force_all, pdl, st);
   return launch_lm_head_simt(h->p, d, force_all, h->p.lm_ctas, st);
 }
 
 // Everything after the init kernel: it depends on the output pointers only, so a captured
 // graph of it can be replayed for any root.
-cudaError_t enqueue_passes(const ddd_handle* h, const DraftIO& io, cudaStream_t st) {
+// With pdl every kernel but the first is launched with programmatic stream serialisation: it
+// may start while its predecessor runs and waits for it on the device (the first LM-head pass
+// follows the init kernel in plain stream order).
+cudaError_t enqueue_passes(const ddd_handle* h, const DraftIO& io, bool pdl, cudaStream_t st) {
   cudaError_t e = cudaSuccess;
   for (int d = 1; d <= h->p.n && e == cudaSuccess; ++d) {
-    e = launch_lm_head(h, d, 0, st);
-    if (e == cudaSuccess) e = launch_select(h->p, io, d, st);
+    e = launch_lm_head(h, d, 0, pdl && d > 1, st);
+    if (e == cudaSuccess) e = launch_select(h->p, io, d, pdl, st);
   }
-  if (e == cudaSuccess) e = launch_rerank(h->p, io, st);
+  if (e == cudaSuccess) e = launch_rerank(h->p, io, pdl, st);
   return e;
+}
+
+// Captures everything after the init kernel into h->exec.  Returns false (and leaves no graph)
+// on any failure.
+bool capture_graph(ddd_handle* h, const DraftIO& io, bool pdl, cudaStream_t st) {
+  if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+    cudaGetLastError();
+    return false;
+  }
+  const cudaError_t e = enqueue_passes(h, io, pdl, st);
+  cudaGraph_t graph = nullptr;
+  const cudaError_t e2 = cudaStreamEndCapture(st, &graph);
+  if (e != cudaSuccess || e2 != cudaSuccess || !graph) {
+    if (graph) cudaGraphDestroy(graph);
+    cudaGetLastError();
+    return false;
+  }
+  const cudaError_t e3 = cudaGraphInstantiate(&h->exec, graph, 0);
+  cudaGraphDestroy(graph);
+  if (e3 != cudaSuccess) {
+    cudaGetLastError();
+    h->exec = nullptr;
+    return false;
+  }
+  h->graph_pdl = pdl;
+  return true;
 }
 
 bool aligned16(const void* q) { return (reinterpret_cast<uintptr_t>(q) & 15u) == 0; }
@@ -181,6 +213,8 @@ int ddd_create(const ddd_config* cfg, const void* W, const void* E, const float*
   h->ws = static_cast<unsigned char*>(workspace);
   h->sm_count = prop.multiProcessorCount;
   h->have_graph = false;
+  h->use_pdl = true;
+  h->graph_pdl = false;
   h->exec = nullptr;
   h->bounce = nullptr;
   h->bounce_bytes = 0;
@@ -212,6 +246,7 @@ int ddd_create(const ddd_config* cfg, const void* W, const void* E, const float*
   p.root_pos = reinterpret_cast<int*>(ws + L.root_pos);
   p.n_active = reinterpret_cast<int*>(ws + L.n_active);
   p.dev_status = reinterpret_cast<int*>(ws + L.dev_status);
+  p.lm_ticket = reinterpret_cast<int*>(ws + L.lm_ticket);
 
   int rc = DDD_OK;
   // Zero the workspace once so that rows never written by a draft hold finite values.
@@ -260,21 +295,9 @@ int ddd_draft(ddd_handle* h, const void* root_hidden, const int32_t* root_token,
     if (!h->have_graph || std::memcmp(&key, &h->key, sizeof key) != 0) {
       if (h->exec) { cudaGraphExecDestroy(h->exec); h->exec = nullptr; }
       h->have_graph = false;
-      if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
-        cudaGetLastError();
-        return DDD_ERR_CUDA;
-      }
-      const cudaError_t e = enqueue_passes(h, io, st);
-      cudaGraph_t graph = nullptr;
-      const cudaError_t e2 = cudaStreamEndCapture(st, &graph);
-      if (e != cudaSuccess || e2 != cudaSuccess || !graph) {
-        if (graph) cudaGraphDestroy(graph);
-        cudaGetLastError();
-        return DDD_ERR_CUDA;
-      }
-      const cudaError_t e3 = cudaGraphInstantiate(&h->exec, graph, 0);
-      cudaGraphDestroy(graph);
-      if (e3 != cudaSuccess) { cudaGetLastError(); h->exec = nullptr; return DDD_ERR_CUDA; }
+      // capture with programmatic dependent launches; if this driver cannot capture or
+      // instantiate them, capture the plain stream-ordered sequence instead
+      if (!(h->use_pdl && capture_graph(h, io, true, st)) && !capture_graph(h, io, false, st)) return DDD_ERR_CUDA;
       h->key = key;
       h->have_graph = true;
     }
@@ -286,7 +309,7 @@ int ddd_draft(ddd_handle* h, const void* root_hidden, const int32_t* root_token,
     return DDD_OK;
   }
   if (launch_init(h->p, io, root_hidden, root_token, root_pos, st) != cudaSuccess ||
-      enqueue_passes(h, io, st) != cudaSuccess) {
+      enqueue_passes(h, io, h->use_pdl, st) != cudaSuccess) {
     cudaGetLastError();
     return DDD_ERR_CUDA;
   }
@@ -358,7 +381,7 @@ int ddd_draft_host(ddd_handle* h, const void* root_hidden, const int32_t* root_t
 int ddd_lm_head_pass(ddd_handle* h, void* cuda_stream) {
   if (!h) return DDD_ERR_INVALID_ARG;
   // Pass index 2 selects the hidden buffer written by the first draft step; all rows are forced live.
-  if (launch_lm_head(h, 2, 1, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) {
+  if (launch_lm_head(h, 2, 1, h->use_pdl, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) {
     cudaGetLastError();
     return DDD_ERR_CUDA;
   }

@@ -44,6 +44,7 @@ struct Params {
   int* stop_depth;                // [B]
   int* root_pos;                  // [B] copy of the caller's root positions
   int* dev_status;                // [1] first error recorded by a kernel during this draft
+  int* lm_ticket;                 // [1] arrival counter of the tensor-core LM-head blocks
 };
 
 // Per-draft pointers (caller-owned device memory).
@@ -86,6 +87,15 @@ __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFullMask, v, o);
   return v;
+}
+
+// Programmatic dependent launch: a kernel launched with the attribute below may start while
+// its predecessor in the stream is still running; griddep_wait() blocks until that predecessor
+// has completed and its writes are visible, griddep_launch_dependents() lets the successor
+// start.  Both are no-ops for kernels launched the ordinary way.
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch_dependents() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
 
 __device__ __forceinline__ float neg_inf() { return __uint_as_float(0xFF800000u); }
@@ -173,7 +183,9 @@ cudaError_t prepare_tree(const Params& p);
 cudaError_t launch_init(const Params& p, const DraftIO& io, const void* root_hidden, const int* root_token,
                         const int* root_pos, cudaStream_t st);
 cudaError_t launch_lm_head_simt(const Params& p, int d, int force_all, int ctas, cudaStream_t st);
-cudaError_t launch_select(const Params& p, const DraftIO& io, int d, cudaStream_t st);
-cudaError_t launch_rerank(const Params& p, const DraftIO& io, cudaStream_t st);
+// pdl: launch with programmatic stream serialisation (the kernel may start before its
+// predecessor has finished and synchronises with it through griddep_wait()).
+cudaError_t launch_select(const Params& p, const DraftIO& io, int d, bool pdl, cudaStream_t st);
+cudaError_t launch_rerank(const Params& p, const DraftIO& io, bool pdl, cudaStream_t st);
 
 }  // namespace ddd

@@ -192,7 +192,23 @@ __global__ void __launch_bounds__(kTcThreads, 1)
 lm_head_tc_kernel(const Params p, const unsigned char* __restrict__ w_packed,
                   const __grid_constant__ CUtensorMap map_h, const int d, const int force_all,
                   const int n_pad, const int stages, const int tmem_cols, const int ksub) {
-  if (!force_all && *p.n_active == 0) return;
+  // The kernel may have been launched while the select kernel of the previous pass is still
+  // running (programmatic dependent launch).  Until griddep_wait() below it touches nothing
+  // that kernel writes, except for one speculative look at the activity counter: if drafting
+  // had already stopped before that kernel, there is nothing to prefetch.
+  const bool spec_active = force_all || *reinterpret_cast<volatile const int*>(p.n_active) != 0;
+  __shared__ int s_ticket;
+  if (threadIdx.x == 0) {
+    // arrival counter, reset by the last block to arrive; a successor kernel can only start once
+    // every block of this one has passed griddep_launch_dependents() below, i.e. after the reset
+    const int t = atomicAdd(p.lm_ticket, 1);
+    if (t == (int)gridDim.x - 1) {
+      atomicExch(p.lm_ticket, 0);
+      __threadfence();
+    }
+    s_ticket = t % (int)gridDim.x;
+  }
+  __syncthreads();
 
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(
@@ -218,7 +234,11 @@ lm_head_tc_kernel(const Params p, const unsigned char* __restrict__ w_packed,
   // this block's contiguous range of 32-row units
   const int n_units = (p.V + kUnitRows - 1) / kUnitRows;
   const int base_units = n_units / (int)gridDim.x, rem_units = n_units % (int)gridDim.x;
-  const int bid = blockIdx.x;
+  // Vocab ranges are handed out in arrival order: the larger ranges go to the blocks that
+  // start first, and the blocks that could only start after the previous select kernel left
+  // its SMs get the smaller ones.  Range (and partial-result slot) `bid` always covers the
+  // same rows, so the result does not depend on which block took it.
+  const int bid = s_ticket;
   const int my_units = base_units + (bid < rem_units ? 1 : 0);
   const int unit0 = bid * base_units + (bid < rem_units ? bid : rem_units);
   // MMA tiles: up to four consecutive units, counted from the start of the block's range.
@@ -230,19 +250,21 @@ lm_head_tc_kernel(const Params p, const unsigned char* __restrict__ w_packed,
   const int total_iters = n_tiles * num_kb;
   const int prefill = total_iters < stages ? total_iters : stages;
   unsigned long long evict_first = 0ull;
-  auto issue = [&](int it, int stage) {
+  auto issue_w = [&](int it, int stage) {
     const int t = it / num_kb, kb = it - t * num_kb;
     const int nu = min(4, my_units - 4 * t);
     const uint32_t full = bar_full + 8u * stage;
-    mbar_expect_tx(full, (uint32_t)ksub * ((uint32_t)nu * kUnitBytes + b_bytes));
+    mbar_expect_tx(full, (uint32_t)ksub * ((uint32_t)nu * kUnitBytes + b_bytes));   // W and h bytes of the stage
     // W: for each 64-element K-block the tile's units are one contiguous run of the packed copy
     const unsigned char* src = w_packed + ((size_t)(kb * ksub) * n_units + (size_t)(unit0 + 4 * t)) * kUnitBytes;
     const uint32_t dst = a_base + (uint32_t)stage * a_stage;
     for (int kk = 0; kk < ksub; ++kk)
       bulk_load_hint(dst + (uint32_t)kk * kABytes, src + (size_t)kk * n_units * kUnitBytes, (uint32_t)nu * kUnitBytes,
                      full, evict_first);
+  };
+  auto issue_h = [&](int it, int stage) {
     // h: ksub K-blocks of all beam rows in one tensor copy
-    tma_load_3d(b_base + (uint32_t)stage * b_stage, &map_h, full, 0, 0, kb * ksub);
+    tma_load_3d(b_base + (uint32_t)stage * b_stage, &map_h, bar_full + 8u * stage, 0, 0, (it % num_kb) * ksub);
   };
 
   if (threadIdx.x == 0) {
@@ -258,9 +280,28 @@ lm_head_tc_kernel(const Params p, const unsigned char* __restrict__ w_packed,
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    // Start streaming right away, while the other warps are still setting up.
+    // W does not depend on the previous kernel: fill the ring with it right away.
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(evict_first));
-    issue(0, 0);
+    if (spec_active)
+      for (int it = 0; it < prefill; ++it) issue_w(it, it);
+  }
+  __syncwarp();
+
+  // ---- from here on the previous kernel's results (hidden rows, row flags, counters) are needed
+  griddep_wait();
+  griddep_launch_dependents();
+  if (!force_all && *p.n_active == 0) {
+    // every sequence has stopped: complete and await the copies already in flight, then leave
+    if (spec_active && threadIdx.x == 0) {
+      for (int it = 0; it < prefill; ++it) issue_h(it, it);
+      for (int it = 0; it < prefill; ++it) mbar_wait(bar_full + 8u * it, 0u, abort_flag, p.dev_status, false);
+    }
+    return;
+  }
+  if (threadIdx.x == 0) {
+    if (!spec_active)
+      for (int it = 0; it < prefill; ++it) issue_w(it, it);
+    for (int it = 0; it < prefill; ++it) issue_h(it, it);
   }
   __syncwarp();
   if (warp == 1) {   // tensor-memory allocation is a warp-wide operation
@@ -284,16 +325,16 @@ lm_head_tc_kernel(const Params p, const unsigned char* __restrict__ w_packed,
   // each warp stays converged for the block-wide barriers and the warp-wide tcgen05 calls.
   if (warp == 0) {
     // ======================================================================= TMA producer
-    if (lane == 0)
-      for (int it = 1; it < prefill; ++it) issue(it, it);
-    __syncwarp();
     int stage = prefill % stages, issued = prefill;
     uint32_t phase = (prefill == stages) ? 1u : 0u;
     bool ok = true;
     for (int it = prefill; it < total_iters; ++it) {
       ok = __all_sync(kFullMask, mbar_wait(bar_empty + 8u * stage, phase ^ 1u, abort_flag, p.dev_status));
       if (!ok) break;
-      if (lane == 0) issue(it, stage);
+      if (lane == 0) {
+        issue_w(it, stage);
+        issue_h(it, stage);
+      }
       __syncwarp();
       ++issued;
       if (++stage == stages) { stage = 0; phase ^= 1u; }
@@ -525,10 +566,19 @@ int tc_plan_create(const Params& p, int sm_count, void* w_packed, TcPlan* plan) 
   return DDD_OK;
 }
 
-cudaError_t launch_lm_head_tc(const Params& p, const TcPlan& plan, int d, int force_all, cudaStream_t st) {
-  lm_head_tc_kernel<<<plan.ctas, kTcThreads, plan.smem, st>>>(p, plan.w_packed, plan.map_h[(d - 1) & 1], d, force_all,
-                                                              plan.n_pad, plan.stages, plan.tmem_cols, plan.ksub);
-  return cudaGetLastError();
+cudaError_t launch_lm_head_tc(const Params& p, const TcPlan& plan, int d, int force_all, bool pdl, cudaStream_t st) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)plan.ctas, 1, 1);
+  cfg.blockDim = dim3(kTcThreads, 1, 1);
+  cfg.dynamicSmemBytes = plan.smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, lm_head_tc_kernel, p, (const unsigned char*)plan.w_packed, plan.map_h[(d - 1) & 1], d,
+                            force_all, plan.n_pad, plan.stages, plan.tmem_cols, plan.ksub);
 }
 
 }  // namespace ddd

@@ -23,6 +23,7 @@ size_t tc_packed_bytes(int vocab, int hidden);
 // Packs W into `w_packed` (device, 1024-byte aligned, tc_packed_bytes), encodes the tensor maps of
 // the hidden buffers and sizes the pipeline.  Synchronises the device.  Returns a DDD_* code.
 int tc_plan_create(const Params& p, int sm_count, void* w_packed, TcPlan* plan);
-cudaError_t launch_lm_head_tc(const Params& p, const TcPlan& plan, int d, int force_all, cudaStream_t st);
+// pdl: launch with programmatic stream serialisation (see griddep_wait in ddd_common.cuh).
+cudaError_t launch_lm_head_tc(const Params& p, const TcPlan& plan, int d, int force_all, bool pdl, cudaStream_t st);
 
 }  // namespace ddd

@@ -39,6 +39,7 @@ __global__ void init_kernel(const Params p, const T* __restrict__ root_hidden,
     if (b == 0) {
       *p.n_active = p.B;
       *p.dev_status = DDD_OK;
+      *p.lm_ticket = 0;
     }
   }
 }
@@ -325,6 +326,10 @@ __device__ void draft_step(const Params& p, int b, int d, const int* sel_flat, c
 // their (max, sum-exp) [rows_max][nc], and the rows' planted columns [rows_max].
 __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Params p, const DraftIO io,
                                                                        const int d, const int lists_in_smem) {
+  // Wait for the LM-head pass, then let the next pass start: it streams W into shared memory
+  // while this kernel works and reads the new hidden rows only after this kernel has finished.
+  griddep_wait();
+  griddep_launch_dependents();
   cg::cluster_group cluster = cg::this_cluster();
   const int crank = (int)cluster.block_rank();
   const int b = blockIdx.x / kSelCluster;
@@ -531,6 +536,7 @@ __device__ int block_exclusive_scan(int v, int* warp_tot /* [32] shared */, int*
 
 // Dynamic shared memory: ordered cum keys [Nn], selection flags / output rows [Nn].
 __global__ void __launch_bounds__(kRerankThreads) rerank_mask_kernel(const Params p, const DraftIO io) {
+  griddep_wait();
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int b = blockIdx.x, tid = threadIdx.x;
   const int k = p.k, T = p.T;
@@ -699,25 +705,36 @@ cudaError_t launch_init(const Params& p, const DraftIO&, const void* root_hidden
   return cudaGetLastError();
 }
 
-cudaError_t launch_select(const Params& p, const DraftIO& io, int d, cudaStream_t st) {
+cudaError_t launch_select(const Params& p, const DraftIO& io, int d, bool pdl, cudaStream_t st) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(p.B * kSelCluster), 1, 1);
   cfg.blockDim = dim3(kSelThreads, 1, 1);
   cfg.dynamicSmemBytes = select_smem(p);
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = kSelCluster;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = pdl ? 2 : 1;
   return cudaLaunchKernelEx(&cfg, select_gate_step_kernel, p, io, d, select_lists_in_smem(p) ? 1 : 0);
 }
 
-cudaError_t launch_rerank(const Params& p, const DraftIO& io, cudaStream_t st) {
-  rerank_mask_kernel<<<p.B, kRerankThreads, rerank_smem(p), st>>>(p, io);
-  return cudaGetLastError();
+cudaError_t launch_rerank(const Params& p, const DraftIO& io, bool pdl, cudaStream_t st) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)p.B, 1, 1);
+  cfg.blockDim = dim3(kRerankThreads, 1, 1);
+  cfg.dynamicSmemBytes = rerank_smem(p);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, rerank_mask_kernel, p, io);
 }
 
 }  // namespace ddd
