@@ -38,6 +38,7 @@ constexpr int kABytes = kBlockM * kBlockK * 2;        // 16384
 constexpr int kChunkCols = 16;          // accumulator columns (beam rows) per epilogue chunk
 constexpr int kSmemLimit = 232448;      // 227 KB opt-in limit per block
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+constexpr int kL2PrefetchBytes = 128 * 1024;   // per block, ahead of the dependency wait (about 64 MB in all)
 
 struct SmemPlan {
   int a, b, zt, key, ms, plant, live, bars, tmem_ptr, abort_flag, total;
@@ -123,6 +124,10 @@ __device__ __forceinline__ void bulk_load_hint(uint32_t dst, const void* src, ui
       "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
       ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(policy)
       : "memory");
+}
+// Asks L2 to fetch a contiguous region (multiple of 16 bytes); nothing lands in shared memory.
+__device__ __forceinline__ void l2_prefetch(const void* src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -286,6 +291,16 @@ lm_head_tc_kernel(const Params p, const unsigned char* __restrict__ w_packed,
       for (int it = 0; it < prefill; ++it) issue_w(it, it);
   }
   __syncwarp();
+  // While the previous kernel is still at work HBM is idle: one more thread asks L2 for the part
+  // of W that follows the ring (first tile, in the order the pipeline will want it), about as
+  // much as the memory system can deliver before the wait below returns.
+  if (spec_active && threadIdx.x == 64) {
+    const int nu0 = min(4, my_units);
+    const int kb_first = prefill * ksub;
+    const int kb_last = min(p.Hd / kBlockK, kb_first + kL2PrefetchBytes / (nu0 * kUnitBytes));
+    for (int kb64 = kb_first; kb64 < kb_last; ++kb64)
+      l2_prefetch(w_packed + ((size_t)kb64 * n_units + (size_t)unit0) * kUnitBytes, (uint32_t)nu0 * kUnitBytes);
+  }
 
   // ---- from here on the previous kernel's results (hidden rows, row flags, counters) are needed
   griddep_wait();
