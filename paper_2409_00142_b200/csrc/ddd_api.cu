@@ -140,13 +140,12 @@ cudaError_t launch_lm_head(const ddd_handle* h, int d, int force_all, bool pdl, 
 
 // Everything after the init kernel: it depends on the output pointers only, so a captured
 // graph of it can be replayed for any root.
-// With pdl every kernel but the first is launched with programmatic stream serialisation: it
-// may start while its predecessor runs and waits for it on the device (the first LM-head pass
-// follows the init kernel in plain stream order).
+// With pdl every kernel after the init kernel is launched with programmatic stream
+// serialisation: it may start while its predecessor runs and waits for it on the device.
 cudaError_t enqueue_passes(const ddd_handle* h, const DraftIO& io, bool pdl, cudaStream_t st) {
   cudaError_t e = cudaSuccess;
   for (int d = 1; d <= h->p.n && e == cudaSuccess; ++d) {
-    e = launch_lm_head(h, d, 0, pdl && d > 1, st);
+    e = launch_lm_head(h, d, 0, pdl, st);
     if (e == cudaSuccess) e = launch_select(h->p, io, d, pdl, st);
   }
   if (e == cudaSuccess) e = launch_rerank(h->p, io, pdl, st);

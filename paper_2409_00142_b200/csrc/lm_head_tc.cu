@@ -200,8 +200,8 @@ lm_head_tc_kernel(const Params p, const unsigned char* __restrict__ w_packed,
   // The kernel may have been launched while the select kernel of the previous pass is still
   // running (programmatic dependent launch).  Until griddep_wait() below it touches nothing
   // that kernel writes, except for one speculative look at the activity counter: if drafting
-  // had already stopped before that kernel, there is nothing to prefetch.
-  const bool spec_active = force_all || *reinterpret_cast<volatile const int*>(p.n_active) != 0;
+  // had already stopped before that kernel, there is nothing to prefetch (pass 1 always runs).
+  const bool spec_active = force_all || d == 1 || *reinterpret_cast<volatile const int*>(p.n_active) != 0;
   __shared__ int s_ticket;
   if (threadIdx.x == 0) {
     // arrival counter, reset by the last block to arrive; a successor kernel can only start once

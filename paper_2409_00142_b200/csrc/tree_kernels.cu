@@ -19,6 +19,7 @@ constexpr int kRerankThreads = 1024;
 template <typename T>
 __global__ void init_kernel(const Params p, const T* __restrict__ root_hidden,
                             const int* __restrict__ root_token, const int* __restrict__ root_pos) {
+  griddep_launch_dependents();   // the first LM-head pass may start streaming W while this runs
   const int b = blockIdx.x;
   T* dst = static_cast<T*>(p.hbuf[0]) + (size_t)b * p.k * p.Hd;
   const T* src = root_hidden + (size_t)b * p.Hd;
@@ -39,7 +40,6 @@ __global__ void init_kernel(const Params p, const T* __restrict__ root_hidden,
     if (b == 0) {
       *p.n_active = p.B;
       *p.dev_status = DDD_OK;
-      *p.lm_ticket = 0;
     }
   }
 }
@@ -570,14 +570,28 @@ __global__ void __launch_bounds__(kRerankThreads) rerank_mask_kernel(const Param
       if ((q & known_mask) == prefix) atomicAdd(&hist[(q >> shift) & 0xFF], 1);
     }
     __syncthreads();
-    if (tid == 0) {
-      int remaining = s_remaining, bin = 255;
-      for (; bin > 0; --bin) {
-        if (hist[bin] >= remaining) break;
-        remaining -= hist[bin];
+    if (tid < 32) {
+      // warp 0 finds the bin holding the `remaining`-th largest key: lane l owns bins 8l .. 8l+7
+      const int remaining = s_remaining;
+      int local[8], mine = 0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { local[i] = hist[8 * tid + i]; mine += local[i]; }
+      int above = mine;                                   // suffix sum over lanes >= tid ...
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_down_sync(kFullMask, above, o);
+        if (tid + o < 32) above += t;
       }
-      s_prefix = prefix | ((uint32_t)bin << shift);
-      s_remaining = remaining;
+      above -= mine;                                      // ... made exclusive: keys in higher lanes' bins
+      if (above < remaining && remaining <= above + mine) {   // exactly one lane
+        int rem = remaining - above, bin = 7;
+        for (; bin > 0; --bin) {
+          if (local[bin] >= rem) break;
+          rem -= local[bin];
+        }
+        s_prefix = prefix | ((uint32_t)(8 * tid + bin) << shift);
+        s_remaining = rem;
+      }
     }
     known_mask |= 0xFFu << shift;
     __syncthreads();
