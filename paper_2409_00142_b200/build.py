@@ -40,7 +40,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     cmd = [nvcc, *NVCC_FLAGS, "-I", os.path.join(ROOT, "include"), "-I", CSRC]
     if verbose:
         cmd += ["-Xptxas", "-v"]
-    cmd += ["-o", tmp, *sources()]
+    cmd += ["-o", tmp, *sources(), "-lcudadevrt"]
     subprocess.run(cmd, check=True)
     os.replace(tmp, LIB)
     return LIB

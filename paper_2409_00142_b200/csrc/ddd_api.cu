@@ -142,34 +142,74 @@ cudaError_t launch_lm_head(const ddd_handle* h, int d, int force_all, bool pdl, 
 // graph of it can be replayed for any root.
 // With pdl every kernel after the init kernel is launched with programmatic stream
 // serialisation: it may start while its predecessor runs and waits for it on the device.
-cudaError_t enqueue_passes(const ddd_handle* h, const DraftIO& io, bool pdl, cudaStream_t st) {
+// Passes first..last are enqueued; the select kernel of pass `cond_pass` (0 = none) switches
+// the graph conditional `cond` on if its sequence goes on.
+cudaError_t enqueue_passes(const ddd_handle* h, const DraftIO& io, bool pdl, int first, int last,
+                           cudaGraphConditionalHandle cond, int cond_pass, cudaStream_t st) {
   cudaError_t e = cudaSuccess;
-  for (int d = 1; d <= h->p.n && e == cudaSuccess; ++d) {
-    e = launch_lm_head(h, d, 0, pdl, st);
-    if (e == cudaSuccess) e = launch_select(h->p, io, d, pdl, st);
+  for (int d = first; d <= last && e == cudaSuccess; ++d) {
+    e = launch_lm_head(h, d, 0, pdl && d > first, st);
+    if (e == cudaSuccess) e = launch_select(h->p, io, d, pdl, cond, d == cond_pass, st);
   }
-  if (e == cudaSuccess) e = launch_rerank(h->p, io, pdl, st);
   return e;
 }
+
+// Passes of a captured draft that always run; the rest sit behind one conditional node that
+// stays off unless some sequence is still drafting after them.  Most drafts stop early, and a
+// pass that has nothing to do still costs two kernel launches.
+constexpr int kUnconditionalPasses = 3;
 
 // Captures everything after the init kernel into h->exec.  Returns false (and leaves no graph)
 // on any failure.
 bool capture_graph(ddd_handle* h, const DraftIO& io, bool pdl, cudaStream_t st) {
-  if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
-    cudaGetLastError();
-    return false;
+  const int n = h->p.n;
+  const int head = n <= kUnconditionalPasses + 1 ? n : kUnconditionalPasses;   // passes outside the conditional
+  cudaGraph_t graph = nullptr, body = nullptr;
+  cudaGraphConditionalHandle cond = 0;
+  bool ok = cudaGraphCreate(&graph, 0) == cudaSuccess;
+  if (ok && head < n) ok = cudaGraphConditionalHandleCreate(&cond, graph, 0, cudaGraphCondAssignDefault) == cudaSuccess;
+  bool capturing = false;
+  if (ok) {
+    ok = cudaStreamBeginCaptureToGraph(st, graph, nullptr, nullptr, 0, cudaStreamCaptureModeThreadLocal) == cudaSuccess;
+    capturing = ok;
   }
-  const cudaError_t e = enqueue_passes(h, io, pdl, st);
-  cudaGraph_t graph = nullptr;
-  const cudaError_t e2 = cudaStreamEndCapture(st, &graph);
-  if (e != cudaSuccess || e2 != cudaSuccess || !graph) {
-    if (graph) cudaGraphDestroy(graph);
-    cudaGetLastError();
-    return false;
+  if (ok) ok = enqueue_passes(h, io, pdl, 1, head, cond, head < n ? head : 0, st) == cudaSuccess;
+  if (ok && head < n) {
+    // splice an IF node between the captured passes and the rerank
+    cudaStreamCaptureStatus status;
+    const cudaGraphNode_t* deps = nullptr;
+    size_t n_deps = 0;
+    ok = cudaStreamGetCaptureInfo(st, &status, nullptr, nullptr, &deps, &n_deps) == cudaSuccess &&
+         status == cudaStreamCaptureStatusActive;
+    cudaGraphNode_t node = nullptr;
+    if (ok) {
+      cudaGraphNodeParams np = {};
+      np.type = cudaGraphNodeTypeConditional;
+      np.conditional.handle = cond;
+      np.conditional.type = cudaGraphCondTypeIf;
+      np.conditional.size = 1;
+      ok = cudaGraphAddNode(&node, graph, deps, n_deps, &np) == cudaSuccess;
+      if (ok) body = np.conditional.phGraph_out[0];
+    }
+    if (ok) ok = cudaStreamUpdateCaptureDependencies(st, &node, 1, cudaStreamSetCaptureDependencies) == cudaSuccess;
   }
-  const cudaError_t e3 = cudaGraphInstantiate(&h->exec, graph, 0);
-  cudaGraphDestroy(graph);
-  if (e3 != cudaSuccess) {
+  // the rerank follows a conditional node, not a kernel: plain dependency
+  if (ok) ok = launch_rerank(h->p, io, pdl && head == n, st) == cudaSuccess;
+  if (capturing) {
+    cudaGraph_t done = nullptr;
+    if (cudaStreamEndCapture(st, &done) != cudaSuccess) ok = false;
+  }
+  if (ok && body) {
+    ok = cudaStreamBeginCaptureToGraph(st, body, nullptr, nullptr, 0, cudaStreamCaptureModeThreadLocal) == cudaSuccess;
+    if (ok) {
+      if (enqueue_passes(h, io, pdl, head + 1, n, cond, 0, st) != cudaSuccess) ok = false;
+      cudaGraph_t done = nullptr;
+      if (cudaStreamEndCapture(st, &done) != cudaSuccess) ok = false;
+    }
+  }
+  if (ok) ok = cudaGraphInstantiate(&h->exec, graph, 0) == cudaSuccess;
+  if (graph) cudaGraphDestroy(graph);
+  if (!ok) {
     cudaGetLastError();
     h->exec = nullptr;
     return false;
@@ -308,7 +348,8 @@ int ddd_draft(ddd_handle* h, const void* root_hidden, const int32_t* root_token,
     return DDD_OK;
   }
   if (launch_init(h->p, io, root_hidden, root_token, root_pos, st) != cudaSuccess ||
-      enqueue_passes(h, io, h->use_pdl, st) != cudaSuccess) {
+      enqueue_passes(h, io, h->use_pdl, 1, h->p.n, 0, 0, st) != cudaSuccess ||
+      launch_rerank(h->p, io, h->use_pdl, st) != cudaSuccess) {
     cudaGetLastError();
     return DDD_ERR_CUDA;
   }

@@ -185,7 +185,9 @@ cudaError_t launch_init(const Params& p, const DraftIO& io, const void* root_hid
 cudaError_t launch_lm_head_simt(const Params& p, int d, int force_all, int ctas, cudaStream_t st);
 // pdl: launch with programmatic stream serialisation (the kernel may start before its
 // predecessor has finished and synchronises with it through griddep_wait()).
-cudaError_t launch_select(const Params& p, const DraftIO& io, int d, bool pdl, cudaStream_t st);
+// set_cond: a sequence that continues after pass d sets the graph conditional `cond` to 1.
+cudaError_t launch_select(const Params& p, const DraftIO& io, int d, bool pdl, cudaGraphConditionalHandle cond,
+                          bool set_cond, cudaStream_t st);
 cudaError_t launch_rerank(const Params& p, const DraftIO& io, bool pdl, cudaStream_t st);
 
 }  // namespace ddd

@@ -325,7 +325,9 @@ __device__ void draft_step(const Params& p, int b, int d, const int* sel_flat, c
 // [rows_max][nc][k] (or only their first keys [rows_max][nc] when the lists do not fit),
 // their (max, sum-exp) [rows_max][nc], and the rows' planted columns [rows_max].
 __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Params p, const DraftIO io,
-                                                                       const int d, const int lists_in_smem) {
+                                                                       const int d, const int lists_in_smem,
+                                                                       const cudaGraphConditionalHandle cond,
+                                                                       const int set_cond) {
   // Wait for the LM-head pass, then let the next pass start: it streams W into shared memory
   // while this kernel works and reads the new hidden rows only after this kernel has finished.
   griddep_wait();
@@ -496,6 +498,9 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
       }
     }
   }
+  // In a captured draft the passes after this one sit behind a conditional node (default: skip);
+  // a sequence that goes on switches them on.
+  if (set_cond && !s_stop && crank == 0 && threadIdx.x == 0) cudaGraphSetConditional(cond, 1);
   if (s_stop) return;       // no block touches another block's shared memory after this point
 
   // ---- phase 3: synthetic draft step for the k new beam rows
@@ -719,7 +724,8 @@ cudaError_t launch_init(const Params& p, const DraftIO&, const void* root_hidden
   return cudaGetLastError();
 }
 
-cudaError_t launch_select(const Params& p, const DraftIO& io, int d, bool pdl, cudaStream_t st) {
+cudaError_t launch_select(const Params& p, const DraftIO& io, int d, bool pdl, cudaGraphConditionalHandle cond,
+                          bool set_cond, cudaStream_t st) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(p.B * kSelCluster), 1, 1);
   cfg.blockDim = dim3(kSelThreads, 1, 1);
@@ -734,7 +740,7 @@ cudaError_t launch_select(const Params& p, const DraftIO& io, int d, bool pdl, c
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = pdl ? 2 : 1;
-  return cudaLaunchKernelEx(&cfg, select_gate_step_kernel, p, io, d, select_lists_in_smem(p) ? 1 : 0);
+  return cudaLaunchKernelEx(&cfg, select_gate_step_kernel, p, io, d, select_lists_in_smem(p) ? 1 : 0, cond, set_cond ? 1 : 0);
 }
 
 cudaError_t launch_rerank(const Params& p, const DraftIO& io, bool pdl, cudaStream_t st) {
