@@ -193,7 +193,7 @@ __device__ void draft_step_cluster(const Params& p, int b, int d, const int* sel
                                    double* row_part /* [k][slots] */, double* row_inv /* [k] */) {
   cg::cluster_group cluster = cg::this_cluster();
   constexpr int N = Chunk<T>::N;
-  constexpr int kBatch = 4;
+  constexpr int kBatch = 2;
   const int k = p.k, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int cpr = p.Hd / N;            // chunks per row
   const int slots = cpr / 32;          // warp-sized groups of chunks per row
@@ -211,7 +211,9 @@ __device__ void draft_step_cluster(const Params& p, int b, int d, const int* sel
     es = (size_t)(tok >= 0 && tok < p.V ? tok : 0) * cpr + col;
     hd = (size_t)(b * k + row) * cpr + col;
   };
-  // pass 1: sum of squares per row
+  // pass 1: sum of squares per row.  The chunks of the first round (usually all there are)
+  // stay in registers for pass 2.
+  uint4 hv0[kBatch], ev0[kBatch];
   for (int q0 = first; q0 - lane < total; q0 += kBatch * stride) {
     uint4 hv[kBatch], ev[kBatch];
 #pragma unroll
@@ -223,6 +225,7 @@ __device__ void draft_step_cluster(const Params& p, int b, int d, const int* sel
         locate(q, hs, es, hd, row);
         hv[i] = Hsrc[hs];
         ev[i] = Esrc[es];
+        if (q0 == first) { hv0[i] = hv[i]; ev0[i] = ev[i]; }
       }
     }
 #pragma unroll
@@ -247,7 +250,7 @@ __device__ void draft_step_cluster(const Params& p, int b, int d, const int* sel
     row_inv[warp] = 1.0 / sqrt(ss / (double)p.Hd + (double)p.eps);
   }
   __syncthreads();
-  // pass 2: scale, round once, store (the inputs come back from the L1 / L2 caches)
+  // pass 2: scale, round once, store (later rounds re-read their inputs from the caches)
   for (int q0 = first; q0 - lane < total; q0 += kBatch * stride) {
     uint4 hv[kBatch], ev[kBatch];
     size_t dst[kBatch];
@@ -259,8 +262,8 @@ __device__ void draft_step_cluster(const Params& p, int b, int d, const int* sel
       if (q < total) {
         size_t hs, es;
         locate(q, hs, es, dst[i], rows[i]);
-        hv[i] = Hsrc[hs];
-        ev[i] = Esrc[es];
+        if (q0 == first) { hv[i] = hv0[i]; ev[i] = ev0[i]; }
+        else { hv[i] = Hsrc[hs]; ev[i] = Esrc[es]; }
       }
     }
 #pragma unroll
@@ -361,20 +364,47 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
   // (a warp copies one LM-head block's list per step: lane q takes the q-th key)
   for (int j = 0; j < n_mine; ++j) {
     const int r = b * k + crank + kSelCluster * j;
-    for (int c = warp; c < nc; c += kSelThreads / 32) {
-      const size_t slot = (size_t)c * R + r;
-      if (lane < kl) keys_s[((size_t)j * nc + c) * kl + lane] = p.part_key[slot * k + lane];
-      if (lane == 31) ms_s[(size_t)j * nc + c] = p.part_ms[slot];
+    constexpr int kW = kSelThreads / 32, kPre = 5;      // five lists per warp are fetched before any is stored
+    for (int c0 = warp; c0 < nc; c0 += kW * kPre) {
+      unsigned long long key[kPre];
+      float2 ms[kPre];
+#pragma unroll
+      for (int i = 0; i < kPre; ++i) {
+        const int c = c0 + kW * i;
+        if (c < nc) {
+          const size_t slot = (size_t)c * R + r;
+          if (lane < kl) key[i] = p.part_key[slot * k + lane];
+          if (lane == 31) ms[i] = p.part_ms[slot];
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < kPre; ++i) {
+        const int c = c0 + kW * i;
+        if (c < nc) {
+          if (lane < kl) keys_s[((size_t)j * nc + c) * kl + lane] = key[i];
+          if (lane == 31) ms_s[(size_t)j * nc + c] = ms[i];
+        }
+      }
     }
     if (threadIdx.x == 0) plant_s[j] = p.row_plant[r];
   }
   __syncthreads();
 
-  // ---- phase 1: one warp per beam row merges the per-block partials of the LM-head pass
+  // ---- phase 1: per beam row of this block, warp j merges the top-k lists while warp j + 4
+  //      adds up the log-sum-exp of the same row
+  __shared__ float lse_s[DDD_MAX_K / kSelCluster];
+  __shared__ unsigned long long plant_key_s[DDD_MAX_K / kSelCluster];
+  constexpr int kRowsPerBlock = DDD_MAX_K / kSelCluster;
+  unsigned long long res = 0ull;
   if (warp < n_mine) {
-    const int pr = crank + kSelCluster * warp, r = b * k + pr;
-    const float2* my_ms = ms_s + (size_t)warp * nc;
+    const int r = b * k + crank + kSelCluster * warp;
     const unsigned long long* my_keys = keys_s + (size_t)warp * nc * kl;
+    if (!lists_in_smem) res = merge_row_kway(p, r, k, nc, my_keys);
+    else if (nc <= 160) res = merge_row_heads<5>(k, nc, my_keys);
+    else res = merge_row_heads<10>(k, nc, my_keys);      // the host keeps nc <= 320 on this path
+  } else if (warp >= kRowsPerBlock && warp < kRowsPerBlock + n_mine) {
+    const int j = warp - kRowsPerBlock;
+    const float2* my_ms = ms_s + (size_t)j * nc;
     // log-sum-exp over all blocks (fixed lane-strided order, then a butterfly: deterministic)
     float M = neg_inf();
     for (int c = lane; c < nc; c += 32) M = fmaxf(M, my_ms[c].x);
@@ -386,7 +416,7 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
     }
     S = warp_sum(S);
     // planted column: its logit is (max of the others) + delta and it was left out of the partials
-    const int pc = plant_s[warp];
+    const int pc = plant_s[j];
     unsigned long long plant_key = 0ull;
     if (pc >= 0) {
       const float zc = M + p.plant_delta;
@@ -395,14 +425,18 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
       M = M2;
       plant_key = make_key(zc, (uint32_t)pc);
     }
-    const float lse = M + logf(S);
-
-    unsigned long long res;
-    if (!lists_in_smem) res = merge_row_kway(p, r, k, nc, my_keys);
-    else if (nc <= 160) res = merge_row_heads<5>(k, nc, my_keys);
-    else res = merge_row_heads<10>(k, nc, my_keys);      // the host keeps nc <= 320 on this path
+    if (lane == 0) {
+      lse_s[j] = M + logf(S);
+      plant_key_s[j] = plant_key;
+    }
+  }
+  __syncthreads();
+  if (warp < n_mine) {
+    const int pr = crank + kSelCluster * warp;
+    const float lse = lse_s[warp];
+    const unsigned long long plant_key = plant_key_s[warp];
     // insert the planted candidate into the sorted result
-    if (pc >= 0) {
+    if (plant_key != 0ull) {
       const int ins = __popc(__ballot_sync(kFullMask, lane < k && res > plant_key));
       const unsigned long long up = __shfl_up_sync(kFullMask, res, 1);
       if (lane == ins) res = plant_key;
@@ -417,20 +451,21 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
       p.tree_token[node] = tok;
       p.tree_parent[node] = p.beam_node[b * k + pr];
       p.tree_cum[node] = cand;
-      // the candidates of all rows meet in block 0
-      cluster.map_shared_rank(cand_key, 0)[flat] = (res != 0ull) ? make_key(cand, (uint32_t)flat) : 0ull;
-      cluster.map_shared_rank(cand_val, 0)[flat] = cand;
-      cluster.map_shared_rank(cand_tok, 0)[flat] = tok;
+      // every block of the cluster gets the candidates of all rows
+      const unsigned long long ckey = (res != 0ull) ? make_key(cand, (uint32_t)flat) : 0ull;
+      for (int rk = 0; rk < kSelCluster; ++rk) {
+        cluster.map_shared_rank(cand_key, rk)[flat] = ckey;
+        cluster.map_shared_rank(cand_val, rk)[flat] = cand;
+        cluster.map_shared_rank(cand_tok, rk)[flat] = tok;
+      }
     }
     if (lane == 0 && io.trace.row_lse) io.trace.row_lse[((size_t)b * p.n + (d - 1)) * k + pr] = lse;
   }
-  cluster.sync();
+  cluster.sync();       // the last time a block touches another block's shared memory before the draft step
 
-  // ---- phase 2: warp 0 of block 0 picks the new beam, evaluates Eq. 1 and takes the stop decision
-  int bk_flat = 0, bk_tok = -1;     // kept by warp 0 of block 0 for the bookkeeping after the barrier
-  float bk_cum = 0.f, bk_H = 0.f;
-  bool bk_stop = false;
-  if (crank == 0 && warp == 0) {
+  // ---- phase 2: warp 0 of every block picks the new beam, evaluates Eq. 1 and takes the stop
+  //      decision (same inputs, same result everywhere; block 0 records it)
+  if (warp == 0) {
     const int n_cand = P * k;
     unsigned long long mine = 0ull;
     if (n_cand <= 128) {
@@ -462,46 +497,44 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
       }
     }
     const bool have = lane < k && mine != 0ull;
-    bk_flat = have ? (int)key_index(mine) : 0;
-    bk_cum = have ? cand_val[bk_flat] : neg_inf();
-    const float M = __shfl_sync(kFullMask, bk_cum, 0);        // sorted descending: entry 0 is the max
-    const float sum = warp_sum(have ? expf(bk_cum - M) : 0.f);
-    bk_H = M + logf(sum);
-    bk_stop = (d == p.n);
-    if (!bk_stop && ((p.check_mask >> (d - 1)) & 1u)) bk_stop = bk_H < p.x;
-    bk_tok = lane < k ? cand_tok[bk_flat] : -1;
-    // every block needs the selection and the decision for the draft step
-    for (int rk = 0; rk < kSelCluster; ++rk) {
-      if (lane < k) {
-        cluster.map_shared_rank(sel_flat, rk)[lane] = bk_flat;
-        cluster.map_shared_rank(sel_tok, rk)[lane] = bk_tok;
-      }
-      if (lane == 0) *cluster.map_shared_rank(&s_stop, rk) = bk_stop ? 1 : 0;
-    }
-  }
-  cluster.sync();
-  // the bookkeeping in global memory is off the other warps' critical path
-  if (crank == 0 && warp == 0) {
+    const int flat = have ? (int)key_index(mine) : 0;
+    const float cum = have ? cand_val[flat] : neg_inf();
+    const float M = __shfl_sync(kFullMask, cum, 0);           // sorted descending: entry 0 is the max
+    const float sum = warp_sum(have ? expf(cum - M) : 0.f);
+    const float H = M + logf(sum);
+    bool stop = (d == p.n);
+    if (!stop && ((p.check_mask >> (d - 1)) & 1u)) stop = H < p.x;
+    const int tok = lane < k ? cand_tok[flat] : -1;
     if (lane < k) {
-      p.beam_node[b * k + lane] = base + bk_flat;
-      p.beam_tok[b * k + lane] = bk_tok;
-      p.beam_cum[b * k + lane] = bk_cum;
-      p.row_plant[b * k + lane] = (p.plant_next && bk_tok >= 0 && bk_tok < p.V) ? p.plant_next[bk_tok] : -1;
-      if (io.trace.beam_sel) io.trace.beam_sel[((size_t)b * p.n + (d - 1)) * k + lane] = bk_flat;
+      sel_flat[lane] = flat;
+      sel_tok[lane] = tok;
     }
-    if (lane == 0) {
-      io.out.H_trace[(size_t)b * p.n + (d - 1)] = bk_H;
-      if (bk_stop) {
-        p.stop_depth[b] = d;
-        p.active[b] = 0;
-        atomicSub(p.n_active, 1);
+    if (lane == 0) s_stop = stop ? 1 : 0;
+    __syncwarp();
+    if (crank == 0) {
+      // block 0 keeps the books in global memory (the other warps of the cluster go on meanwhile)
+      if (lane < k) {
+        p.beam_node[b * k + lane] = base + flat;
+        p.beam_tok[b * k + lane] = tok;
+        p.beam_cum[b * k + lane] = cum;
+        p.row_plant[b * k + lane] = (p.plant_next && tok >= 0 && tok < p.V) ? p.plant_next[tok] : -1;
+        if (io.trace.beam_sel) io.trace.beam_sel[((size_t)b * p.n + (d - 1)) * k + lane] = flat;
+      }
+      if (lane == 0) {
+        io.out.H_trace[(size_t)b * p.n + (d - 1)] = H;
+        if (stop) {
+          p.stop_depth[b] = d;
+          p.active[b] = 0;
+          atomicSub(p.n_active, 1);
+        }
       }
     }
   }
+  __syncthreads();
   // In a captured draft the passes after this one sit behind a conditional node (default: skip);
   // a sequence that goes on switches them on.
   if (set_cond && !s_stop && crank == 0 && threadIdx.x == 0) cudaGraphSetConditional(cond, 1);
-  if (s_stop) return;       // no block touches another block's shared memory after this point
+  if (s_stop) return;       // every block takes this branch alike
 
   // ---- phase 3: synthetic draft step for the k new beam rows
   if (p.dtype == DDD_DTYPE_BF16)
