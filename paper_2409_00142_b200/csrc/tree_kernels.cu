@@ -333,6 +333,8 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
                                                                        const int set_cond) {
   // Wait for the LM-head pass, then let the next pass start: it streams W into shared memory
   // while this kernel works and reads the new hidden rows only after this kernel has finished.
+  // (That burst slows this kernel's own few loads by 2-3 us each; releasing the next pass
+  // later was measured and lost more than it won.)
   griddep_wait();
   griddep_launch_dependents();
   cg::cluster_group cluster = cg::this_cluster();
@@ -359,34 +361,53 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
   __shared__ double row_part[DDD_MAX_K * 64];
   __shared__ double row_inv[DDD_MAX_K];
   __shared__ int s_stop;
+  __shared__ float beam_cum_s[DDD_MAX_K / kSelCluster];
+  __shared__ int beam_node_s[DDD_MAX_K / kSelCluster];
 
   // ---- phase 0: the block fetches everything phase 1 needs for its rows in one round trip
   // (a warp copies one LM-head block's list per step: lane q takes the q-th key)
-  for (int j = 0; j < n_mine; ++j) {
-    const int r = b * k + crank + kSelCluster * j;
-    constexpr int kW = kSelThreads / 32, kPre = 5;      // five lists per warp are fetched before any is stored
+  // All loads of all rows are issued before the first value is used: a round trip to memory
+  // costs this lone block a microsecond or two, so they must not queue up behind each other.
+  {
+    constexpr int kW = kSelThreads / 32, kPre = 5, kRows = 2;   // two rows x five lists per warp and batch
+    for (int j0 = 0; j0 < n_mine; j0 += kRows)
     for (int c0 = warp; c0 < nc; c0 += kW * kPre) {
-      unsigned long long key[kPre];
-      float2 ms[kPre];
+      unsigned long long key[kRows][kPre];
+      float2 ms[kRows][kPre];
 #pragma unroll
-      for (int i = 0; i < kPre; ++i) {
-        const int c = c0 + kW * i;
-        if (c < nc) {
-          const size_t slot = (size_t)c * R + r;
-          if (lane < kl) key[i] = p.part_key[slot * k + lane];
-          if (lane == 31) ms[i] = p.part_ms[slot];
+      for (int j = 0; j < kRows; ++j) {
+        if (j0 + j >= n_mine) continue;
+        const int r = b * k + crank + kSelCluster * (j0 + j);
+#pragma unroll
+        for (int i = 0; i < kPre; ++i) {
+          const int c = c0 + kW * i;
+          if (c < nc) {
+            const size_t slot = (size_t)c * R + r;
+            if (lane < kl) key[j][i] = p.part_key[slot * k + lane];
+            if (lane == 31) ms[j][i] = p.part_ms[slot];
+          }
         }
       }
+      // the few scalars phase 1 needs ride along with the first batch
+      if (j0 == 0 && c0 == warp && warp == 0 && lane < n_mine) {
+        const int r = b * k + crank + kSelCluster * lane;
+        plant_s[lane] = p.row_plant[r];
+        beam_cum_s[lane] = p.beam_cum[r];
+        beam_node_s[lane] = p.beam_node[r];
+      }
 #pragma unroll
-      for (int i = 0; i < kPre; ++i) {
-        const int c = c0 + kW * i;
-        if (c < nc) {
-          if (lane < kl) keys_s[((size_t)j * nc + c) * kl + lane] = key[i];
-          if (lane == 31) ms_s[(size_t)j * nc + c] = ms[i];
+      for (int j = 0; j < kRows; ++j) {
+        if (j0 + j >= n_mine) continue;
+#pragma unroll
+        for (int i = 0; i < kPre; ++i) {
+          const int c = c0 + kW * i;
+          if (c < nc) {
+            if (lane < kl) keys_s[((size_t)(j0 + j) * nc + c) * kl + lane] = key[j][i];
+            if (lane == 31) ms_s[(size_t)(j0 + j) * nc + c] = ms[j][i];
+          }
         }
       }
     }
-    if (threadIdx.x == 0) plant_s[j] = p.row_plant[r];
   }
   __syncthreads();
 
@@ -445,11 +466,11 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
     if (lane < k) {
       const float lp = (res != 0ull) ? fminf(key_value(res) - lse, 0.f) : neg_inf();
       const int tok = (res != 0ull) ? (int)key_index(res) : -1;
-      const float cand = p.beam_cum[b * k + pr] + lp;
+      const float cand = beam_cum_s[warp] + lp;
       const int flat = pr * k + lane;
       const size_t node = (size_t)b * p.Nn + base + flat;
       p.tree_token[node] = tok;
-      p.tree_parent[node] = p.beam_node[b * k + pr];
+      p.tree_parent[node] = beam_node_s[warp];
       p.tree_cum[node] = cand;
       // every block of the cluster gets the candidates of all rows
       const unsigned long long ckey = (res != 0ull) ? make_key(cand, (uint32_t)flat) : 0ull;
