@@ -554,6 +554,9 @@ int tc_plan_create(const Params& p, int sm_count, void* w_packed, TcPlan* plan) 
   int ksub = 4;
   while (ksub > 1 && (p.Hd % (kBlockK * ksub) != 0 || smem_plan(3, ksub, n_pad, p.R, p.k).total + 1024 > kSmemLimit))
     ksub /= 2;
+  // with many beam rows the h slice of a stage outweighs the W tile; two K-blocks in a ring of
+  // two stages still beat one K-block per stage (half as many pipeline steps)
+  if (ksub == 1 && p.Hd % (kBlockK * 2) == 0 && smem_plan(2, 2, n_pad, p.R, p.k).total + 1024 <= kSmemLimit) ksub = 2;
   int stages = 0;
   for (int s = 8; s >= 2; --s) {
     if (smem_plan(s, ksub, n_pad, p.R, p.k).total + 1024 <= kSmemLimit) { stages = s; break; }
