@@ -55,6 +55,8 @@ def parse_args():
     ap.add_argument("--cpu-sample", type=int, default=None, help="drafts the CPU baseline times")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true")
+    ap.add_argument("--launch-mode", default="graph", choices=["graph", "stream", "plain"],
+                    help="plain: ordinary stream-ordered launches, the mode profilers can follow")
     return ap.parse_args()
 
 
@@ -196,8 +198,13 @@ def mean_stop_depth(eng, roots_dev, device):
         eng.draft(r["root_hidden"], r["root_token"], r["root_pos"])
         torch.cuda.synchronize(device)
         assert int(eng.out["status"].item()) == 0, "device reported an error status"
-        depths += eng.out["stop_depth"].cpu().tolist()
-    return sum(depths) / len(depths)
+        depths.append(eng.out["stop_depth"].cpu().tolist())     # one list per draft (one entry per sequence)
+    return depths
+
+
+def _mean(depth_lists):
+    flat = [d for lst in depth_lists for d in lst]
+    return sum(flat) / len(flat)
 
 
 def run_reference(args):
@@ -259,10 +266,13 @@ def main():
     stream = torch.cuda.Stream(device)
 
     with torch.cuda.stream(stream):
-        eng = P.DraftEngine(cfg, weights, device=local, launch_mode=P.DDD_LAUNCH_GRAPH, with_trace=False)
+        mode = {"graph": P.DDD_LAUNCH_GRAPH, "stream": P.DDD_LAUNCH_STREAM, "plain": P.DDD_LAUNCH_PLAIN}[args.launch_mode]
+        eng = P.DraftEngine(cfg, weights, device=local, launch_mode=mode, with_trace=False)
         roots_dev = [{k: v.to(device) for k, v in r.items()} for r in roots_host]
         torch.cuda.synchronize(device)
-        depth_mean = mean_stop_depth(eng, roots_dev, device)
+        depth_lists = mean_stop_depth(eng, roots_dev, device)
+        depth_mean = _mean(depth_lists)
+        stop_depths = [max(lst) for lst in depth_lists]     # passes each draft needs
 
         sampler = ClockSampler(local)
         sampler.start()
@@ -307,7 +317,7 @@ def main():
                     ex = P.DraftEngine(cx, {"W": eng.W, "E": eng.E, "bias": eng.bias,
                                             "plant_next": eng.plant_next}, device=local,
                                        launch_mode=P.DDD_LAUNCH_GRAPH, with_trace=False)
-                    dm = mean_stop_depth(ex, roots_dev, device)
+                    dm = _mean(mean_stop_depth(ex, roots_dev, device))
                     msx, _ = timed_drafts(ex, roots_dev, max(3, args.steps // 4), args.warmup, world, device)
                     sweep[str(x)] = {"drafts_per_sec": drafts_total / (msx / 1e3), "mean_stop_depth": dm}
                     ex.close()
@@ -330,7 +340,7 @@ def main():
         e2e_ms = max_over_ranks(e2e_ms, world, device)
         h2d = sum(v.numel() * v.element_size() for v in pinned[0].values()) * n_per_rank
         d2h = sum(v.numel() * v.element_size() for v in host_out.values()) * n_per_rank
-        launches = P.ddd_launches_per_draft(eng.handle) * n_per_rank * args.steps
+        launches = sum(P.ddd_launches_per_draft(eng.handle, dd) for dd in stop_depths) * args.steps
         blocks = P.ddd_lm_head_blocks(eng.handle)
         eng.close()
 
@@ -349,7 +359,7 @@ def main():
                    "threshold": cfg.threshold, "drafts_per_step": n_per_rank * world,
                    "mean_stop_depth": depth_mean, "parallelism": f"replicas{world}",
                    "l2": "inputs larger than L2: every pass streams W (%.0f MB) from HBM" % (w_bytes / 1e6),
-                   "launch": "cuda_graph"},
+                   "launch": args.launch_mode},
         "clocks": clocks,
         "e2e": {"value": n_per_rank * world * cfg.batch / (e2e_ms / 1e3), "unit": UNIT,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},

@@ -59,8 +59,13 @@ enum { DDD_DTYPE_FP32 = 0, DDD_DTYPE_BF16 = 1 };
 /* Which LM-head kernel runs a pass.  AUTO picks TCGEN05 for bf16 and SIMT for fp32. */
 enum { DDD_LM_HEAD_AUTO = 0, DDD_LM_HEAD_SIMT = 1, DDD_LM_HEAD_TCGEN05 = 2 };
 
-/* How a draft is enqueued.  GRAPH replays one captured CUDA graph per draft. */
-enum { DDD_LAUNCH_STREAM = 0, DDD_LAUNCH_GRAPH = 1 };
+/* How a draft is enqueued.  STREAM launches kernel by kernel, each allowed to start while its
+ * predecessor still runs (programmatic dependent launch; they synchronise on the device).
+ * GRAPH replays one captured CUDA graph per draft, in which the passes after the third sit
+ * behind a conditional node that only a still-drafting sequence switches on.  PLAIN launches
+ * kernel by kernel in ordinary stream order, one after the other: the slowest, and the one
+ * profilers can follow. */
+enum { DDD_LAUNCH_STREAM = 0, DDD_LAUNCH_GRAPH = 1, DDD_LAUNCH_PLAIN = 2 };
 
 #define DDD_MAX_K 32          /* beam width limit                                  */
 #define DDD_MAX_DEPTH 32      /* check_mask has one bit per step                   */
@@ -198,11 +203,14 @@ int ddd_draft_host(ddd_handle *h, const void *root_hidden, const int32_t *root_t
 int ddd_lm_head_pass(ddd_handle *h, void *cuda_stream);
 
 /*
- * Number of kernels one ddd_draft enqueues (they all launch even if the gate stops early;
- * kernels of skipped passes exit at once), and the number of thread blocks the LM-head
- * kernel uses.  Pure host queries; negative on a NULL handle.
+ * ddd_launches_per_draft: kernels one ddd_draft launches when a sequence of the batch needs
+ * `passes_needed` LM-head passes (its largest stop depth).  Outside graph mode every pass is
+ * launched (kernels of passes after the stop exit at once); in graph mode the passes after the
+ * third are launched only if some sequence is still drafting then.
+ * ddd_lm_head_blocks: thread blocks of the LM-head kernel.
+ * Pure host queries; negative on a NULL handle.
  */
-int ddd_launches_per_draft(const ddd_handle *h);
+int ddd_launches_per_draft(const ddd_handle *h, int32_t passes_needed);
 int ddd_lm_head_blocks(const ddd_handle *h);
 
 /*

@@ -12,7 +12,7 @@ _lib = None
 
 DDD_DTYPE_FP32, DDD_DTYPE_BF16 = 0, 1
 DDD_LM_HEAD_AUTO, DDD_LM_HEAD_SIMT, DDD_LM_HEAD_TCGEN05 = 0, 1, 2
-DDD_LAUNCH_STREAM, DDD_LAUNCH_GRAPH = 0, 1
+DDD_LAUNCH_STREAM, DDD_LAUNCH_GRAPH, DDD_LAUNCH_PLAIN = 0, 1, 2
 
 
 class DddError(RuntimeError):
@@ -69,7 +69,7 @@ def load_library():
     lib.ddd_lm_head_pass.restype = ctypes.c_int
     lib.ddd_lm_head_pass.argtypes = [vp, vp]
     lib.ddd_launches_per_draft.restype = ctypes.c_int
-    lib.ddd_launches_per_draft.argtypes = [vp]
+    lib.ddd_launches_per_draft.argtypes = [vp, ctypes.c_int32]
     lib.ddd_lm_head_blocks.restype = ctypes.c_int
     lib.ddd_lm_head_blocks.argtypes = [vp]
     lib.ddd_lm_head_topk_noalloc.restype = ctypes.c_int
@@ -131,8 +131,8 @@ def ddd_lm_head_pass(handle: int, stream: int) -> None:
         raise DddError(rc, "ddd_lm_head_pass")
 
 
-def ddd_launches_per_draft(handle: int) -> int:
-    return int(load_library().ddd_launches_per_draft(handle))
+def ddd_launches_per_draft(handle: int, passes_needed: int) -> int:
+    return int(load_library().ddd_launches_per_draft(handle, int(passes_needed)))
 
 
 def ddd_lm_head_blocks(handle: int) -> int:

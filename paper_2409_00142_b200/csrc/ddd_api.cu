@@ -41,7 +41,7 @@ int validate(const ddd_config* c) {
   if (!(c->rms_eps >= 0.f)) return DDD_ERR_INVALID_ARG;
   if (c->device < 0) return DDD_ERR_INVALID_ARG;
   if (c->lm_head_kernel < DDD_LM_HEAD_AUTO || c->lm_head_kernel > DDD_LM_HEAD_TCGEN05) return DDD_ERR_INVALID_ARG;
-  if (c->launch_mode != DDD_LAUNCH_STREAM && c->launch_mode != DDD_LAUNCH_GRAPH) return DDD_ERR_INVALID_ARG;
+  if (c->launch_mode < DDD_LAUNCH_STREAM || c->launch_mode > DDD_LAUNCH_PLAIN) return DDD_ERR_INVALID_ARG;
   if (c->lm_head_kernel == DDD_LM_HEAD_TCGEN05 && (c->dtype != DDD_DTYPE_BF16 || c->hidden % 64 != 0))
     return DDD_ERR_UNSUPPORTED;
   return DDD_OK;
@@ -252,7 +252,7 @@ int ddd_create(const ddd_config* cfg, const void* W, const void* E, const float*
   h->ws = static_cast<unsigned char*>(workspace);
   h->sm_count = prop.multiProcessorCount;
   h->have_graph = false;
-  h->use_pdl = true;
+  h->use_pdl = cfg->launch_mode != DDD_LAUNCH_PLAIN;
   h->graph_pdl = false;
   h->exec = nullptr;
   h->bounce = nullptr;
@@ -428,9 +428,13 @@ int ddd_lm_head_pass(ddd_handle* h, void* cuda_stream) {
   return DDD_OK;
 }
 
-int ddd_launches_per_draft(const ddd_handle* h) {
+int ddd_launches_per_draft(const ddd_handle* h, int32_t passes_needed) {
   if (!h) return DDD_ERR_INVALID_ARG;
-  return 2 + 2 * h->p.n;   // init, (LM head + select) per pass, rerank
+  const int n = h->p.n;
+  int passes = n;
+  if (h->cfg.launch_mode == DDD_LAUNCH_GRAPH && n > kUnconditionalPasses + 1 && passes_needed <= kUnconditionalPasses)
+    passes = kUnconditionalPasses;
+  return 2 + 2 * passes;   // init, (LM head + select) per launched pass, rerank
 }
 
 int ddd_lm_head_blocks(const ddd_handle* h) {

@@ -63,7 +63,7 @@ def test_create_rejects_bad_arguments_without_a_device():
     assert lib.ddd_draft_host(None, fake, fake, fake, None, None) == -1
     assert lib.ddd_lm_head_pass(None, None) == -1
     assert lib.ddd_destroy(None) == -1
-    assert lib.ddd_launches_per_draft(None) < 0 and lib.ddd_lm_head_blocks(None) < 0
+    assert lib.ddd_launches_per_draft(None, 1) < 0 and lib.ddd_lm_head_blocks(None) < 0
 
 
 def test_strerror_covers_every_code():

@@ -138,6 +138,9 @@ def test_k1_greedy_chain_and_k_equal_to_limit():
 def test_graph_mode_host_variant_and_determinism():
     cfg = small_cases()["7b"]
     roots = S.make_roots(cfg, 1)
+    eng_p = engine_for(cfg, TC, P.DDD_LAUNCH_PLAIN)
+    a0 = parity.run_gpu(eng_p, roots)
+    eng_p.close()
     eng_s = engine_for(cfg, TC, P.DDD_LAUNCH_STREAM)
     a = parity.run_gpu(eng_s, roots)
     a2 = parity.run_gpu(eng_s, roots)
@@ -148,6 +151,7 @@ def test_graph_mode_host_variant_and_determinism():
         other = S.make_roots(cfg, 2)
         c = parity.run_gpu(eng_g, other)            # new input pointers: re-captured
     for name in a:
+        np.testing.assert_array_equal(a[name], a0[name], err_msg=name)    # plain launches == overlapped launches
         np.testing.assert_array_equal(a[name], a2[name], err_msg=name)    # run-to-run identical
         np.testing.assert_array_equal(a[name], b[name], err_msg=name)     # graph == stream
         np.testing.assert_array_equal(b[name], b2[name], err_msg=name)
@@ -158,7 +162,9 @@ def test_graph_mode_host_variant_and_determinism():
                      roots["root_pos"].pin_memory(), host_out)
     for name in host_out:
         np.testing.assert_array_equal(host_out[name].numpy(), a[name], err_msg=name)
-    assert P.ddd_launches_per_draft(eng_s.handle) == 2 + 2 * cfg.max_depth
+    assert P.ddd_launches_per_draft(eng_s.handle, 1) == 2 + 2 * cfg.max_depth
+    assert P.ddd_launches_per_draft(eng_g.handle, 2) == 2 + 2 * 3
+    assert P.ddd_launches_per_draft(eng_g.handle, 4) == 2 + 2 * cfg.max_depth
     assert 1 <= P.ddd_lm_head_blocks(eng_s.handle) <= 512
     eng_s.close()
     eng_g.close()
