@@ -323,6 +323,37 @@ def main():
                     ex.close()
                 extra["threshold_sweep"] = sweep
 
+        # ---- where the gate lives: the paper checks the heuristic on the host after a synchronisation
+        # (Section 2; its "Strict" variants of Section 3.4 do so after every draft call); here the check
+        # is on the device.  Same drafts, same results, host-gated: launch pass, synchronise, read, decide.
+        if not args.no_sweep:
+            def host_gated_rate(engine, reps):
+                for r in roots_dev[:4]:
+                    engine.draft_host_gated(r["root_hidden"], r["root_token"], r["root_pos"])
+                torch.cuda.synchronize(device)
+                t0 = time.perf_counter()
+                for _ in range(reps):
+                    for r in roots_dev:
+                        engine.draft_host_gated(r["root_hidden"], r["root_token"], r["root_pos"])
+                torch.cuda.synchronize(device)
+                return reps * n_per_rank * cfg.batch / (time.perf_counter() - t0)
+
+            reps = max(2, args.steps // 20)
+            extra["gate_placement"] = {"device_gate_drafts_per_sec": value,
+                                       "host_gate_drafts_per_sec": host_gated_rate(eng, reps),
+                                       "note": "per rank; host gate = stream sync + 4-byte read after every pass"}
+            # the paper's own parameters (Section 3.2): n = 11, S = {5, 7, 9}, x = -0.3, w = 10
+            pmask = sum(1 << (s_ - 1) for s_ in (5, 7, 9))
+            pcfg = cfg.replace(max_depth=11, check_mask=pmask, threshold=-0.3, k=10)
+            pe = P.DraftEngine(pcfg, {"W": eng.W, "E": eng.E, "bias": eng.bias, "plant_next": eng.plant_next},
+                               device=local, launch_mode=mode, with_trace=False)
+            pdm = _mean(mean_stop_depth(pe, roots_dev, device))
+            pms, _ = timed_drafts(pe, roots_dev, max(3, args.steps // 4), args.warmup, world, device)
+            extra["paper_parameters"] = {"n": 11, "S": [5, 7, 9], "x": -0.3, "w": 10, "mean_stop_depth": pdm,
+                                         "device_gate_drafts_per_sec": drafts_total / (pms / 1e3),
+                                         "host_gate_drafts_per_sec": host_gated_rate(pe, reps)}
+            pe.close()
+
         # ---- end to end through the host-buffer entry point (pinned host memory, copies inside)
         host_out = eng.make_host_out(pinned=True)
         pinned = [{k: v.pin_memory() for k, v in r.items()} for r in roots_host]

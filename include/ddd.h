@@ -184,6 +184,18 @@ int ddd_draft(ddd_handle *h, const void *root_hidden, const int32_t *root_token,
               void *cuda_stream);
 
 /*
+ * The same draft the way the paper runs it (Section 2, Section 3.4 "Strict"): after every
+ * LM-head pass the HOST synchronises the stream, reads how many sequences are still drafting
+ * and only then launches the next pass.  Arguments and results are those of ddd_draft (DEVICE
+ * buffers); the call returns after the rerank has been enqueued, with *passes_run (HOST, may be
+ * NULL) = number of passes launched.  It exists to measure what the device-resident gate of
+ * ddd_draft saves; results are identical.  Errors: INVALID_ARG, ALIGNMENT, CUDA.
+ */
+int ddd_draft_host_gated(ddd_handle *h, const void *root_hidden, const int32_t *root_token,
+                         const int32_t *root_pos, const ddd_output *out, const ddd_trace *trace,
+                         void *cuda_stream, int32_t *passes_run);
+
+/*
  * Same draft with HOST buffers: copies the inputs to staging space inside the workspace,
  * runs the draft, copies every ddd_output field back and synchronises the stream before
  * returning.  All pointers (inputs and the fields of `out`) are HOST pointers; pinned

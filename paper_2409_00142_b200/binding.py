@@ -64,6 +64,9 @@ def load_library():
                                ctypes.POINTER(ctypes.c_void_p)]
     lib.ddd_draft.restype = ctypes.c_int
     lib.ddd_draft.argtypes = [vp, vp, i32p, i32p, ctypes.POINTER(DddOutput), ctypes.POINTER(DddTrace), vp]
+    lib.ddd_draft_host_gated.restype = ctypes.c_int
+    lib.ddd_draft_host_gated.argtypes = [vp, vp, i32p, i32p, ctypes.POINTER(DddOutput), ctypes.POINTER(DddTrace), vp,
+                                         ctypes.POINTER(ctypes.c_int32)]
     lib.ddd_draft_host.restype = ctypes.c_int
     lib.ddd_draft_host.argtypes = [vp, vp, i32p, i32p, ctypes.POINTER(DddOutput), vp]
     lib.ddd_lm_head_pass.restype = ctypes.c_int
@@ -85,7 +88,7 @@ def load_library():
 
 def exported_symbols():
     """Names this binding expects the library to export (all of include/ddd.h)."""
-    return ["ddd_workspace_bytes", "ddd_create", "ddd_draft", "ddd_draft_host", "ddd_lm_head_pass",
+    return ["ddd_workspace_bytes", "ddd_create", "ddd_draft", "ddd_draft_host", "ddd_draft_host_gated", "ddd_lm_head_pass",
             "ddd_launches_per_draft", "ddd_lm_head_blocks", "ddd_lm_head_topk_noalloc", "ddd_destroy",
             "ddd_strerror"]
 
@@ -116,6 +119,19 @@ def ddd_draft(handle: int, root_hidden: int, root_token: int, root_pos: int, out
                                   ctypes.byref(trace) if trace is not None else None, stream)
     if rc != 0:
         raise DddError(rc, "ddd_draft")
+
+
+def ddd_draft_host_gated(handle: int, root_hidden: int, root_token: int, root_pos: int, out: DddOutput,
+                         trace: Optional[DddTrace], stream: int) -> int:
+    """The paper's control flow: a host synchronisation and decision after every pass.  Returns the
+    number of passes launched."""
+    n = ctypes.c_int32(0)
+    rc = load_library().ddd_draft_host_gated(handle, root_hidden, root_token, root_pos, ctypes.byref(out),
+                                             ctypes.byref(trace) if trace is not None else None, stream,
+                                             ctypes.byref(n))
+    if rc != 0:
+        raise DddError(rc, "ddd_draft_host_gated")
+    return int(n.value)
 
 
 def ddd_draft_host(handle: int, root_hidden: int, root_token: int, root_pos: int, out: DddOutput,
@@ -228,6 +244,11 @@ class DraftEngine:
         assert root_pos.is_cuda and root_pos.dtype == self.torch.int32
         ddd_draft(self.handle, root_hidden.data_ptr(), root_token.data_ptr(), root_pos.data_ptr(),
                   self.c_out, self.c_trace, self.stream_ptr())
+
+    def draft_host_gated(self, root_hidden, root_token, root_pos) -> int:
+        """Like draft(), but the host waits and decides after every pass (the paper's "Strict" flow)."""
+        return ddd_draft_host_gated(self.handle, root_hidden.data_ptr(), root_token.data_ptr(), root_pos.data_ptr(),
+                                    self.c_out, self.c_trace, self.stream_ptr())
 
     def draft_host(self, root_hidden, root_token, root_pos, host_out: Dict) -> None:
         """Host-buffer variant: CPU tensors in, CPU tensors (same names as self.out) out."""

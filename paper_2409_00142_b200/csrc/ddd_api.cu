@@ -356,6 +356,37 @@ int ddd_draft(ddd_handle* h, const void* root_hidden, const int32_t* root_token,
   return DDD_OK;
 }
 
+int ddd_draft_host_gated(ddd_handle* h, const void* root_hidden, const int32_t* root_token, const int32_t* root_pos,
+                         const ddd_output* out, const ddd_trace* trace, void* cuda_stream, int32_t* passes_run) {
+  if (passes_run) *passes_run = 0;
+  if (!h || !root_hidden || !root_token || !root_pos || !out) return DDD_ERR_INVALID_ARG;
+  if (!out->n_out || !out->stop_depth || !out->token || !out->parent || !out->depth || !out->position ||
+      !out->cum || !out->mask || !out->H_trace || !out->status)
+    return DDD_ERR_INVALID_ARG;
+  if (!aligned16(root_hidden)) return DDD_ERR_ALIGNMENT;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  DraftIO io;
+  io.out = *out;
+  if (trace) io.trace = *trace; else std::memset(&io.trace, 0, sizeof io.trace);
+  cudaError_t e = launch_init(h->p, io, root_hidden, root_token, root_pos, st);
+  int d = 1;
+  for (; d <= h->p.n && e == cudaSuccess; ++d) {
+    e = enqueue_passes(h, io, h->use_pdl, d, d, 0, 0, st);
+    // the host decides: wait for the pass, read how many sequences are still drafting
+    int still = 0;
+    if (e == cudaSuccess) e = cudaMemcpyAsync(&still, h->p.n_active, sizeof still, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess || still == 0) break;
+  }
+  if (passes_run) *passes_run = d <= h->p.n ? d : h->p.n;
+  if (e == cudaSuccess) e = launch_rerank(h->p, io, false, st);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return DDD_ERR_CUDA;
+  }
+  return DDD_OK;
+}
+
 int ddd_draft_host(ddd_handle* h, const void* root_hidden, const int32_t* root_token, const int32_t* root_pos,
                    const ddd_output* out, void* cuda_stream) {
   if (!h || !root_hidden || !root_token || !root_pos || !out) return DDD_ERR_INVALID_ARG;

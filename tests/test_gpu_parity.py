@@ -170,6 +170,22 @@ def test_graph_mode_host_variant_and_determinism():
     eng_g.close()
 
 
+def test_host_gated_draft_equals_device_gated_draft():
+    # the paper's control flow (host sync and decision after every pass) must give the same tree
+    cfg = small_cases()["7b"]
+    eng = engine_for(cfg, TC, P.DDD_LAUNCH_STREAM)
+    for i in (0, 3):
+        roots = S.make_roots(cfg, i)
+        a = parity.run_gpu(eng, roots)
+        dev = parity.to_device(roots, eng.device)
+        passes = eng.draft_host_gated(dev["root_hidden"], dev["root_token"], dev["root_pos"])
+        b = {k: v.numpy() for k, v in eng.results().items()}
+        assert passes == int(a["stop_depth"].max())
+        for name in a:
+            np.testing.assert_array_equal(a[name], b[name], err_msg=name)
+    eng.close()
+
+
 def test_simt_and_tensor_core_kernels_agree():
     cfg = small_cases()["70b_batch"]
     roots = S.make_roots(cfg, 5)
