@@ -3,6 +3,7 @@
 // variant.  No device memory is allocated here; the only allocation is a small pinned host
 // bounce buffer used by ddd_draft_host.
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 
@@ -12,6 +13,13 @@
 using namespace ddd;
 
 namespace {
+
+// Clears the sticky CUDA error; with DDD_DEBUG set in the environment, says what it was.
+void note_cuda_error(int line) {
+  const cudaError_t e = cudaGetLastError();
+  static const bool verbose = std::getenv("DDD_DEBUG") != nullptr;
+  if (verbose) std::fprintf(stderr, "[ddd] CUDA failure near ddd_api.cu:%d: %s\n", line, cudaGetErrorString(e));
+}
 
 constexpr size_t kAlign = 256;
 size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
@@ -166,20 +174,22 @@ bool capture_graph(ddd_handle* h, const DraftIO& io, bool pdl, cudaStream_t st) 
   const int head = n <= kUnconditionalPasses + 1 ? n : kUnconditionalPasses;   // passes outside the conditional
   cudaGraph_t graph = nullptr, body = nullptr;
   cudaGraphConditionalHandle cond = 0;
-  bool ok = cudaGraphCreate(&graph, 0) == cudaSuccess;
-  if (ok && head < n) ok = cudaGraphConditionalHandleCreate(&cond, graph, 0, cudaGraphCondAssignDefault) == cudaSuccess;
+  int step = 0;   // which call failed, for the diagnostic
+  auto good = [&](cudaError_t e, int id) { if (e != cudaSuccess && step == 0) step = id; return e == cudaSuccess; };
+  bool ok = good(cudaGraphCreate(&graph, 0), 1);
+  if (ok && head < n) ok = good(cudaGraphConditionalHandleCreate(&cond, graph, 0, cudaGraphCondAssignDefault), 2);
   bool capturing = false;
   if (ok) {
-    ok = cudaStreamBeginCaptureToGraph(st, graph, nullptr, nullptr, 0, cudaStreamCaptureModeThreadLocal) == cudaSuccess;
+    ok = good(cudaStreamBeginCaptureToGraph(st, graph, nullptr, nullptr, 0, cudaStreamCaptureModeThreadLocal), 3);
     capturing = ok;
   }
-  if (ok) ok = enqueue_passes(h, io, pdl, 1, head, cond, head < n ? head : 0, st) == cudaSuccess;
+  if (ok) ok = good(enqueue_passes(h, io, pdl, 1, head, cond, head < n ? head : 0, st), 4);
   if (ok && head < n) {
     // splice an IF node between the captured passes and the rerank
     cudaStreamCaptureStatus status;
     const cudaGraphNode_t* deps = nullptr;
     size_t n_deps = 0;
-    ok = cudaStreamGetCaptureInfo(st, &status, nullptr, nullptr, &deps, &n_deps) == cudaSuccess &&
+    ok = good(cudaStreamGetCaptureInfo(st, &status, nullptr, nullptr, &deps, &n_deps), 5) &&
          status == cudaStreamCaptureStatusActive;
     cudaGraphNode_t node = nullptr;
     if (ok) {
@@ -188,29 +198,29 @@ bool capture_graph(ddd_handle* h, const DraftIO& io, bool pdl, cudaStream_t st) 
       np.conditional.handle = cond;
       np.conditional.type = cudaGraphCondTypeIf;
       np.conditional.size = 1;
-      ok = cudaGraphAddNode(&node, graph, deps, n_deps, &np) == cudaSuccess;
+      ok = good(cudaGraphAddNode(&node, graph, deps, n_deps, &np), 6);
       if (ok) body = np.conditional.phGraph_out[0];
     }
-    if (ok) ok = cudaStreamUpdateCaptureDependencies(st, &node, 1, cudaStreamSetCaptureDependencies) == cudaSuccess;
+    if (ok) ok = good(cudaStreamUpdateCaptureDependencies(st, &node, 1, cudaStreamSetCaptureDependencies), 7);
   }
   // the rerank follows a conditional node, not a kernel: plain dependency
-  if (ok) ok = launch_rerank(h->p, io, pdl && head == n, st) == cudaSuccess;
+  if (ok) ok = good(launch_rerank(h->p, io, pdl && head == n, st), 8);
   if (capturing) {
     cudaGraph_t done = nullptr;
-    if (cudaStreamEndCapture(st, &done) != cudaSuccess) ok = false;
+    if (!good(cudaStreamEndCapture(st, &done), 9)) ok = false;
   }
   if (ok && body) {
-    ok = cudaStreamBeginCaptureToGraph(st, body, nullptr, nullptr, 0, cudaStreamCaptureModeThreadLocal) == cudaSuccess;
+    ok = good(cudaStreamBeginCaptureToGraph(st, body, nullptr, nullptr, 0, cudaStreamCaptureModeThreadLocal), 10);
     if (ok) {
-      if (enqueue_passes(h, io, pdl, head + 1, n, cond, 0, st) != cudaSuccess) ok = false;
+      if (!good(enqueue_passes(h, io, pdl, head + 1, n, cond, 0, st), 11)) ok = false;
       cudaGraph_t done = nullptr;
-      if (cudaStreamEndCapture(st, &done) != cudaSuccess) ok = false;
+      if (!good(cudaStreamEndCapture(st, &done), 12)) ok = false;
     }
   }
-  if (ok) ok = cudaGraphInstantiate(&h->exec, graph, 0) == cudaSuccess;
+  if (ok) ok = good(cudaGraphInstantiate(&h->exec, graph, 0), 13);
   if (graph) cudaGraphDestroy(graph);
   if (!ok) {
-    cudaGetLastError();
+    note_cuda_error(1000 + step);   // 1000 + index of the capture step that failed
     h->exec = nullptr;
     return false;
   }
@@ -307,7 +317,7 @@ int ddd_create(const ddd_config* cfg, const void* W, const void* E, const float*
   }
   if (rc == DDD_OK && prepare_tree(p) != cudaSuccess) rc = DDD_ERR_CUDA;
   if (rc != DDD_OK) {
-    cudaGetLastError();
+    note_cuda_error(__LINE__);
     delete h;
     return rc;
   }
@@ -342,7 +352,7 @@ int ddd_draft(ddd_handle* h, const void* root_hidden, const int32_t* root_token,
     }
     if (launch_init(h->p, io, root_hidden, root_token, root_pos, st) != cudaSuccess ||
         cudaGraphLaunch(h->exec, st) != cudaSuccess) {
-      cudaGetLastError();
+      note_cuda_error(__LINE__);
       return DDD_ERR_CUDA;
     }
     return DDD_OK;
@@ -350,7 +360,7 @@ int ddd_draft(ddd_handle* h, const void* root_hidden, const int32_t* root_token,
   if (launch_init(h->p, io, root_hidden, root_token, root_pos, st) != cudaSuccess ||
       enqueue_passes(h, io, h->use_pdl, 1, h->p.n, 0, 0, st) != cudaSuccess ||
       launch_rerank(h->p, io, h->use_pdl, st) != cudaSuccess) {
-    cudaGetLastError();
+    note_cuda_error(__LINE__);
     return DDD_ERR_CUDA;
   }
   return DDD_OK;
@@ -381,7 +391,7 @@ int ddd_draft_host_gated(ddd_handle* h, const void* root_hidden, const int32_t* 
   if (passes_run) *passes_run = d <= h->p.n ? d : h->p.n;
   if (e == cudaSuccess) e = launch_rerank(h->p, io, false, st);
   if (e != cudaSuccess) {
-    cudaGetLastError();
+    note_cuda_error(__LINE__);
     return DDD_ERR_CUDA;
   }
   return DDD_OK;
@@ -399,7 +409,7 @@ int ddd_draft_host(ddd_handle* h, const void* root_hidden, const int32_t* root_t
   const size_t need = (L.in_bytes > L.out_bytes ? L.in_bytes : L.out_bytes);
   if (!h->bounce) {
     if (cudaMallocHost(reinterpret_cast<void**>(&h->bounce), need) != cudaSuccess) {
-      cudaGetLastError();
+      note_cuda_error(__LINE__);
       return DDD_ERR_CUDA;
     }
     h->bounce_bytes = need;
@@ -411,7 +421,7 @@ int ddd_draft_host(ddd_handle* h, const void* root_hidden, const int32_t* root_t
   std::memcpy(h->bounce + (L.in_token - L.in_hidden), root_token, B * 4);
   std::memcpy(h->bounce + (L.in_pos - L.in_hidden), root_pos, B * 4);
   if (cudaMemcpyAsync(h->ws + L.in_hidden, h->bounce, L.in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) {
-    cudaGetLastError();
+    note_cuda_error(__LINE__);
     return DDD_ERR_CUDA;
   }
   unsigned char* ob = h->ws + L.out_block;
@@ -432,7 +442,7 @@ int ddd_draft_host(ddd_handle* h, const void* root_hidden, const int32_t* root_t
   // one device-to-host copy of the packed results, then scatter to the caller's arrays
   if (cudaMemcpyAsync(h->bounce, ob, L.out_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
       cudaStreamSynchronize(st) != cudaSuccess) {
-    cudaGetLastError();
+    note_cuda_error(__LINE__);
     return DDD_ERR_CUDA;
   }
   const unsigned char* hb = h->bounce;
@@ -453,7 +463,7 @@ int ddd_lm_head_pass(ddd_handle* h, void* cuda_stream) {
   if (!h) return DDD_ERR_INVALID_ARG;
   // Pass index 2 selects the hidden buffer written by the first draft step; all rows are forced live.
   if (launch_lm_head(h, 2, 1, h->use_pdl, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) {
-    cudaGetLastError();
+    note_cuda_error(__LINE__);
     return DDD_ERR_CUDA;
   }
   return DDD_OK;

@@ -177,6 +177,21 @@ __device__ __forceinline__ void row_tile_update(const float* zrow, int tok0, int
 }
 
 // ---------------------------------------------------------------------------- launchers (host)
+// Lets a kernel use as much dynamic shared memory as the device allows.  The limit is a
+// property of the function, shared by every handle of the process, so it is set to the
+// maximum rather than to one handle's need (a later, smaller handle would otherwise lower it
+// under an earlier one).
+template <typename Kernel>
+inline cudaError_t allow_max_dynamic_smem(Kernel kernel) {
+  int dev = 0, optin = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+  cudaFuncAttributes fa;
+  if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa, kernel);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, optin - (int)fa.sharedSizeBytes);
+}
+
 // Each returns the cudaError_t of its launch / attribute call.
 cudaError_t prepare_simt(const Params& p);
 cudaError_t prepare_tree(const Params& p);

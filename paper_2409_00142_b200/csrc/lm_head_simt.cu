@@ -136,12 +136,10 @@ size_t simt_smem(const Params& p) {
 }  // namespace
 
 cudaError_t prepare_simt(const Params& p) {
-  const int smem = (int)simt_smem(p);
-  cudaError_t e = cudaFuncSetAttribute(lm_head_simt_kernel<float>,
-                                       cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (simt_smem(p) > 200 * 1024) return cudaErrorInvalidValue;
+  cudaError_t e = allow_max_dynamic_smem(lm_head_simt_kernel<float>);
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(lm_head_simt_kernel<__nv_bfloat16>,
-                              cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  return allow_max_dynamic_smem(lm_head_simt_kernel<__nv_bfloat16>);
 }
 
 cudaError_t launch_lm_head_simt(const Params& p, int d, int force_all, int ctas, cudaStream_t st) {

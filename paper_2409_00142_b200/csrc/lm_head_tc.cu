@@ -578,9 +578,7 @@ int tc_plan_create(const Params& p, int sm_count, void* w_packed, TcPlan* plan) 
   for (int i = 0; i < 2; ++i)
     if (!encode_hidden_3d(&plan->map_h[i], p.hbuf[i], (uint64_t)p.R, (uint64_t)p.Hd, (uint32_t)n_pad, (uint32_t)ksub))
       return DDD_ERR_CUDA;
-  if (cudaFuncSetAttribute(lm_head_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan->smem) !=
-      cudaSuccess)
-    return DDD_ERR_CUDA;
+  if (allow_max_dynamic_smem(lm_head_tc_kernel) != cudaSuccess) return DDD_ERR_CUDA;
   return DDD_OK;
 }
 

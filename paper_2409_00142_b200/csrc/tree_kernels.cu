@@ -761,11 +761,10 @@ size_t rerank_smem(const Params& p) { return (size_t)p.Nn * (sizeof(uint32_t) + 
 
 // ---------------------------------------------------------------------------- launchers
 cudaError_t prepare_tree(const Params& p) {
-  cudaError_t e = cudaFuncSetAttribute(select_gate_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)select_smem(p));
+  if (select_smem(p) > 180 * 1024 || rerank_smem(p) > 200 * 1024) return cudaErrorInvalidValue;
+  cudaError_t e = allow_max_dynamic_smem(select_gate_step_kernel);
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(rerank_mask_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              (int)rerank_smem(p));
+  return allow_max_dynamic_smem(rerank_mask_kernel);
 }
 
 cudaError_t launch_init(const Params& p, const DraftIO&, const void* root_hidden, const int* root_token,

@@ -170,6 +170,22 @@ def test_graph_mode_host_variant_and_determinism():
     eng_g.close()
 
 
+def test_handles_of_different_sizes_coexist():
+    # kernel attributes (dynamic shared memory limit) are per process: a smaller handle created
+    # later must not take room away from a larger one created earlier
+    big = small_cases()["128k_zipf"]
+    small = big.replace(k=2, max_depth=2, total_tokens=3)
+    eng_big = engine_for(big, TC)
+    eng_small = engine_for(small, TC)
+    roots = S.make_roots(big, 0)
+    g = parity.run_gpu(eng_big, roots)
+    parity.compare_with_oracle(big, weights_for(big), roots, g)
+    g2 = parity.run_gpu(eng_small, S.make_roots(small, 0))
+    parity.compare_with_oracle(small, weights_for(small), S.make_roots(small, 0), g2)
+    eng_big.close()
+    eng_small.close()
+
+
 def test_host_gated_draft_equals_device_gated_draft():
     # the paper's control flow (host sync and decision after every pass) must give the same tree
     cfg = small_cases()["7b"]
