@@ -134,6 +134,32 @@ def test_k1_greedy_chain_and_k_equal_to_limit():
             eng.close()
 
 
+def edge_cases():
+    base = S.scaled_down(S.CONFIGS["llama2_7b"], 128, 1000, threshold=NEG)
+    return {
+        "single_pass": base.replace(max_depth=1, total_tokens=20),                 # n = 1: no draft step at all
+        "m_exceeds_tree": base.replace(k=3, max_depth=2, total_tokens=50),         # fewer nodes than m: padded rows
+        "vocab_just_above_k": base.replace(vocab=40, k=8, max_depth=3, total_tokens=30),
+        "odd_vocab": base.replace(vocab=1001, k=5, max_depth=3, total_tokens=25),  # not a multiple of 8 or 32
+        "hidden_64": S.scaled_down(S.CONFIGS["llama2_7b"], 64, 700, threshold=NEG, k=6, max_depth=3, total_tokens=20),
+        "rows_256": base.replace(batch=8, k=32, max_depth=2, total_tokens=100),    # B * k at its limit
+        "mask_1024_rows": base.replace(k=32, max_depth=3, total_tokens=1023),      # widest mask: 32 words per row
+        "one_token": base.replace(k=2, max_depth=4, total_tokens=1),
+    }
+
+
+@pytest.mark.parametrize("kernel", [SIMT, TC], ids=["simt", "tcgen05"])
+@pytest.mark.parametrize("case", list(edge_cases()))
+def test_edge_shapes_match_oracle(case, kernel):
+    cfg = edge_cases()[case]
+    eng = engine_for(cfg, kernel)
+    for i in range(2):
+        roots = S.make_roots(cfg, i)
+        g = parity.run_gpu(eng, roots)
+        parity.compare_with_oracle(cfg, weights_for(cfg), roots, g)
+    eng.close()
+
+
 # ----------------------------------------------------------------------------- launch modes
 def test_graph_mode_host_variant_and_determinism():
     cfg = small_cases()["7b"]
