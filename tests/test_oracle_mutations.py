@@ -1,0 +1,106 @@
+"""The pins must notice plausible mistakes: each case below plants one mistake in the CPU
+oracle (never in the CUDA path) and expects a named pin from test_oracle_pins.py to fail."""
+import math
+
+import numpy as np
+import pytest
+
+from oracle import ddd_oracle as O
+from tests import test_oracle_pins as pins
+
+
+def _h_mean(logprobsum):                      # Eq. 1 with a mean instead of a sum
+    a = np.asarray(logprobsum, dtype=np.float64)
+    return float(a.max() + math.log(np.exp(a - a.max()).mean()))
+
+
+def _h_extra_term(logprobsum):                # the garbled upper bound taken literally: w + 1 terms
+    a = np.append(np.asarray(logprobsum, dtype=np.float64), 0.0)
+    return float(a.max() + math.log(np.exp(a - a.max()).sum()))
+
+
+def _topk_high_index_first(scores, k):        # ties resolved towards the larger index
+    s = np.asarray(scores, dtype=np.float64)
+    return np.lexsort((-np.arange(len(s)), -s))[:k]
+
+
+def _softmax_unnormalised(z_row):             # forgets the log-sum-exp
+    return np.minimum(z_row - z_row.max(), 0.0)
+
+
+def _step_eps_outside(h_parent, e_row, eps, dtype):
+    u = h_parent + e_row
+    return O.round_to_storage(u / (math.sqrt(float(np.mean(u * u))) + 1.0), dtype)
+
+
+def _step_no_embedding(h_parent, e_row, eps, dtype):
+    u = h_parent
+    return O.round_to_storage(u / math.sqrt(float(np.mean(u * u)) + eps), dtype)
+
+
+def _mask_without_self(parent_slot):
+    rows = []
+    for i, p in enumerate(parent_slot):
+        rows.append(1 if p < 0 else (rows[p] | (1 << p)))
+    return rows
+
+
+def _rerank_lowest(cum, m):                   # keeps the worst nodes
+    n = len(cum)
+    return np.sort(O.topk_desc(-np.asarray(cum), min(m, n)) + 1)
+
+
+def _plant_added(z_row, column, delta):       # adds delta to the column instead of replacing it
+    z_row = z_row.copy()
+    if column >= 0:
+        z_row[column] += delta
+    return z_row
+
+
+def _logits_transposed_scale(W, h, scale, bias):   # scale applied to the bias as well
+    z = ORIG["lm_head_logits"](W, h, 1.0, bias)
+    return scale * z
+
+
+ORIG = {name: getattr(O, name) for name in (
+    "heuristic_H", "topk_desc", "log_softmax_row", "draft_step", "tree_mask_rows", "rerank", "apply_plant",
+    "lm_head_logits")}
+
+CASES = [
+    ("heuristic_H", _h_mean, pins.test_uniform_closed_form_H_and_tiebreaks, ()),
+    ("heuristic_H", _h_extra_term, pins.test_greedy_chain_k1, ()),
+    ("topk_desc", _topk_high_index_first, pins.test_topk_desc_ties_and_order, ()),
+    ("topk_desc", _topk_high_index_first, pins.test_uniform_closed_form_H_and_tiebreaks, ()),
+    ("log_softmax_row", _softmax_unnormalised, pins.test_log_softmax_invariants_and_library, ()),
+    ("log_softmax_row", _softmax_unnormalised, pins.test_tree_scores_equal_brute_force_path_table, (5, 3, 3, "fp32")),
+    ("draft_step", _step_eps_outside, pins.test_draft_step_textbook_rmsnorm, ()),
+    ("draft_step", _step_no_embedding, pins.test_tree_scores_equal_brute_force_path_table, (5, 3, 3, "fp32")),
+    ("tree_mask_rows", _mask_without_self, pins.test_mask_two_constructions_agree, ()),
+    ("rerank", _rerank_lowest, pins.test_rerank_plain_definition_and_invariants, ()),
+    ("apply_plant", _plant_added, pins.test_plant_closed_form, ()),
+    ("lm_head_logits", _logits_transposed_scale, pins.test_logits_match_library_matmul, ("bf16",)),
+]
+
+
+@pytest.mark.parametrize("name,mutant,pin,args", CASES,
+                         ids=[f"{c[0]}:{c[1].__name__}->{c[2].__name__}" for c in CASES])
+def test_pin_catches_planted_mistake(monkeypatch, name, mutant, pin, args):
+    pin(*args)                                   # green on the real oracle
+    monkeypatch.setattr(O, name, mutant)
+    with pytest.raises(AssertionError):
+        pin(*args)
+
+
+def test_gate_strictness_mistake_is_caught(monkeypatch):
+    # "H <= x" instead of "H < x": the equality case of the hand-threshold pin must fail.
+    src = O.draft.__code__
+    real = O.heuristic_H
+
+    def nudged(logprobsum):                      # makes H a hair smaller, so that H == x turns into H < x
+        return np.nextafter(real(logprobsum), -np.inf)
+
+    pins.test_stop_depth_against_hand_thresholds()
+    monkeypatch.setattr(O, "heuristic_H", nudged)
+    with pytest.raises(AssertionError):
+        pins.test_stop_depth_against_hand_thresholds()
+    assert O.draft.__code__ is src
