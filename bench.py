@@ -55,6 +55,8 @@ def parse_args():
     ap.add_argument("--cpu-sample", type=int, default=None, help="drafts the CPU baseline times")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true")
+    ap.add_argument("--width-sweep", action="store_true",
+                    help="also time fixed-depth-6 drafts at beam widths 5, 10, 20, 32 (cf. the paper's appendix)")
     ap.add_argument("--launch-mode", default="graph", choices=["graph", "stream", "plain"],
                     help="plain: ordinary stream-ordered launches, the mode profilers can follow")
     return ap.parse_args()
@@ -353,6 +355,18 @@ def main():
                                          "device_gate_drafts_per_sec": drafts_total / (pms / 1e3),
                                          "host_gate_drafts_per_sec": host_gated_rate(pe, reps)}
             pe.close()
+
+        # ---- beam width vs run time at fixed depth 6 (the paper's appendix reports an almost flat curve)
+        if args.width_sweep:
+            sweep_w = {}
+            for kw in (5, 10, 20, 32):
+                wc = cfg.replace(k=kw, max_depth=6, threshold=NEG, total_tokens=60)
+                we = P.DraftEngine(wc, {"W": eng.W, "E": eng.E, "bias": eng.bias, "plant_next": eng.plant_next},
+                                   device=local, launch_mode=mode, with_trace=False)
+                wms, _ = timed_drafts(we, roots_dev, max(3, args.steps // 8), args.warmup, world, device)
+                sweep_w[str(kw)] = {"us_per_draft": 1e3 * wms / n_per_rank, "us_per_expansion_step": 1e3 * wms / n_per_rank / 6}
+                we.close()
+            extra["beam_width_sweep_depth6"] = sweep_w
 
         # ---- end to end through the host-buffer entry point (pinned host memory, copies inside)
         host_out = eng.make_host_out(pinned=True)
