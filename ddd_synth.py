@@ -2,8 +2,9 @@
 
 This module only *draws numbers*: weights, embeddings, biases, planted-token
 tables and per-draft roots, each rounded to the storage dtype of the
-configuration.  It contains none of the method's arithmetic (no logits, no
-softmax, no top-k, no tree logic), so both the CPU oracle and the CUDA path can
+configuration, plus random tree shapes and target choices for the verification
+helpers.  It contains none of the method's arithmetic (no logits, no
+softmax, no top-k, no search and no acceptance logic), so both the CPU oracle and the CUDA path can
 be fed from it without sharing any computation.
 
 The paper evaluates on MT-bench with Vicuna / LLaMA2-Chat targets and trained
@@ -165,6 +166,40 @@ def make_roots(cfg: DraftConfig, draft_index: int) -> Dict[str, torch.Tensor]:
         "root_token": torch.from_numpy(tok),
         "root_pos": torch.from_numpy(pos),
     }
+
+
+def random_tree(rng: np.random.Generator, n_rows: int, vocab: int, max_children: int = 4):
+    """A random emitted tree for the verification helpers: rows in generation order (row 0 the
+    root, every parent row below its child's), the tokens of siblings distinct.
+    Returns (token [n_rows], parent [n_rows]) as int64 arrays."""
+    max_children = min(max_children, vocab)
+    parent, token = [-1], [int(rng.integers(vocab))]
+    used = {0: set()}
+    for i in range(1, n_rows):
+        while True:
+            p = int(rng.integers(i))
+            if len(used[p]) < max_children:
+                break
+        t = int(rng.integers(vocab))
+        while t in used[p]:
+            t = int(rng.integers(vocab))
+        used[p].add(t)
+        used[i] = set()
+        parent.append(p)
+        token.append(t)
+    return np.array(token, dtype=np.int64), np.array(parent, dtype=np.int64)
+
+
+def target_choices_along(rng: np.random.Generator, token, parent, n_rows: int, goal_row: int, vocab: int):
+    """Synthetic target choices [n_rows] for a tree: along the root path of `goal_row` the target
+    picks the path's next token, everywhere else a random token of the vocabulary (which may or
+    may not be some child's token)."""
+    target = rng.integers(vocab, size=n_rows).astype(np.int64)
+    r = int(goal_row)
+    while r > 0:
+        target[int(parent[r])] = int(token[r])
+        r = int(parent[r])
+    return target
 
 
 def shard_draft_indices(n_drafts: int, rank: int, world_size: int):

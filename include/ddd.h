@@ -257,6 +257,48 @@ int ddd_lm_head_topk_noalloc(const void *W, const float *bias, const void *hidde
                              int32_t rows, int32_t hidden, int32_t vocab, int32_t k, float logit_scale,
                              int32_t *out_token, float *out_logprob, float *out_lse, void *cuda_stream);
 
+/*
+ * What the verification step needs from a finished tree.  With T = t_rows and L = max_depth + 1,
+ * per sequence b (all DEVICE pointers, all required):
+ *   n_accepted[b]        draft tokens the greedy walk accepted (0..max_depth)
+ *   accepted_rows[b][j]  output row of the j-th accepted token, j < n_accepted; -1 after that
+ *   next_token[b]        the target's token after the last accepted row (the token that is
+ *                        always gained, even when no draft token is accepted)
+ *   n_leaves[b]          rows of the tree without a child among the emitted rows
+ *   leaf_paths[b][l][j]  for the l-th leaf in ascending row order, the rows from the root
+ *                        (j = 0, always row 0) down to the leaf; -1 after the leaf and in
+ *                        the rows l >= n_leaves
+ *   status[0]            DDD_OK, or DDD_ERR_INVALID_ARG if some sequence's rows were not a tree
+ *                        (a parent index not below its child's, or a path longer than L); that
+ *                        sequence then reports 0 accepted, next_token -1 and 0 leaves
+ */
+typedef struct {
+  int32_t *n_accepted;    /* [B]            */
+  int32_t *accepted_rows; /* [B][max_depth] */
+  int32_t *next_token;    /* [B]            */
+  int32_t *n_leaves;      /* [B]            */
+  int32_t *leaf_paths;    /* [B][T][L]      */
+  int32_t *status;        /* [1]            */
+} ddd_verify_output;
+
+/*
+ * Greedy acceptance walk and leaf-path table over the rows ddd_draft emitted.  (Section 1: the
+ * target model verifies the tree in one call; at temperature 0 a draft token is accepted when it
+ * is the target's own choice after its parent, which makes acceptance a walk from the root.)
+ *   n_out, token, parent   DEVICE, as in ddd_output ([B], [B][T], [B][T]); row 0 is the root
+ *   target_argmax          DEVICE [B][T] int32: the target's choice of next token after row i
+ *                          (its argmax at that row's position under the tree mask); rows
+ *                          >= n_out are ignored
+ * The walk starts at row 0 and moves to the child of the current row whose token equals
+ * target_argmax of the current row (the lowest such row, should siblings repeat a token) until
+ * there is none.  Needs no handle and no workspace; enqueues two small kernels on `cuda_stream`
+ * and returns without waiting.  Limits: 1 <= t_rows <= DDD_MAX_TOTAL + 1, 1 <= max_depth <=
+ * DDD_MAX_DEPTH, batch >= 1.  Errors: INVALID_ARG, CUDA.
+ */
+int ddd_verify_greedy(int32_t batch, int32_t t_rows, int32_t max_depth, const int32_t *n_out,
+                      const int32_t *token, const int32_t *parent, const int32_t *target_argmax,
+                      const ddd_verify_output *out /* HOST struct */, void *cuda_stream);
+
 /* Releases host state (and the captured graph).  Device memory stays with the caller. */
 int ddd_destroy(ddd_handle *h);
 

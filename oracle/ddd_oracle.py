@@ -21,6 +21,10 @@ oracle *is* the algorithm:
   * rerank / tree mask      - Section 1 (the whole tree is fed to the target with an
                               adjusted attention mask); the top-m rule is this
                               library's stated reading, the paper leaves it to EAGLE-2.
+  * acceptance walk         - Section 1 (the target verifies the tree in one call; at
+                              temperature 0 a draft token is accepted iff it is the
+                              target's own choice after its parent) and the root-to-leaf
+                              path table of the emitted tree.
 
 Parity status: every function below is pinned by tests in tests/test_oracle_pins.py
 (brute-force path enumeration, closed forms, invariants, library routines).
@@ -437,6 +441,47 @@ def draft(cfg, weights: Dict, root_hidden, root_token, root_pos,
         r.cum = r.tree_cum[node_id]
         r.mask = tree_mask_rows(r.parent)
     return res
+
+
+def greedy_accept(token: Sequence[int], parent: Sequence[int], n_out: int,
+                  target_argmax: Sequence[int]):
+    """Section 1, verification at temperature 0.  Rows 0..n_out-1 are a tree (row 0 the root,
+    parent[i] the parent's row).  target_argmax[i] is the target's choice of the token that
+    follows row i.  Starting at the root, the child of the current row that carries exactly that
+    token is accepted and becomes the current row; the walk ends when no child does.
+    Returns (accepted rows in order, the target's token after the last accepted row)."""
+    cur = 0
+    accepted: List[int] = []
+    while True:
+        want = int(target_argmax[cur])
+        nxt = -1
+        for i in range(1, n_out):
+            if int(parent[i]) == cur and int(token[i]) == want:
+                nxt = i
+                break
+        if nxt < 0:
+            return accepted, want
+        accepted.append(nxt)
+        cur = nxt
+
+
+def leaf_paths(parent: Sequence[int], n_out: int) -> List[List[int]]:
+    """Root-to-leaf row lists of the emitted tree, one per leaf, leaves in ascending row order.
+    A leaf is a row that no emitted row names as its parent."""
+    has_child = [False] * n_out
+    for i in range(1, n_out):
+        has_child[int(parent[i])] = True
+    paths = []
+    for leaf in range(n_out):
+        if has_child[leaf]:
+            continue
+        path = []
+        r = leaf
+        while r >= 0:
+            path.append(r)
+            r = int(parent[r])
+        paths.append(path[::-1])
+    return paths
 
 
 def mask_words(mask_rows: Sequence[int], t_max: int) -> np.ndarray:

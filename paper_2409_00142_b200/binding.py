@@ -41,6 +41,11 @@ class DddTrace(ctypes.Structure):
         "node_id", "tree_token", "tree_parent", "tree_cum", "beam_sel", "row_lse")]
 
 
+class DddVerifyOutput(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in (
+        "n_accepted", "accepted_rows", "next_token", "n_leaves", "leaf_paths", "status")]
+
+
 def library_path() -> str:
     return os.path.join(_HERE, _LIB_NAME)
 
@@ -78,6 +83,9 @@ def load_library():
     lib.ddd_lm_head_topk_noalloc.restype = ctypes.c_int
     lib.ddd_lm_head_topk_noalloc.argtypes = [vp, vp, vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
                                              ctypes.c_int32, ctypes.c_int32, ctypes.c_float, vp, vp, vp, vp]
+    lib.ddd_verify_greedy.restype = ctypes.c_int
+    lib.ddd_verify_greedy.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, i32p, i32p, i32p, i32p,
+                                      ctypes.POINTER(DddVerifyOutput), vp]
     lib.ddd_destroy.restype = ctypes.c_int
     lib.ddd_destroy.argtypes = [vp]
     lib.ddd_strerror.restype = ctypes.c_char_p
@@ -89,8 +97,8 @@ def load_library():
 def exported_symbols():
     """Names this binding expects the library to export (all of include/ddd.h)."""
     return ["ddd_workspace_bytes", "ddd_create", "ddd_draft", "ddd_draft_host", "ddd_draft_host_gated", "ddd_lm_head_pass",
-            "ddd_launches_per_draft", "ddd_lm_head_blocks", "ddd_lm_head_topk_noalloc", "ddd_destroy",
-            "ddd_strerror"]
+            "ddd_launches_per_draft", "ddd_lm_head_blocks", "ddd_lm_head_topk_noalloc", "ddd_verify_greedy",
+            "ddd_destroy", "ddd_strerror"]
 
 
 # ----------------------------------------------------------------------------- same-name wrappers
@@ -164,6 +172,15 @@ def ddd_lm_head_topk_noalloc(W: int, bias: Optional[int], hidden_rows: int, dtyp
                                                  logit_scale, out_token, out_logprob, out_lse, stream)
     if rc != 0:
         raise DddError(rc, "ddd_lm_head_topk_noalloc")
+
+
+def ddd_verify_greedy(batch: int, t_rows: int, max_depth: int, n_out: int, token: int, parent: int,
+                      target_argmax: int, out: DddVerifyOutput, stream: int) -> None:
+    """Greedy acceptance walk and leaf-path table of emitted trees.  Pointers are device addresses."""
+    rc = load_library().ddd_verify_greedy(batch, t_rows, max_depth, n_out, token, parent, target_argmax,
+                                          ctypes.byref(out), stream)
+    if rc != 0:
+        raise DddError(rc, "ddd_verify_greedy")
 
 
 def ddd_destroy(handle: int) -> None:
@@ -258,6 +275,29 @@ class DraftEngine:
 
     def make_host_out(self, pinned: bool = True) -> Dict:
         return {name: self.torch.zeros(t.shape, dtype=t.dtype, pin_memory=pinned) for name, t in self.out.items()}
+
+    def verify_greedy(self, target_argmax) -> Dict:
+        """Runs the acceptance walk on the tree of the last draft.  `target_argmax` is a device int32
+        tensor [B][T]; returns device tensors named like the fields of ddd_verify_output."""
+        torch = self.torch
+        B, T, n = self.cfg.batch, self.cfg.total_tokens + 1, self.cfg.max_depth
+        assert target_argmax.is_cuda and target_argmax.dtype == torch.int32 and target_argmax.is_contiguous()
+        assert tuple(target_argmax.shape) == (B, T)
+        if getattr(self, "verify_out", None) is None:
+            i32, dev = torch.int32, self.device
+            self.verify_out = {
+                "n_accepted": torch.zeros(B, dtype=i32, device=dev),
+                "accepted_rows": torch.zeros(B, n, dtype=i32, device=dev),
+                "next_token": torch.zeros(B, dtype=i32, device=dev),
+                "n_leaves": torch.zeros(B, dtype=i32, device=dev),
+                "leaf_paths": torch.zeros(B, T, n + 1, dtype=i32, device=dev),
+                "status": torch.zeros(1, dtype=i32, device=dev),
+            }
+            self.c_verify_out = DddVerifyOutput(**{name: t.data_ptr() for name, t in self.verify_out.items()})
+        ddd_verify_greedy(B, T, n, self.out["n_out"].data_ptr(), self.out["token"].data_ptr(),
+                          self.out["parent"].data_ptr(), target_argmax.data_ptr(), self.c_verify_out,
+                          self.stream_ptr())
+        return self.verify_out
 
     def lm_head_pass(self) -> None:
         ddd_lm_head_pass(self.handle, self.stream_ptr())

@@ -67,6 +67,22 @@ def test_create_rejects_bad_arguments_without_a_device():
     assert lib.ddd_launches_per_draft(None, 1) < 0 and lib.ddd_lm_head_blocks(None) < 0
 
 
+def test_verify_greedy_rejects_bad_arguments_without_a_device():
+    fake = 0x10000   # never dereferenced: every call below fails validation first
+    out = P.DddVerifyOutput(**{name: fake for name, _ in P.DddVerifyOutput._fields_})
+    for sizes in [(0, 4, 4), (1, 0, 4), (1, 1025, 4), (1, 4, 0), (1, 4, 33)]:
+        with pytest.raises(P.DddError) as err:
+            P.ddd_verify_greedy(*sizes, fake, fake, fake, fake, out, 0)
+        assert err.value.code == -1, sizes
+    for missing in range(4):
+        ptrs = [fake] * 4
+        ptrs[missing] = None
+        with pytest.raises(P.DddError):
+            P.ddd_verify_greedy(1, 4, 4, *ptrs, out, 0)
+    with pytest.raises(P.DddError):
+        P.ddd_verify_greedy(1, 4, 4, fake, fake, fake, fake, P.DddVerifyOutput(), 0)
+
+
 def test_strerror_covers_every_code():
     seen = {P.ddd_strerror(c) for c in range(0, -7, -1)}
     assert len(seen) == 7 and "unknown error code" not in seen

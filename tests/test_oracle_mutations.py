@@ -62,9 +62,40 @@ def _logits_transposed_scale(W, h, scale, bias):   # scale applied to the bias a
     return scale * z
 
 
+def _accept_any_row_with_the_token(token, parent, n_out, target_argmax):   # forgets the parent link
+    cur, accepted = 0, []
+    while True:
+        want = int(target_argmax[cur])
+        nxt = next((i for i in range(cur + 1, n_out) if int(token[i]) == want), -1)
+        if nxt < 0:
+            return accepted, want
+        accepted.append(nxt)
+        cur = nxt
+
+
+def _accept_one_step_only(token, parent, n_out, target_argmax):             # stops after the first match
+    accepted, nxt = ORIG["greedy_accept"](token, parent, n_out, target_argmax)
+    return accepted[:1], (int(target_argmax[accepted[0]]) if accepted else nxt)
+
+
+def _leaf_paths_leaf_first(parent, n_out):                                  # paths not reversed
+    return [p[::-1] for p in ORIG["leaf_paths"](parent, n_out)]
+
+
+def _leaf_paths_every_row(parent, n_out):                                   # inner rows listed as leaves too
+    out = []
+    for leaf in range(n_out):
+        path, r = [], leaf
+        while r >= 0:
+            path.append(r)
+            r = int(parent[r])
+        out.append(path[::-1])
+    return out
+
+
 ORIG = {name: getattr(O, name) for name in (
     "heuristic_H", "topk_desc", "log_softmax_row", "draft_step", "tree_mask_rows", "rerank", "apply_plant",
-    "lm_head_logits")}
+    "lm_head_logits", "greedy_accept", "leaf_paths")}
 
 CASES = [
     ("heuristic_H", _h_mean, pins.test_uniform_closed_form_H_and_tiebreaks, ()),
@@ -79,6 +110,11 @@ CASES = [
     ("rerank", _rerank_lowest, pins.test_rerank_plain_definition_and_invariants, ()),
     ("apply_plant", _plant_added, pins.test_plant_closed_form, ()),
     ("lm_head_logits", _logits_transposed_scale, pins.test_logits_match_library_matmul, ("bf16",)),
+    ("greedy_accept", _accept_any_row_with_the_token, pins.test_greedy_accept_against_consistency_definition, ()),
+    ("greedy_accept", _accept_one_step_only, pins.test_greedy_accept_chain_closed_form, ()),
+    ("greedy_accept", _accept_one_step_only, pins.test_acceptance_on_a_drafted_tree_follows_a_planted_path, ()),
+    ("leaf_paths", _leaf_paths_leaf_first, pins.test_leaf_paths_cover_the_tree, ()),
+    ("leaf_paths", _leaf_paths_every_row, pins.test_leaf_paths_cover_the_tree, ()),
 ]
 
 

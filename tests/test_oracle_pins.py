@@ -436,3 +436,96 @@ def test_admissible_topk_bands():
     assert O.admissible_topk(s, [1, 0, 2], 3, 2e-3)                 # wrong order
     assert not O.admissible_topk(s, [1, 0, 2], 3, 2e-3, ordered=False)
     assert O.admissible_topk(s, [0, 0, 1], 3, 2e-3)                 # duplicates
+
+
+# --------------------------------------------------------------------------- acceptance walk, leaf paths
+def _path_to(parent, i):
+    path = []
+    while i >= 0:
+        path.append(i)
+        i = int(parent[i])
+    return path[::-1]
+
+
+def test_greedy_accept_against_consistency_definition():
+    """Accepted rows = exactly the rows whose whole root path agrees with the target: each row on
+    the path carries the token the target chose after that row's parent (Section 1)."""
+    rng = np.random.default_rng(11)
+    n_agree = []
+    for trial in range(200):
+        n_rows = int(rng.integers(1, 40))
+        vocab = int(rng.integers(3, 9))          # small vocabulary: agreements are common
+        token, parent = S.random_tree(rng, n_rows, vocab)
+        target = rng.integers(vocab, size=n_rows)
+        consistent = []
+        for i in range(1, n_rows):
+            path = _path_to(parent, i)
+            if all(token[j] == target[parent[j]] for j in path[1:]):
+                consistent.append(i)
+        # sibling tokens are distinct, so the consistent rows lie on one root path
+        consistent.sort(key=lambda i: len(_path_to(parent, i)))
+        for a, b in zip(consistent, consistent[1:]):
+            assert parent[b] == a
+        accepted, nxt = O.greedy_accept(token, parent, n_rows, target)
+        assert accepted == consistent
+        last = accepted[-1] if accepted else 0
+        assert nxt == target[last]
+        n_agree.append(len(accepted))
+    assert max(n_agree) >= 3 and min(n_agree) == 0          # the cases exercise both ends
+
+
+def test_greedy_accept_chain_closed_form():
+    """A k = 1 chain whose first j tokens match the target accepts exactly j tokens."""
+    n = 9
+    token = np.arange(100, 100 + n)
+    parent = np.arange(-1, n - 1)
+    for j in range(n):
+        target = np.full(n, -7)
+        target[:j] = token[1:j + 1]               # the target agrees after rows 0..j-1
+        accepted, nxt = O.greedy_accept(token, parent, n, target)
+        assert accepted == list(range(1, j + 1))
+        assert nxt == -7
+    # every draft token accepted: the bonus token is the target's choice after the last row
+    target = np.append(token[1:], 555)
+    accepted, nxt = O.greedy_accept(token, parent, n, target)
+    assert accepted == list(range(1, n)) and nxt == 555
+    # rows beyond n_out do not take part
+    accepted, nxt = O.greedy_accept(token, parent, 4, target)
+    assert accepted == [1, 2, 3] and nxt == token[4]
+
+
+def test_leaf_paths_cover_the_tree():
+    rng = np.random.default_rng(5)
+    for trial in range(100):
+        n_rows = int(rng.integers(1, 60))
+        token, parent = S.random_tree(rng, n_rows, 50)
+        paths = O.leaf_paths(parent, n_rows)
+        leaves = [p[-1] for p in paths]
+        assert leaves == sorted(set(range(n_rows)) - set(int(x) for x in parent[1:]))
+        covered = set()
+        for p in paths:
+            assert p[0] == 0
+            for a, b in zip(p, p[1:]):
+                assert parent[b] == a
+            covered.update(p)
+        assert covered == set(range(n_rows))
+        # the ancestor mask of a leaf (a separately pinned construction) marks exactly its path
+        mask = O.tree_mask_rows(list(parent))
+        for p in paths:
+            assert mask[p[-1]] == sum(1 << r for r in p)
+
+
+def test_acceptance_on_a_drafted_tree_follows_a_planted_path():
+    """Target choices planted along one emitted row's ancestors: the walk accepts that path."""
+    cfg = S.CONFIGS["tiny"].replace(batch=1, threshold=-1e30)
+    w = S.make_weights(cfg)
+    res = O.draft(cfg, w, **S.make_roots(cfg, 0))[0]
+    n_out = res.n_out
+    deepest = int(np.argmax(res.depth[:n_out]))
+    path = _path_to(res.parent, deepest)
+    target = np.full(n_out, cfg.vocab)            # a token no draft row can carry
+    for a, b in zip(path, path[1:]):
+        target[a] = res.token[b]
+    accepted, nxt = O.greedy_accept(res.token, res.parent, n_out, target)
+    assert accepted == path[1:] and nxt == cfg.vocab
+    assert len(accepted) == res.depth[deepest]
