@@ -61,8 +61,10 @@ enum { DDD_LM_HEAD_AUTO = 0, DDD_LM_HEAD_SIMT = 1, DDD_LM_HEAD_TCGEN05 = 2 };
 
 /* How a draft is enqueued.  STREAM launches kernel by kernel, each allowed to start while its
  * predecessor still runs (programmatic dependent launch; they synchronise on the device).
- * GRAPH replays one captured CUDA graph per draft, in which the passes after the third sit
- * behind a conditional node that only a still-drafting sequence switches on.  PLAIN launches
+ * GRAPH replays one captured CUDA graph per draft, in which the passes are cut into groups (after
+ * checked steps: passes 1-3, 4-5, 6-8, 9-12, ... when every step is checked) and every group
+ * but the first sits behind a conditional node that only a still-drafting sequence switches
+ * on, so that a draft that stops early launches little that has nothing to do.  PLAIN launches
  * kernel by kernel in ordinary stream order, one after the other: the slowest, and the one
  * profilers can follow. */
 enum { DDD_LAUNCH_STREAM = 0, DDD_LAUNCH_GRAPH = 1, DDD_LAUNCH_PLAIN = 2 };
@@ -217,8 +219,8 @@ int ddd_lm_head_pass(ddd_handle *h, void *cuda_stream);
 /*
  * ddd_launches_per_draft: kernels one ddd_draft launches when a sequence of the batch needs
  * `passes_needed` LM-head passes (its largest stop depth).  Outside graph mode every pass is
- * launched (kernels of passes after the stop exit at once); in graph mode the passes after the
- * third are launched only if some sequence is still drafting then.
+ * launched (kernels of passes after the stop exit at once); in graph mode the passes up to the
+ * end of the group that holds pass `passes_needed` are launched.
  * ddd_lm_head_blocks: thread blocks of the LM-head kernel.
  * Pure host queries; negative on a NULL handle.
  */

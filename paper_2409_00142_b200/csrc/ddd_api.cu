@@ -112,6 +112,9 @@ Layout make_layout(const ddd_config* c) {
   return L;
 }
 
+constexpr int kFirstBoundary = 3;    // first pass after which a captured draft may end early
+constexpr int kMaxGraphLevels = 4;   // nested IF nodes of a captured draft
+
 struct GraphKey {
   ddd_output out;
   ddd_trace trace;
@@ -134,6 +137,9 @@ struct ddd_handle {
   bool have_graph;
   bool use_pdl;    // programmatic dependent launch between the kernels of a draft
   bool graph_pdl;  // whether the captured graph uses it
+  int bounds[kMaxGraphLevels];   // passes after which a captured draft may end early (IF nodes), ascending
+  int n_bounds;
+  int graph_bounds;   // how many of them the captured graph has
   // pinned host bounce buffer for ddd_draft_host
   unsigned char* bounce;
   size_t bounce_bytes;
@@ -162,34 +168,62 @@ cudaError_t enqueue_passes(const ddd_handle* h, const DraftIO& io, bool pdl, int
   return e;
 }
 
-// Passes of a captured draft that always run; the rest sit behind one conditional node that
-// stays off unless some sequence is still drafting after them.  Most drafts stop early, and a
-// pass that has nothing to do still costs two kernel launches.
-constexpr int kUnconditionalPasses = 3;
+// Where a captured draft may end early.  A pass that has nothing left to do still costs two
+// kernel launches (about 4 us), and most drafts stop long before pass n, so the passes are cut
+// into groups: group 0 (passes 1..b1) always runs, every later group sits in the body of an IF
+// node that only a sequence still drafting after the previous group switches on; the bodies
+// nest.  Boundaries are put after checked steps only (nothing can stop elsewhere), the first
+// not before pass 3, the groups growing by one pass each (3, 5, 8, 12 when every step is
+// checked), at most kMaxGraphLevels of them: a skipped or entered IF node costs about as much as
+// an idle pass, so a deep draft should not cross many.
 
-// Captures everything after the init kernel into h->exec.  Returns false (and leaves no graph)
-// on any failure.
-bool capture_graph(ddd_handle* h, const DraftIO& io, bool pdl, cudaStream_t st) {
+int graph_boundaries(const ddd_config& cfg, int* bounds /* [kMaxGraphLevels] */) {
+  const int n = cfg.max_depth;
+  int count = 0;
+  if (n <= kFirstBoundary + 1) return 0;
+  int want = kFirstBoundary, gap = 2;
+  for (int d = kFirstBoundary; d < n && count < kMaxGraphLevels; ++d) {
+    if (d < want || !((cfg.check_mask >> (d - 1)) & 1u)) continue;
+    bounds[count++] = d;
+    want = d + gap;
+    ++gap;
+  }
+  return count;
+}
+
+struct CaptureLog {
+  int step = 0;   // which call failed first, for the diagnostic
+  bool good(cudaError_t e, int id) {
+    if (e != cudaSuccess && step == 0) step = id;
+    return e == cudaSuccess;
+  }
+};
+
+// Captures group `level` (passes first..bounds[level], or first..n for the last group) into
+// `graph`, followed by the IF node that guards the next group; the top level ends with the rerank.
+bool capture_level(ddd_handle* h, const DraftIO& io, bool pdl, cudaStream_t st, cudaGraph_t graph,
+                   const int* bounds, int n_bounds, int level, int first, CaptureLog& log) {
   const int n = h->p.n;
-  const int head = n <= kUnconditionalPasses + 1 ? n : kUnconditionalPasses;   // passes outside the conditional
-  cudaGraph_t graph = nullptr, body = nullptr;
+  const bool has_if = level < n_bounds;
+  const int last = has_if ? bounds[level] : n;
+  const int id = 10 * level;
   cudaGraphConditionalHandle cond = 0;
-  int step = 0;   // which call failed, for the diagnostic
-  auto good = [&](cudaError_t e, int id) { if (e != cudaSuccess && step == 0) step = id; return e == cudaSuccess; };
-  bool ok = good(cudaGraphCreate(&graph, 0), 1);
-  if (ok && head < n) ok = good(cudaGraphConditionalHandleCreate(&cond, graph, 0, cudaGraphCondAssignDefault), 2);
+  cudaGraph_t body = nullptr;
+  bool ok = true;
+  if (has_if) ok = log.good(cudaGraphConditionalHandleCreate(&cond, graph, 0, cudaGraphCondAssignDefault), id + 2);
   bool capturing = false;
   if (ok) {
-    ok = good(cudaStreamBeginCaptureToGraph(st, graph, nullptr, nullptr, 0, cudaStreamCaptureModeThreadLocal), 3);
+    ok = log.good(cudaStreamBeginCaptureToGraph(st, graph, nullptr, nullptr, 0, cudaStreamCaptureModeThreadLocal),
+                  id + 3);
     capturing = ok;
   }
-  if (ok) ok = good(enqueue_passes(h, io, pdl, 1, head, cond, head < n ? head : 0, st), 4);
-  if (ok && head < n) {
-    // splice an IF node between the captured passes and the rerank
+  if (ok) ok = log.good(enqueue_passes(h, io, pdl, first, last, cond, has_if ? last : 0, st), id + 4);
+  if (ok && has_if) {
+    // splice the IF node in behind the captured passes
     cudaStreamCaptureStatus status;
     const cudaGraphNode_t* deps = nullptr;
     size_t n_deps = 0;
-    ok = good(cudaStreamGetCaptureInfo(st, &status, nullptr, nullptr, &deps, &n_deps), 5) &&
+    ok = log.good(cudaStreamGetCaptureInfo(st, &status, nullptr, nullptr, &deps, &n_deps), id + 5) &&
          status == cudaStreamCaptureStatusActive;
     cudaGraphNode_t node = nullptr;
     if (ok) {
@@ -198,33 +232,37 @@ bool capture_graph(ddd_handle* h, const DraftIO& io, bool pdl, cudaStream_t st) 
       np.conditional.handle = cond;
       np.conditional.type = cudaGraphCondTypeIf;
       np.conditional.size = 1;
-      ok = good(cudaGraphAddNode(&node, graph, deps, n_deps, &np), 6);
+      ok = log.good(cudaGraphAddNode(&node, graph, deps, n_deps, &np), id + 6);
       if (ok) body = np.conditional.phGraph_out[0];
     }
-    if (ok) ok = good(cudaStreamUpdateCaptureDependencies(st, &node, 1, cudaStreamSetCaptureDependencies), 7);
+    if (ok) ok = log.good(cudaStreamUpdateCaptureDependencies(st, &node, 1, cudaStreamSetCaptureDependencies), id + 7);
   }
-  // the rerank follows a conditional node, not a kernel: plain dependency
-  if (ok) ok = good(launch_rerank(h->p, io, pdl && head == n, st), 8);
+  // the rerank follows a conditional node, not a kernel, unless there is none: plain dependency
+  if (ok && level == 0) ok = log.good(launch_rerank(h->p, io, pdl && !has_if, st), id + 8);
   if (capturing) {
     cudaGraph_t done = nullptr;
-    if (!good(cudaStreamEndCapture(st, &done), 9)) ok = false;
+    if (!log.good(cudaStreamEndCapture(st, &done), id + 9)) ok = false;
   }
-  if (ok && body) {
-    ok = good(cudaStreamBeginCaptureToGraph(st, body, nullptr, nullptr, 0, cudaStreamCaptureModeThreadLocal), 10);
-    if (ok) {
-      if (!good(enqueue_passes(h, io, pdl, head + 1, n, cond, 0, st), 11)) ok = false;
-      cudaGraph_t done = nullptr;
-      if (!good(cudaStreamEndCapture(st, &done), 12)) ok = false;
-    }
-  }
-  if (ok) ok = good(cudaGraphInstantiate(&h->exec, graph, 0), 13);
+  if (ok && body) ok = capture_level(h, io, pdl, st, body, bounds, n_bounds, level + 1, last + 1, log);
+  return ok;
+}
+
+// Captures everything after the init kernel into h->exec, with IF nodes after the first
+// `n_bounds` boundaries.  Returns false (and leaves no graph) on any failure.
+bool capture_graph(ddd_handle* h, const DraftIO& io, bool pdl, int n_bounds, cudaStream_t st) {
+  cudaGraph_t graph = nullptr;
+  CaptureLog log;
+  bool ok = log.good(cudaGraphCreate(&graph, 0), 1);
+  if (ok) ok = capture_level(h, io, pdl, st, graph, h->bounds, n_bounds, 0, 1, log);
+  if (ok) ok = log.good(cudaGraphInstantiate(&h->exec, graph, 0), 99);
   if (graph) cudaGraphDestroy(graph);
   if (!ok) {
-    note_cuda_error(1000 + step);   // 1000 + index of the capture step that failed
+    note_cuda_error(1000 + log.step);   // 1000 + 10 * group + index of the capture step that failed
     h->exec = nullptr;
     return false;
   }
   h->graph_pdl = pdl;
+  h->graph_bounds = n_bounds;
   return true;
 }
 
@@ -262,6 +300,8 @@ int ddd_create(const ddd_config* cfg, const void* W, const void* E, const float*
   h->ws = static_cast<unsigned char*>(workspace);
   h->sm_count = prop.multiProcessorCount;
   h->have_graph = false;
+  h->n_bounds = graph_boundaries(*cfg, h->bounds);
+  h->graph_bounds = 0;
   h->use_pdl = cfg->launch_mode != DDD_LAUNCH_PLAIN;
   h->graph_pdl = false;
   h->exec = nullptr;
@@ -345,8 +385,13 @@ int ddd_draft(ddd_handle* h, const void* root_hidden, const int32_t* root_token,
       if (h->exec) { cudaGraphExecDestroy(h->exec); h->exec = nullptr; }
       h->have_graph = false;
       // capture with programmatic dependent launches; if this driver cannot capture or
-      // instantiate them, capture the plain stream-ordered sequence instead
-      if (!(h->use_pdl && capture_graph(h, io, true, st)) && !capture_graph(h, io, false, st)) return DDD_ERR_CUDA;
+      // instantiate them, capture the plain stream-ordered sequence instead; likewise fall back
+      // from nested IF nodes to a single one
+      const int one = h->n_bounds < 1 ? h->n_bounds : 1;
+      if (!(h->use_pdl && capture_graph(h, io, true, h->n_bounds, st)) &&
+          !(h->use_pdl && one != h->n_bounds && capture_graph(h, io, true, one, st)) &&
+          !capture_graph(h, io, false, one, st))
+        return DDD_ERR_CUDA;
       h->key = key;
       h->have_graph = true;
     }
@@ -473,8 +518,11 @@ int ddd_launches_per_draft(const ddd_handle* h, int32_t passes_needed) {
   if (!h) return DDD_ERR_INVALID_ARG;
   const int n = h->p.n;
   int passes = n;
-  if (h->cfg.launch_mode == DDD_LAUNCH_GRAPH && n > kUnconditionalPasses + 1 && passes_needed <= kUnconditionalPasses)
-    passes = kUnconditionalPasses;
+  if (h->cfg.launch_mode == DDD_LAUNCH_GRAPH) {
+    const int nb = h->have_graph ? h->graph_bounds : h->n_bounds;
+    for (int j = nb - 1; j >= 0; --j)
+      if (passes_needed <= h->bounds[j]) passes = h->bounds[j];   // the group that holds the last needed pass
+  }
   return 2 + 2 * passes;   // init, (LM head + select) per launched pass, rerank
 }
 

@@ -189,11 +189,49 @@ def test_graph_mode_host_variant_and_determinism():
     for name in host_out:
         np.testing.assert_array_equal(host_out[name].numpy(), a[name], err_msg=name)
     assert P.ddd_launches_per_draft(eng_s.handle, 1) == 2 + 2 * cfg.max_depth
-    assert P.ddd_launches_per_draft(eng_g.handle, 2) == 2 + 2 * 3
-    assert P.ddd_launches_per_draft(eng_g.handle, 4) == 2 + 2 * cfg.max_depth
+    # captured drafts end early after passes 3, 5 and 8 (every step checked, n = 12)
+    assert cfg.max_depth == 12 and cfg.check_mask & 0xFFF == 0xFFF
+    for needed, launched in [(1, 3), (2, 3), (3, 3), (4, 5), (5, 5), (6, 8), (8, 8), (9, 12), (12, 12)]:
+        assert P.ddd_launches_per_draft(eng_g.handle, needed) == 2 + 2 * launched, needed
     assert 1 <= P.ddd_lm_head_blocks(eng_s.handle) <= 512
     eng_s.close()
     eng_g.close()
+
+
+@pytest.mark.parametrize("schedule", ["every_step", "paper_5_7_9", "only_4"])
+def test_captured_drafts_of_every_stop_depth_equal_stream_launches(schedule):
+    # the captured graph nests its conditional groups; whatever depth a draft stops at, inside a
+    # group, at its end or at n, the results are those of the kernel-by-kernel launches
+    base = small_cases()["7b"]
+    if schedule == "every_step":
+        cfgs = [base.replace(threshold=x) for x in (-1.0, -3.0, -5.0, -7.0, -9.0, -12.0, -16.0, -22.0, NEG)]
+    elif schedule == "paper_5_7_9":
+        mask = sum(1 << (s - 1) for s in (5, 7, 9))
+        cfgs = [base.replace(max_depth=11, check_mask=mask, threshold=x) for x in (-0.3, -9.0, -13.0, -17.0, NEG)]
+    else:
+        cfgs = [base.replace(max_depth=6, check_mask=1 << 3, threshold=x) for x in (-0.5, NEG)]
+    seen = set()
+    stream = torch.cuda.Stream()
+    for cfg in cfgs:
+        eng_s = engine_for(cfg, TC, P.DDD_LAUNCH_STREAM)
+        eng_g = engine_for(cfg, TC, P.DDD_LAUNCH_GRAPH)
+        for i in range(3):
+            roots = S.make_roots(cfg, i)
+            a = parity.run_gpu(eng_s, roots)
+            with torch.cuda.stream(stream):
+                b = parity.run_gpu(eng_g, roots)
+            for name in a:
+                np.testing.assert_array_equal(a[name], b[name], err_msg=f"{name} x={cfg.threshold}")
+            seen.update(a["stop_depth"].tolist())
+        parity.compare_with_oracle(cfg, weights_for(cfg), roots, b)
+        eng_s.close()
+        eng_g.close()
+    if schedule == "every_step":
+        assert len(seen) >= 6 and min(seen) <= 2 and max(seen) == 12, sorted(seen)
+    elif schedule == "paper_5_7_9":
+        assert seen <= {5, 7, 9, 11} and len(seen) >= 2, sorted(seen)
+    else:
+        assert seen <= {4, 6}, sorted(seen)
 
 
 def test_handles_of_different_sizes_coexist():
