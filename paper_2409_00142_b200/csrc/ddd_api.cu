@@ -200,7 +200,7 @@ struct CaptureLog {
 };
 
 // Captures group `level` (passes first..bounds[level], or first..n for the last group) into
-// `graph`, followed by the IF node that guards the next group; the top level ends with the rerank.
+// `graph`, followed by the IF node that guards the next group.
 bool capture_level(ddd_handle* h, const DraftIO& io, bool pdl, cudaStream_t st, cudaGraph_t graph,
                    const int* bounds, int n_bounds, int level, int first, CaptureLog& log) {
   const int n = h->p.n;
@@ -237,8 +237,6 @@ bool capture_level(ddd_handle* h, const DraftIO& io, bool pdl, cudaStream_t st, 
     }
     if (ok) ok = log.good(cudaStreamUpdateCaptureDependencies(st, &node, 1, cudaStreamSetCaptureDependencies), id + 7);
   }
-  // the rerank follows a conditional node, not a kernel, unless there is none: plain dependency
-  if (ok && level == 0) ok = log.good(launch_rerank(h->p, io, pdl && !has_if, st), id + 8);
   if (capturing) {
     cudaGraph_t done = nullptr;
     if (!log.good(cudaStreamEndCapture(st, &done), id + 9)) ok = false;
@@ -403,8 +401,7 @@ int ddd_draft(ddd_handle* h, const void* root_hidden, const int32_t* root_token,
     return DDD_OK;
   }
   if (launch_init(h->p, io, root_hidden, root_token, root_pos, st) != cudaSuccess ||
-      enqueue_passes(h, io, h->use_pdl, 1, h->p.n, 0, 0, st) != cudaSuccess ||
-      launch_rerank(h->p, io, h->use_pdl, st) != cudaSuccess) {
+      enqueue_passes(h, io, h->use_pdl, 1, h->p.n, 0, 0, st) != cudaSuccess) {
     note_cuda_error(__LINE__);
     return DDD_ERR_CUDA;
   }
@@ -434,7 +431,6 @@ int ddd_draft_host_gated(ddd_handle* h, const void* root_hidden, const int32_t* 
     if (e != cudaSuccess || still == 0) break;
   }
   if (passes_run) *passes_run = d <= h->p.n ? d : h->p.n;
-  if (e == cudaSuccess) e = launch_rerank(h->p, io, false, st);
   if (e != cudaSuccess) {
     note_cuda_error(__LINE__);
     return DDD_ERR_CUDA;
@@ -523,7 +519,7 @@ int ddd_launches_per_draft(const ddd_handle* h, int32_t passes_needed) {
     for (int j = nb - 1; j >= 0; --j)
       if (passes_needed <= h->bounds[j]) passes = h->bounds[j];   // the group that holds the last needed pass
   }
-  return 2 + 2 * passes;   // init, (LM head + select) per launched pass, rerank
+  return 1 + 2 * passes;   // init, then (LM head + select) per launched pass
 }
 
 int ddd_lm_head_blocks(const ddd_handle* h) {

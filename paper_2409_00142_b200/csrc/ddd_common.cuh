@@ -203,6 +203,5 @@ cudaError_t launch_lm_head_simt(const Params& p, int d, int force_all, int ctas,
 // set_cond: a sequence that continues after pass d sets the graph conditional `cond` to 1.
 cudaError_t launch_select(const Params& p, const DraftIO& io, int d, bool pdl, cudaGraphConditionalHandle cond,
                           bool set_cond, cudaStream_t st);
-cudaError_t launch_rerank(const Params& p, const DraftIO& io, bool pdl, cudaStream_t st);
 
 }  // namespace ddd

@@ -320,6 +320,187 @@ __device__ void draft_step(const Params& p, int b, int d, const int* sel_flat, c
     draft_step_warp<T>(p, b, d, sel_flat, sel_tok);
 }
 
+// ---------------------------------------------------------------------------- rerank + mask
+__device__ __forceinline__ int node_depth(int id, int k) {
+  if (id == 0) return 0;
+  if (id <= k) return 1;
+  return 2 + (id - 1 - k) / (k * k);
+}
+
+// Block-wide exclusive prefix sum of one int per thread (kRerankThreads threads).
+__device__ int block_exclusive_scan(int v, int* warp_tot /* [32] shared */, int* total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(kFullMask, inc, o);
+    if (lane >= o) inc += t;
+  }
+  __syncthreads();                 // protect warp_tot from its previous use
+  if (lane == 31) warp_tot[warp] = inc;
+  __syncthreads();
+  int offset = 0, tot = 0;
+  for (int w = 0; w < kRerankThreads / 32; ++w) {
+    const int t = warp_tot[w];
+    if (w < warp) offset += t;
+    tot += t;
+  }
+  *total = tot;
+  return offset + inc - v;
+}
+
+// Final step of a sequence, run by one block of kRerankThreads threads right after the pass at
+// which the sequence stopped (D): keep the m best nodes, emit the rows and the ancestor mask.
+// smem_raw: ordered cum keys [Nn] (32 bit), then selection flags / output rows [Nn] (16 bit).  `last` says that this
+// was the last sequence of the batch still drafting: that block also reports the device status.
+__device__ void rerank_mask_block(const Params& p, const DraftIO& io, const int b, const int D, const bool last,
+                                  unsigned char* smem_raw) {
+  const int tid = threadIdx.x;
+  const int k = p.k, T = p.T;
+  const int N = (D >= 1) ? k + (D - 1) * k * k : 0;     // generated non-root nodes
+  uint32_t* key = reinterpret_cast<uint32_t*>(smem_raw);           // key of node id i+1 at [i]
+  short* slot_of = reinterpret_cast<short*>(key + p.Nn);            // output row of node id (< 1024), -1 = dropped
+  __shared__ int hist[256];
+  __shared__ int warp_tot[32];
+  __shared__ uint32_t s_prefix;
+  __shared__ int s_remaining;
+  __shared__ int out_parent[DDD_MAX_TOTAL + 1];
+
+  const float* cum = p.tree_cum + (size_t)b * p.Nn;
+  const int* tparent = p.tree_parent + (size_t)b * p.Nn;
+  const int* ttoken = p.tree_token + (size_t)b * p.Nn;
+  for (int i = tid; i < N; i += kRerankThreads) key[i] = float_to_ordered(cum[i + 1]);
+  const int m_eff = min(p.m, N);
+  if (tid == 0) { s_prefix = 0u; s_remaining = m_eff; }
+  __syncthreads();
+
+  // ---- radix select: value of the m_eff-th largest key and how many of its ties to keep
+  uint32_t known_mask = 0u;
+  for (int pass = 3; pass >= 0 && m_eff > 0; --pass) {
+    const int shift = 8 * pass;
+    for (int i = tid; i < 256; i += kRerankThreads) hist[i] = 0;
+    __syncthreads();
+    const uint32_t prefix = s_prefix;
+    for (int i = tid; i < N; i += kRerankThreads) {
+      const uint32_t q = key[i];
+      if ((q & known_mask) == prefix) atomicAdd(&hist[(q >> shift) & 0xFF], 1);
+    }
+    __syncthreads();
+    if (tid < 32) {
+      // warp 0 finds the bin holding the `remaining`-th largest key: lane l owns bins 8l .. 8l+7
+      const int remaining = s_remaining;
+      int local[8], mine = 0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { local[i] = hist[8 * tid + i]; mine += local[i]; }
+      int above = mine;                                   // suffix sum over lanes >= tid ...
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_down_sync(kFullMask, above, o);
+        if (tid + o < 32) above += t;
+      }
+      above -= mine;                                      // ... made exclusive: keys in higher lanes' bins
+      if (above < remaining && remaining <= above + mine) {   // exactly one lane
+        int rem = remaining - above, bin = 7;
+        for (; bin > 0; --bin) {
+          if (local[bin] >= rem) break;
+          rem -= local[bin];
+        }
+        s_prefix = prefix | ((uint32_t)(8 * tid + bin) << shift);
+        s_remaining = rem;
+      }
+    }
+    known_mask |= 0xFFu << shift;
+    __syncthreads();
+  }
+  const uint32_t thr = s_prefix;
+  const int keep_ties = s_remaining;      // among keys equal to thr, the lowest node ids win
+
+  // ---- selection flags in node-id order; each thread owns a contiguous chunk of ids
+  const int chunk = (N + kRerankThreads - 1) / kRerankThreads;
+  const int lo = min(N, tid * chunk), hi = min(N, lo + chunk);
+  int n_eq = 0;
+  for (int i = lo; i < hi; ++i) n_eq += (key[i] == thr);
+  int tot_unused;
+  int eq_before = block_exclusive_scan(n_eq, warp_tot, &tot_unused);
+  int n_sel = 0;
+  for (int i = lo; i < hi; ++i) {
+    const uint32_t q = key[i];
+    bool sel = false;
+    if (m_eff > 0) {
+      if (q > thr) sel = true;
+      else if (q == thr) sel = (eq_before++ < keep_ties);
+    }
+    slot_of[i + 1] = sel ? 1 : 0;
+    n_sel += sel;
+  }
+  int n_selected;
+  int sel_before = block_exclusive_scan(n_sel, warp_tot, &n_selected);
+  for (int i = lo; i < hi; ++i) {
+    const bool sel = slot_of[i + 1] != 0;
+    slot_of[i + 1] = sel ? (short)(1 + sel_before) : (short)-1;
+    sel_before += sel;
+  }
+  if (tid == 0) slot_of[0] = 0;
+  __syncthreads();
+
+  // ---- emit rows: the root, then the kept nodes in ascending node id
+  const int n_out = 1 + n_selected;
+  const size_t ob = (size_t)b * T;
+  for (int id = tid; id <= N; id += kRerankThreads) {
+    const int slot = slot_of[id];
+    if (slot < 0 || slot >= T) continue;
+    const int dep = node_depth(id, k);
+    const int par = (id == 0) ? -1 : slot_of[tparent[id]];
+    out_parent[slot] = par;
+    io.out.token[ob + slot] = ttoken[id];
+    io.out.parent[ob + slot] = par;
+    io.out.depth[ob + slot] = dep;
+    io.out.position[ob + slot] = p.root_pos[b] + dep;
+    io.out.cum[ob + slot] = cum[id];
+    if (io.trace.node_id) io.trace.node_id[ob + slot] = id;
+  }
+  for (int slot = n_out + tid; slot < T; slot += kRerankThreads) {
+    io.out.token[ob + slot] = -1;
+    io.out.parent[ob + slot] = -1;
+    io.out.depth[ob + slot] = -1;
+    io.out.position[ob + slot] = -1;
+    io.out.cum[ob + slot] = 0.f;
+    if (io.trace.node_id) io.trace.node_id[ob + slot] = -1;
+  }
+  if (tid == 0) {
+    io.out.n_out[b] = n_out;
+    io.out.stop_depth[b] = D;
+    if (last) *io.out.status = *reinterpret_cast<volatile int*>(p.dev_status);
+  }
+  __syncthreads();
+
+  // ---- ancestor mask: row i has bit j set iff j is i or an ancestor of i
+  for (int slot = tid; slot < T; slot += kRerankThreads) {
+    uint32_t* row = io.out.mask + (ob + slot) * p.W32;
+    for (int w = 0; w < p.W32; ++w) {
+      uint32_t bits = 0u;
+      if (slot < n_out) {
+        int a = slot;
+        for (int guard = 0; a >= 0 && guard <= DDD_MAX_DEPTH; ++guard) {
+          if ((a >> 5) == w) bits |= 1u << (a & 31);
+          a = out_parent[a];
+        }
+      }
+      row[w] = bits;
+    }
+  }
+  // copy the generated tree for replay, if asked for
+  if (io.trace.tree_token) {
+    for (int id = tid; id < p.Nn; id += kRerankThreads) {
+      const bool gen = id <= N;
+      const size_t o = (size_t)b * p.Nn + id;
+      io.trace.tree_token[o] = gen ? ttoken[id] : -1;
+      if (io.trace.tree_parent) io.trace.tree_parent[o] = gen ? tparent[id] : -1;
+      if (io.trace.tree_cum) io.trace.tree_cum[o] = gen ? cum[id] : 0.f;
+    }
+  }
+}
+
 // One cluster of kSelCluster blocks per sequence.  Beam row pr is merged by block pr % 8
 // (warp pr / 8), which first copies that row's partial lists into its shared memory; the
 // candidates go to block 0 through distributed shared memory, block 0 picks the new beam and
@@ -361,6 +542,7 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
   __shared__ double row_part[DDD_MAX_K * 64];
   __shared__ double row_inv[DDD_MAX_K];
   __shared__ int s_stop;
+  __shared__ bool s_last;
   __shared__ float beam_cum_s[DDD_MAX_K / kSelCluster];
   __shared__ int beam_node_s[DDD_MAX_K / kSelCluster];
 
@@ -546,7 +728,7 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
         if (stop) {
           p.stop_depth[b] = d;
           p.active[b] = 0;
-          atomicSub(p.n_active, 1);
+          s_last = atomicSub(p.n_active, 1) == 1;
         }
       }
     }
@@ -555,193 +737,18 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
   // In a captured draft the passes after this one sit behind a conditional node (default: skip);
   // a sequence that goes on switches them on.
   if (set_cond && !s_stop && crank == 0 && threadIdx.x == 0) cudaGraphSetConditional(cond, 1);
-  if (s_stop) return;       // every block takes this branch alike
+  if (s_stop) {             // every block takes this branch alike
+    // the sequence is finished: block 0 goes straight on to the rerank and the mask (the nodes the
+    // other blocks appended in this pass are visible since the cluster barrier above)
+    if (crank == 0) rerank_mask_block(p, io, b, d, s_last, smem_raw);
+    return;
+  }
 
   // ---- phase 3: synthetic draft step for the k new beam rows
   if (p.dtype == DDD_DTYPE_BF16)
     draft_step<__nv_bfloat16>(p, b, d, sel_flat, sel_tok, row_part, row_inv);
   else
     draft_step<float>(p, b, d, sel_flat, sel_tok, row_part, row_inv);
-}
-
-// ---------------------------------------------------------------------------- rerank + mask
-__device__ __forceinline__ int node_depth(int id, int k) {
-  if (id == 0) return 0;
-  if (id <= k) return 1;
-  return 2 + (id - 1 - k) / (k * k);
-}
-
-// Block-wide exclusive prefix sum of one int per thread (kRerankThreads threads).
-__device__ int block_exclusive_scan(int v, int* warp_tot /* [32] shared */, int* total) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  int inc = v;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const int t = __shfl_up_sync(kFullMask, inc, o);
-    if (lane >= o) inc += t;
-  }
-  __syncthreads();                 // protect warp_tot from its previous use
-  if (lane == 31) warp_tot[warp] = inc;
-  __syncthreads();
-  int offset = 0, tot = 0;
-  for (int w = 0; w < kRerankThreads / 32; ++w) {
-    const int t = warp_tot[w];
-    if (w < warp) offset += t;
-    tot += t;
-  }
-  *total = tot;
-  return offset + inc - v;
-}
-
-// Dynamic shared memory: ordered cum keys [Nn], selection flags / output rows [Nn].
-__global__ void __launch_bounds__(kRerankThreads) rerank_mask_kernel(const Params p, const DraftIO io) {
-  griddep_wait();
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  const int b = blockIdx.x, tid = threadIdx.x;
-  const int k = p.k, T = p.T;
-  const int D = p.stop_depth[b];
-  const int N = (D >= 1) ? k + (D - 1) * k * k : 0;     // generated non-root nodes
-  uint32_t* key = reinterpret_cast<uint32_t*>(smem_raw);           // key of node id i+1 at [i]
-  int* slot_of = reinterpret_cast<int*>(key + p.Nn);                // output row of node id, -1 = dropped
-  __shared__ int hist[256];
-  __shared__ int warp_tot[32];
-  __shared__ uint32_t s_prefix;
-  __shared__ int s_remaining;
-  __shared__ int out_parent[DDD_MAX_TOTAL + 1];
-
-  const float* cum = p.tree_cum + (size_t)b * p.Nn;
-  const int* tparent = p.tree_parent + (size_t)b * p.Nn;
-  const int* ttoken = p.tree_token + (size_t)b * p.Nn;
-  for (int i = tid; i < N; i += kRerankThreads) key[i] = float_to_ordered(cum[i + 1]);
-  const int m_eff = min(p.m, N);
-  if (tid == 0) { s_prefix = 0u; s_remaining = m_eff; }
-  __syncthreads();
-
-  // ---- radix select: value of the m_eff-th largest key and how many of its ties to keep
-  uint32_t known_mask = 0u;
-  for (int pass = 3; pass >= 0 && m_eff > 0; --pass) {
-    const int shift = 8 * pass;
-    for (int i = tid; i < 256; i += kRerankThreads) hist[i] = 0;
-    __syncthreads();
-    const uint32_t prefix = s_prefix;
-    for (int i = tid; i < N; i += kRerankThreads) {
-      const uint32_t q = key[i];
-      if ((q & known_mask) == prefix) atomicAdd(&hist[(q >> shift) & 0xFF], 1);
-    }
-    __syncthreads();
-    if (tid < 32) {
-      // warp 0 finds the bin holding the `remaining`-th largest key: lane l owns bins 8l .. 8l+7
-      const int remaining = s_remaining;
-      int local[8], mine = 0;
-#pragma unroll
-      for (int i = 0; i < 8; ++i) { local[i] = hist[8 * tid + i]; mine += local[i]; }
-      int above = mine;                                   // suffix sum over lanes >= tid ...
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int t = __shfl_down_sync(kFullMask, above, o);
-        if (tid + o < 32) above += t;
-      }
-      above -= mine;                                      // ... made exclusive: keys in higher lanes' bins
-      if (above < remaining && remaining <= above + mine) {   // exactly one lane
-        int rem = remaining - above, bin = 7;
-        for (; bin > 0; --bin) {
-          if (local[bin] >= rem) break;
-          rem -= local[bin];
-        }
-        s_prefix = prefix | ((uint32_t)(8 * tid + bin) << shift);
-        s_remaining = rem;
-      }
-    }
-    known_mask |= 0xFFu << shift;
-    __syncthreads();
-  }
-  const uint32_t thr = s_prefix;
-  const int keep_ties = s_remaining;      // among keys equal to thr, the lowest node ids win
-
-  // ---- selection flags in node-id order; each thread owns a contiguous chunk of ids
-  const int chunk = (N + kRerankThreads - 1) / kRerankThreads;
-  const int lo = min(N, tid * chunk), hi = min(N, lo + chunk);
-  int n_eq = 0;
-  for (int i = lo; i < hi; ++i) n_eq += (key[i] == thr);
-  int tot_unused;
-  int eq_before = block_exclusive_scan(n_eq, warp_tot, &tot_unused);
-  int n_sel = 0;
-  for (int i = lo; i < hi; ++i) {
-    const uint32_t q = key[i];
-    bool sel = false;
-    if (m_eff > 0) {
-      if (q > thr) sel = true;
-      else if (q == thr) sel = (eq_before++ < keep_ties);
-    }
-    slot_of[i + 1] = sel ? 1 : 0;
-    n_sel += sel;
-  }
-  int n_selected;
-  int sel_before = block_exclusive_scan(n_sel, warp_tot, &n_selected);
-  for (int i = lo; i < hi; ++i) {
-    const bool sel = slot_of[i + 1] != 0;
-    slot_of[i + 1] = sel ? 1 + sel_before : -1;
-    sel_before += sel;
-  }
-  if (tid == 0) slot_of[0] = 0;
-  __syncthreads();
-
-  // ---- emit rows: the root, then the kept nodes in ascending node id
-  const int n_out = 1 + n_selected;
-  const size_t ob = (size_t)b * T;
-  for (int id = tid; id <= N; id += kRerankThreads) {
-    const int slot = slot_of[id];
-    if (slot < 0 || slot >= T) continue;
-    const int dep = node_depth(id, k);
-    const int par = (id == 0) ? -1 : slot_of[tparent[id]];
-    out_parent[slot] = par;
-    io.out.token[ob + slot] = ttoken[id];
-    io.out.parent[ob + slot] = par;
-    io.out.depth[ob + slot] = dep;
-    io.out.position[ob + slot] = p.root_pos[b] + dep;
-    io.out.cum[ob + slot] = cum[id];
-    if (io.trace.node_id) io.trace.node_id[ob + slot] = id;
-  }
-  for (int slot = n_out + tid; slot < T; slot += kRerankThreads) {
-    io.out.token[ob + slot] = -1;
-    io.out.parent[ob + slot] = -1;
-    io.out.depth[ob + slot] = -1;
-    io.out.position[ob + slot] = -1;
-    io.out.cum[ob + slot] = 0.f;
-    if (io.trace.node_id) io.trace.node_id[ob + slot] = -1;
-  }
-  if (tid == 0) {
-    io.out.n_out[b] = n_out;
-    io.out.stop_depth[b] = D;
-    if (b == 0) *io.out.status = *p.dev_status;
-  }
-  __syncthreads();
-
-  // ---- ancestor mask: row i has bit j set iff j is i or an ancestor of i
-  for (int slot = tid; slot < T; slot += kRerankThreads) {
-    uint32_t* row = io.out.mask + (ob + slot) * p.W32;
-    for (int w = 0; w < p.W32; ++w) {
-      uint32_t bits = 0u;
-      if (slot < n_out) {
-        int a = slot;
-        for (int guard = 0; a >= 0 && guard <= DDD_MAX_DEPTH; ++guard) {
-          if ((a >> 5) == w) bits |= 1u << (a & 31);
-          a = out_parent[a];
-        }
-      }
-      row[w] = bits;
-    }
-  }
-  // copy the generated tree for replay, if asked for
-  if (io.trace.tree_token) {
-    for (int id = tid; id < p.Nn; id += kRerankThreads) {
-      const bool gen = id <= N;
-      const size_t o = (size_t)b * p.Nn + id;
-      io.trace.tree_token[o] = gen ? ttoken[id] : -1;
-      if (io.trace.tree_parent) io.trace.tree_parent[o] = gen ? tparent[id] : -1;
-      if (io.trace.tree_cum) io.trace.tree_cum[o] = gen ? cum[id] : 0.f;
-    }
-  }
 }
 
 // Can the partial lists of a block's rows live in its shared memory?  (Host and device agree
@@ -754,17 +761,26 @@ size_t select_smem_bytes(const Params& p, bool lists) {
 bool select_lists_in_smem(const Params& p) {
   return p.lm_ctas <= 320 && select_smem_bytes(p, true) <= 160 * 1024;
 }
-size_t select_smem(const Params& p) { return select_smem_bytes(p, select_lists_in_smem(p)); }
-size_t rerank_smem(const Params& p) { return (size_t)p.Nn * (sizeof(uint32_t) + sizeof(int)); }
+size_t rerank_smem(const Params& p) { return (size_t)p.Nn * (sizeof(uint32_t) + sizeof(short)); }
+// the select kernel's dynamic shared memory also serves the rerank that follows a stop
+size_t select_smem(const Params& p) {
+  const size_t a = select_smem_bytes(p, select_lists_in_smem(p)), b = rerank_smem(p);
+  return a > b ? a : b;
+}
 
 }  // namespace
 
 // ---------------------------------------------------------------------------- launchers
 cudaError_t prepare_tree(const Params& p) {
-  if (select_smem(p) > 180 * 1024 || rerank_smem(p) > 200 * 1024) return cudaErrorInvalidValue;
-  cudaError_t e = allow_max_dynamic_smem(select_gate_step_kernel);
+  // static + dynamic shared memory of the select kernel must fit one block's limit
+  cudaFuncAttributes fa;
+  cudaError_t e = cudaFuncGetAttributes(&fa, select_gate_step_kernel);
   if (e != cudaSuccess) return e;
-  return allow_max_dynamic_smem(rerank_mask_kernel);
+  int dev = 0, limit = 0;
+  if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+  if ((e = cudaDeviceGetAttribute(&limit, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev)) != cudaSuccess) return e;
+  if (fa.sharedSizeBytes + select_smem(p) > (size_t)limit) return cudaErrorInvalidValue;
+  return allow_max_dynamic_smem(select_gate_step_kernel);
 }
 
 cudaError_t launch_init(const Params& p, const DraftIO&, const void* root_hidden, const int* root_token,
@@ -794,20 +810,6 @@ cudaError_t launch_select(const Params& p, const DraftIO& io, int d, bool pdl, c
   cfg.attrs = attr;
   cfg.numAttrs = pdl ? 2 : 1;
   return cudaLaunchKernelEx(&cfg, select_gate_step_kernel, p, io, d, select_lists_in_smem(p) ? 1 : 0, cond, set_cond ? 1 : 0);
-}
-
-cudaError_t launch_rerank(const Params& p, const DraftIO& io, bool pdl, cudaStream_t st) {
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)p.B, 1, 1);
-  cfg.blockDim = dim3(kRerankThreads, 1, 1);
-  cfg.dynamicSmemBytes = rerank_smem(p);
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = pdl ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, rerank_mask_kernel, p, io);
 }
 
 }  // namespace ddd

@@ -188,11 +188,11 @@ def test_graph_mode_host_variant_and_determinism():
                      roots["root_pos"].pin_memory(), host_out)
     for name in host_out:
         np.testing.assert_array_equal(host_out[name].numpy(), a[name], err_msg=name)
-    assert P.ddd_launches_per_draft(eng_s.handle, 1) == 2 + 2 * cfg.max_depth
+    assert P.ddd_launches_per_draft(eng_s.handle, 1) == 1 + 2 * cfg.max_depth
     # captured drafts end early after passes 3, 5 and 8 (every step checked, n = 12)
     assert cfg.max_depth == 12 and cfg.check_mask & 0xFFF == 0xFFF
     for needed, launched in [(1, 3), (2, 3), (3, 3), (4, 5), (5, 5), (6, 8), (8, 8), (9, 12), (12, 12)]:
-        assert P.ddd_launches_per_draft(eng_g.handle, needed) == 2 + 2 * launched, needed
+        assert P.ddd_launches_per_draft(eng_g.handle, needed) == 1 + 2 * launched, needed
     assert 1 <= P.ddd_lm_head_blocks(eng_s.handle) <= 512
     eng_s.close()
     eng_g.close()
