@@ -174,13 +174,15 @@ cudaError_t enqueue_passes(const ddd_handle* h, const DraftIO& io, bool pdl, int
 // node that only a sequence still drafting after the previous group switches on; the bodies
 // nest.  Boundaries are put after checked steps only (nothing can stop elsewhere), the first
 // not before pass 3, the groups growing by one pass each (3, 5, 8, 12 when every step is
-// checked), at most kMaxGraphLevels of them: a skipped or entered IF node costs about as much as
-// an idle pass, so a deep draft should not cross many.
+// checked), at most kMaxGraphLevels of them: entering an IF body costs about as much as two to
+// three idle passes, so a deep draft should not cross many.  None at all when the threshold is so
+// low that drafting always runs to pass n.
 
 int graph_boundaries(const ddd_config& cfg, int* bounds /* [kMaxGraphLevels] */) {
   const int n = cfg.max_depth;
   int count = 0;
   if (n <= kFirstBoundary + 1) return 0;
+  if (!(cfg.threshold > -1e30f)) return 0;   // no finite H is below such a threshold: fixed-depth drafting
   int want = kFirstBoundary, gap = 2;
   for (int d = kFirstBoundary; d < n && count < kMaxGraphLevels; ++d) {
     if (d < want || !((cfg.check_mask >> (d - 1)) & 1u)) continue;

@@ -224,6 +224,8 @@ def test_captured_drafts_of_every_stop_depth_equal_stream_launches(schedule):
                 np.testing.assert_array_equal(a[name], b[name], err_msg=f"{name} x={cfg.threshold}")
             seen.update(a["stop_depth"].tolist())
         parity.compare_with_oracle(cfg, weights_for(cfg), roots, b)
+        if cfg.threshold == NEG:      # fixed-depth drafting: no conditional groups at all
+            assert P.ddd_launches_per_draft(eng_g.handle, 1) == 1 + 2 * cfg.max_depth
         eng_s.close()
         eng_g.close()
     if schedule == "every_step":
