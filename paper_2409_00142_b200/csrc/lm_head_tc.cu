@@ -40,16 +40,23 @@ constexpr int kSmemLimit = 232448;      // 227 KB opt-in limit per block
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 constexpr int kL2PrefetchBytes = 128 * 1024;   // per block, ahead of the dependency wait (about 64 MB in all)
 
+// Accumulator chunks (of kChunkCols beam rows) the epilogue can take out of tensor memory at a
+// time: one per group of four epilogue warps, each of which reads one lane quarter.
+__host__ __device__ inline int epi_group(int R) {
+  const int n_chunks = (R + kChunkCols - 1) / kChunkCols;
+  return n_chunks < kEpiWarps / 4 ? n_chunks : kEpiWarps / 4;
+}
+
 struct SmemPlan {
   int a, b, zt, key, ms, plant, live, bars, tmem_ptr, abort_flag, total;
 };
 
-__host__ __device__ inline SmemPlan smem_plan(int stages, int ksub, int n_pad, int R, int k) {
+__host__ __device__ inline SmemPlan smem_plan(int stages, int ksub, int n_pad, int R, int k, int cpg) {
   SmemPlan s;
   int off = 0;
   s.a = off; off += stages * ksub * kABytes;
   s.b = off; off += stages * ksub * n_pad * kBlockK * 2;
-  s.zt = off; off += kChunkCols * kTile * 4;
+  s.zt = off; off += cpg * kChunkCols * kTile * 4;
   s.key = off; off += R * k * 8;
   s.ms = off; off += R * 8;
   s.plant = off; off += R * 4;
@@ -196,7 +203,7 @@ __device__ __forceinline__ uint32_t make_instr_desc(int n) {
 __global__ void __launch_bounds__(kTcThreads, 1)
 lm_head_tc_kernel(const Params p, const unsigned char* __restrict__ w_packed,
                   const __grid_constant__ CUtensorMap map_h, const int d, const int force_all,
-                  const int n_pad, const int stages, const int tmem_cols, const int ksub) {
+                  const int n_pad, const int stages, const int tmem_cols, const int ksub, const int cpg) {
   // The kernel may have been launched while the select kernel of the previous pass is still
   // running (programmatic dependent launch).  Until griddep_wait() below it touches nothing
   // that kernel writes, except for one speculative look at the activity counter: if drafting
@@ -218,7 +225,7 @@ lm_head_tc_kernel(const Params p, const unsigned char* __restrict__ w_packed,
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(
       (reinterpret_cast<uintptr_t>(smem_dyn) + 1023u) & ~static_cast<uintptr_t>(1023u));
-  const SmemPlan sp = smem_plan(stages, ksub, n_pad, p.R, p.k);
+  const SmemPlan sp = smem_plan(stages, ksub, n_pad, p.R, p.k, cpg);
   float* zt = reinterpret_cast<float*>(smem + sp.zt);
   unsigned long long* st_key = reinterpret_cast<unsigned long long*>(smem + sp.key);
   float2* st_ms = reinterpret_cast<float2*>(smem + sp.ms);
@@ -254,22 +261,27 @@ lm_head_tc_kernel(const Params p, const unsigned char* __restrict__ w_packed,
   // One (tile, K-group) step of the pipeline: which packed chunk it reads and where it lands.
   const int total_iters = n_tiles * num_kb;
   const int prefill = total_iters < stages ? total_iters : stages;
+  // Both are called by all 32 lanes of warp 0.  Issuing a copy occupies the issuing thread for a
+  // few hundred cycles whatever its size, so the copies of a stage go out from different lanes in
+  // one warp-wide instruction: lane kk sends K-block kk of W, lane ksub the h slice.
   unsigned long long evict_first = 0ull;
   auto issue_w = [&](int it, int stage) {
     const int t = it / num_kb, kb = it - t * num_kb;
     const int nu = min(4, my_units - 4 * t);
     const uint32_t full = bar_full + 8u * stage;
-    mbar_expect_tx(full, (uint32_t)ksub * ((uint32_t)nu * kUnitBytes + b_bytes));   // W and h bytes of the stage
+    if (lane == 0) mbar_expect_tx(full, (uint32_t)ksub * ((uint32_t)nu * kUnitBytes + b_bytes));   // W and h bytes
+    __syncwarp();
     // W: for each 64-element K-block the tile's units are one contiguous run of the packed copy
     const unsigned char* src = w_packed + ((size_t)(kb * ksub) * n_units + (size_t)(unit0 + 4 * t)) * kUnitBytes;
     const uint32_t dst = a_base + (uint32_t)stage * a_stage;
-    for (int kk = 0; kk < ksub; ++kk)
-      bulk_load_hint(dst + (uint32_t)kk * kABytes, src + (size_t)kk * n_units * kUnitBytes, (uint32_t)nu * kUnitBytes,
+    if (lane < ksub)
+      bulk_load_hint(dst + (uint32_t)lane * kABytes, src + (size_t)lane * n_units * kUnitBytes, (uint32_t)nu * kUnitBytes,
                      full, evict_first);
   };
   auto issue_h = [&](int it, int stage) {
     // h: ksub K-blocks of all beam rows in one tensor copy
-    tma_load_3d(b_base + (uint32_t)stage * b_stage, &map_h, bar_full + 8u * stage, 0, 0, (it % num_kb) * ksub);
+    if (lane == ksub)
+      tma_load_3d(b_base + (uint32_t)stage * b_stage, &map_h, bar_full + 8u * stage, 0, 0, (it % num_kb) * ksub);
   };
 
   if (threadIdx.x == 0) {
@@ -285,6 +297,9 @@ lm_head_tc_kernel(const Params p, const unsigned char* __restrict__ w_packed,
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncwarp();
+  if (warp == 0) {
     // W does not depend on the previous kernel: fill the ring with it right away.
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(evict_first));
     if (spec_active)
@@ -307,13 +322,14 @@ lm_head_tc_kernel(const Params p, const unsigned char* __restrict__ w_packed,
   griddep_launch_dependents();
   if (!force_all && *p.n_active == 0) {
     // every sequence has stopped: complete and await the copies already in flight, then leave
-    if (spec_active && threadIdx.x == 0) {
+    if (spec_active && warp == 0) {
       for (int it = 0; it < prefill; ++it) issue_h(it, it);
+      __syncwarp();
       for (int it = 0; it < prefill; ++it) mbar_wait(bar_full + 8u * it, 0u, abort_flag, p.dev_status, false);
     }
     return;
   }
-  if (threadIdx.x == 0) {
+  if (warp == 0) {
     if (!spec_active)
       for (int it = 0; it < prefill; ++it) issue_w(it, it);
     for (int it = 0; it < prefill; ++it) issue_h(it, it);
@@ -346,10 +362,8 @@ lm_head_tc_kernel(const Params p, const unsigned char* __restrict__ w_packed,
     for (int it = prefill; it < total_iters; ++it) {
       ok = __all_sync(kFullMask, mbar_wait(bar_empty + 8u * stage, phase ^ 1u, abort_flag, p.dev_status));
       if (!ok) break;
-      if (lane == 0) {
-        issue_w(it, stage);
-        issue_h(it, stage);
-      }
+      issue_w(it, stage);
+      issue_h(it, stage);
       __syncwarp();
       ++issued;
       if (++stage == stages) { stage = 0; phase ^= 1u; }
@@ -406,9 +420,12 @@ lm_head_tc_kernel(const Params p, const unsigned char* __restrict__ w_packed,
     }
   } else {
     // ======================================================================= epilogue
-    const int quarter = warp & 3;            // tensor-memory lanes this warp may read (loader warps)
-    const int ew = warp - 2;                 // owner of beam rows r with r % kEpiWarps == ew
-    const bool loader = ew < 4;              // warps 2..5 cover the four lane quarters
+    // Warp ew reads lane quarter ew % 4 of chunk ew / 4 of the current group of chunks, so up to
+    // 64 beam rows leave tensor memory between two barriers; then every warp folds the rows r
+    // with r % kEpiWarps == ew.
+    const int quarter = warp & 3;            // tensor-memory lanes this warp may read
+    const int ew = warp - 2;
+    const int lw = ew >> 2;                  // chunk of the group this warp loads
     const int n_chunks = (p.R + kChunkCols - 1) / kChunkCols;
     bool ok = true;
     for (int t = 0; t < n_tiles && ok; ++t) {
@@ -416,7 +433,7 @@ lm_head_tc_kernel(const Params p, const unsigned char* __restrict__ w_packed,
       const uint32_t acc_phase = (uint32_t)(t >> 1) & 1u;
       const int rows = min(4, my_units - 4 * t) * kUnitRows;
       const int row0 = (unit0 + 4 * t) * kUnitRows;
-      // The four warps must leave this wait together (they share named barrier 1 below).
+      // All epilogue warps must leave this wait together (they share named barrier 1 below).
       ok = epilogue_all(mbar_wait(bar_tfull + 8u * acc, acc_phase, abort_flag, p.dev_status, false));
       if (!ok) break;
       tc_fence_after();
@@ -424,28 +441,28 @@ lm_head_tc_kernel(const Params p, const unsigned char* __restrict__ w_packed,
       const int v = row0 + vrow;
       const bool v_ok = vrow < rows && v < p.V;
       const float bias = (v_ok && p.bias) ? p.bias[v] : 0.f;
-      for (int ch = 0; ch < n_chunks; ++ch) {
-        const int c0 = ch * kChunkCols;
-        if (loader) {
+      for (int g0 = 0; g0 < n_chunks; g0 += cpg) {
+        const int ch = g0 + lw;
+        if (lw < cpg && ch < n_chunks) {
+          const int c0 = ch * kChunkCols;
           float accv[16];
           tc_load_16cols(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * n_pad + c0), accv);
-          if (ch == n_chunks - 1) {
-            // accumulator fully read by this warp: hand it back to the MMA warp
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_tempty + 8u * acc);
-          }
 #pragma unroll
           for (int c = 0; c < kChunkCols; ++c) {
             const int r = c0 + c;
             float z = neg_inf();
             if (v_ok && r < p.R && s_plant[r] != v) z = fmaf(accv[c], p.s, bias);
-            zt[c * kTile + vrow] = z;
+            zt[(lw * kChunkCols + c) * kTile + vrow] = z;
           }
+          tc_fence_before();
         }
         epilogue_barrier();
-        for (int rr = ew; rr < kChunkCols; rr += kEpiWarps) {
-          const int r = c0 + rr;
+        if (g0 + cpg >= n_chunks && ew < 4 && lane == 0) {
+          // every warp has read its part of the accumulator: hand it back to the MMA warp
+          mbar_arrive(bar_tempty + 8u * acc);
+        }
+        for (int rr = ew; rr < cpg * kChunkCols; rr += kEpiWarps) {
+          const int r = g0 * kChunkCols + rr;
           if (r >= p.R || !s_live[r]) continue;
           float2 ms = st_ms[r];
           unsigned long long key = lane < p.k ? st_key[r * p.k + lane] : 0ull;
@@ -549,17 +566,24 @@ int tc_plan_create(const Params& p, int sm_count, void* w_packed, TcPlan* plan) 
   const int n_units = (p.V + kUnitRows - 1) / kUnitRows;
   int ctas = sm_count < n_units ? sm_count : n_units;
   if (ctas > kMaxLmCtas) ctas = kMaxLmCtas;
-  // K-blocks per stage: as many as still leave a ring of three stages (the producer thread
-  // pays a fixed few hundred cycles per copy it issues, so few large copies win), at most 4.
-  int ksub = 4;
-  while (ksub > 1 && (p.Hd % (kBlockK * ksub) != 0 || smem_plan(3, ksub, n_pad, p.R, p.k).total + 1024 > kSmemLimit))
+  // K-blocks per stage: as many as still leave a ring of two stages, at most 4.  A pipeline step
+  // has a fixed cost of about half a microsecond (barrier round trip, copy issue), so few large
+  // stages win over many small ones: measured with 32 and 64 beam rows, two stages of four
+  // K-blocks beat five of two by 5-7 %.
+  // The epilogue takes up to four chunks of 16 beam rows out of tensor memory between two
+  // barriers, 8 KB of shared memory each; it gives way to the stage size when both do not fit.
+  int ksub = 4, cpg = epi_group(p.R);
+  auto fits = [&](int st, int ks, int cg) { return smem_plan(st, ks, n_pad, p.R, p.k, cg).total + 1024 <= kSmemLimit; };
+  for (;;) {
+    if (p.Hd % (kBlockK * ksub) == 0 && fits(2, ksub, cpg)) break;
+    if (cpg > 1) { cpg /= 2; continue; }
+    if (ksub == 1) break;
     ksub /= 2;
-  // with many beam rows the h slice of a stage outweighs the W tile; two K-blocks in a ring of
-  // two stages still beat one K-block per stage (half as many pipeline steps)
-  if (ksub == 1 && p.Hd % (kBlockK * 2) == 0 && smem_plan(2, 2, n_pad, p.R, p.k).total + 1024 <= kSmemLimit) ksub = 2;
+    cpg = epi_group(p.R);
+  }
   int stages = 0;
   for (int s = 8; s >= 2; --s) {
-    if (smem_plan(s, ksub, n_pad, p.R, p.k).total + 1024 <= kSmemLimit) { stages = s; break; }
+    if (fits(s, ksub, cpg)) { stages = s; break; }
   }
   if (stages == 0) return DDD_ERR_UNSUPPORTED;
   plan->ksub = ksub;
@@ -567,7 +591,8 @@ int tc_plan_create(const Params& p, int sm_count, void* w_packed, TcPlan* plan) 
   plan->n_pad = n_pad;
   plan->stages = stages;
   plan->tmem_cols = cols;
-  plan->smem = (size_t)smem_plan(stages, ksub, n_pad, p.R, p.k).total + 1024;
+  plan->epi_chunks = cpg;
+  plan->smem = (size_t)smem_plan(stages, ksub, n_pad, p.R, p.k, cpg).total + 1024;
   plan->w_packed = static_cast<unsigned char*>(w_packed);
   {
     const size_t chunks = tc_packed_bytes(p.V, p.Hd) / kUnitBytes;
@@ -594,7 +619,7 @@ cudaError_t launch_lm_head_tc(const Params& p, const TcPlan& plan, int d, int fo
   cfg.attrs = attr;
   cfg.numAttrs = pdl ? 1 : 0;
   return cudaLaunchKernelEx(&cfg, lm_head_tc_kernel, p, (const unsigned char*)plan.w_packed, plan.map_h[(d - 1) & 1], d,
-                            force_all, plan.n_pad, plan.stages, plan.tmem_cols, plan.ksub);
+                            force_all, plan.n_pad, plan.stages, plan.tmem_cols, plan.ksub, plan.epi_chunks);
 }
 
 }  // namespace ddd

@@ -14,6 +14,7 @@ struct TcPlan {
   int n_pad;              // MMA N: beam rows rounded up to a multiple of 16
   int stages;             // depth of the shared-memory ring
   int ksub;               // 64-element K-blocks per stage
+  int epi_chunks;         // 16-row accumulator chunks the epilogue unloads per barrier pair (1..4)
   int tmem_cols;          // allocated tensor-memory columns (power of two)
   size_t smem;            // dynamic shared memory per block
 };
