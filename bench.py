@@ -35,7 +35,7 @@ NEG = -1e30
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes (read + write) of one LM-head launch from the ncu capture summarised under
 # profiles/, valid only while the kernel source is the one that was profiled.
-NCU_TRAFFIC = {"llama2_7b": {"bytes": 265.9e6, "source_sha256_16": "b6a5f31373c10d45",
+NCU_TRAFFIC = {"llama2_7b": {"bytes": 265.6e6, "source_sha256_16": "9270d077708fda9d",
                              "profile": "profiles/lm_head_tc_llama2_7b.md"}}
 CLOCK_QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
                "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
