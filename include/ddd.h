@@ -200,9 +200,12 @@ int ddd_draft_host_gated(ddd_handle *h, const void *root_hidden, const int32_t *
 /*
  * Same draft with HOST buffers: copies the inputs to staging space inside the workspace,
  * runs the draft, copies every ddd_output field back and synchronises the stream before
- * returning.  All pointers (inputs and the fields of `out`) are HOST pointers; pinned
- * memory makes the copies asynchronous but is not required.  Returns the device status
- * (e.g. DDD_ERR_TIMEOUT) if the draft itself reported one.
+ * returning.  All pointers (inputs and the fields of `out`) are HOST pointers of ordinary or
+ * pinned memory: the call packs them into one pinned buffer of its own (allocated on the first
+ * call), so there is one copy in each direction.  In DDD_LAUNCH_GRAPH mode with a non-default
+ * stream the whole call is a single graph launch (input copy, first kernel, passes, output
+ * copy), captured on the first call per stream.  Returns the device status (e.g.
+ * DDD_ERR_TIMEOUT) if the draft itself reported one.
  */
 int ddd_draft_host(ddd_handle *h, const void *root_hidden, const int32_t *root_token,
                    const int32_t *root_pos, const ddd_output *out, void *cuda_stream);

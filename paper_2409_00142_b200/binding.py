@@ -269,7 +269,11 @@ class DraftEngine:
 
     def draft_host(self, root_hidden, root_token, root_pos, host_out: Dict) -> None:
         """Host-buffer variant: CPU tensors in, CPU tensors (same names as self.out) out."""
-        c_out = DddOutput(**{name: host_out[name].data_ptr() for name in self.out})
+        cached = getattr(self, "_host_out_struct", None)
+        if cached is None or cached[0] is not host_out:       # marshal the ten pointers once per buffer set
+            cached = (host_out, DddOutput(**{name: host_out[name].data_ptr() for name in self.out}))
+            self._host_out_struct = cached
+        c_out = cached[1]
         ddd_draft_host(self.handle, root_hidden.data_ptr(), root_token.data_ptr(), root_pos.data_ptr(),
                        c_out, self.stream_ptr())
 

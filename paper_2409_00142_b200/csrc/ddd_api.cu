@@ -133,6 +133,8 @@ struct ddd_handle {
   TcPlan tc;
   // graph cache (one entry)
   cudaGraphExec_t exec;
+  cudaGraphExec_t exec_host;    // ddd_draft_host's graph: input copy, init, passes, output copy
+  cudaStream_t host_stream;     // stream exec_host was captured on
   GraphKey key;
   bool have_graph;
   bool use_pdl;    // programmatic dependent launch between the kernels of a draft
@@ -158,11 +160,14 @@ cudaError_t launch_lm_head(const ddd_handle* h, int d, int force_all, bool pdl, 
 // serialisation: it may start while its predecessor runs and waits for it on the device.
 // Passes first..last are enqueued; the select kernel of pass `cond_pass` (0 = none) switches
 // the graph conditional `cond` on if its sequence goes on.
+// `after_kernel`: the first LM-head launch directly follows a kernel of this library in the same
+// stream or capture (the init kernel), so it may be a programmatic dependent too.
 cudaError_t enqueue_passes(const ddd_handle* h, const DraftIO& io, bool pdl, int first, int last,
-                           cudaGraphConditionalHandle cond, int cond_pass, cudaStream_t st) {
+                           cudaGraphConditionalHandle cond, int cond_pass, cudaStream_t st,
+                           bool after_kernel = false) {
   cudaError_t e = cudaSuccess;
   for (int d = first; d <= last && e == cudaSuccess; ++d) {
-    e = launch_lm_head(h, d, 0, pdl && d > first, st);
+    e = launch_lm_head(h, d, 0, pdl && (d > first || after_kernel), st);
     if (e == cudaSuccess) e = launch_select(h->p, io, d, pdl, cond, d == cond_pass, st);
   }
   return e;
@@ -203,8 +208,11 @@ struct CaptureLog {
 
 // Captures group `level` (passes first..bounds[level], or first..n for the last group) into
 // `graph`, followed by the IF node that guards the next group.
+// With `host_wrap` the top level also holds what ddd_draft_host puts around a draft: the copy of
+// the packed inputs from the pinned bounce buffer, the init kernel on the staged inputs, and,
+// last, the copy of the packed results back to the bounce buffer.
 bool capture_level(ddd_handle* h, const DraftIO& io, bool pdl, cudaStream_t st, cudaGraph_t graph,
-                   const int* bounds, int n_bounds, int level, int first, CaptureLog& log) {
+                   const int* bounds, int n_bounds, int level, int first, CaptureLog& log, bool host_wrap) {
   const int n = h->p.n;
   const bool has_if = level < n_bounds;
   const int last = has_if ? bounds[level] : n;
@@ -219,7 +227,14 @@ bool capture_level(ddd_handle* h, const DraftIO& io, bool pdl, cudaStream_t st, 
                   id + 3);
     capturing = ok;
   }
-  if (ok) ok = log.good(enqueue_passes(h, io, pdl, first, last, cond, has_if ? last : 0, st), id + 4);
+  const bool wrap = host_wrap && level == 0;
+  if (ok && wrap) {
+    const Layout& L = h->L;
+    ok = log.good(cudaMemcpyAsync(h->ws + L.in_hidden, h->bounce, L.in_bytes, cudaMemcpyHostToDevice, st), id + 1) &&
+         log.good(launch_init(h->p, io, h->ws + L.in_hidden, reinterpret_cast<const int*>(h->ws + L.in_token),
+                              reinterpret_cast<const int*>(h->ws + L.in_pos), st), id + 1);
+  }
+  if (ok) ok = log.good(enqueue_passes(h, io, pdl, first, last, cond, has_if ? last : 0, st, wrap), id + 4);
   if (ok && has_if) {
     // splice the IF node in behind the captured passes
     cudaStreamCaptureStatus status;
@@ -239,31 +254,46 @@ bool capture_level(ddd_handle* h, const DraftIO& io, bool pdl, cudaStream_t st, 
     }
     if (ok) ok = log.good(cudaStreamUpdateCaptureDependencies(st, &node, 1, cudaStreamSetCaptureDependencies), id + 7);
   }
+  if (ok && wrap)
+    ok = log.good(cudaMemcpyAsync(h->bounce, h->ws + h->L.out_block, h->L.out_bytes, cudaMemcpyDeviceToHost, st), id + 8);
   if (capturing) {
     cudaGraph_t done = nullptr;
     if (!log.good(cudaStreamEndCapture(st, &done), id + 9)) ok = false;
   }
-  if (ok && body) ok = capture_level(h, io, pdl, st, body, bounds, n_bounds, level + 1, last + 1, log);
+  if (ok && body) ok = capture_level(h, io, pdl, st, body, bounds, n_bounds, level + 1, last + 1, log, host_wrap);
   return ok;
 }
 
 // Captures everything after the init kernel into h->exec, with IF nodes after the first
 // `n_bounds` boundaries.  Returns false (and leaves no graph) on any failure.
-bool capture_graph(ddd_handle* h, const DraftIO& io, bool pdl, int n_bounds, cudaStream_t st) {
+bool capture_graph(ddd_handle* h, const DraftIO& io, bool pdl, int n_bounds, cudaStream_t st,
+                   bool host_wrap = false) {
   cudaGraph_t graph = nullptr;
+  cudaGraphExec_t* exec = host_wrap ? &h->exec_host : &h->exec;
   CaptureLog log;
   bool ok = log.good(cudaGraphCreate(&graph, 0), 1);
-  if (ok) ok = capture_level(h, io, pdl, st, graph, h->bounds, n_bounds, 0, 1, log);
-  if (ok) ok = log.good(cudaGraphInstantiate(&h->exec, graph, 0), 99);
+  if (ok) ok = capture_level(h, io, pdl, st, graph, h->bounds, n_bounds, 0, 1, log, host_wrap);
+  if (ok) ok = log.good(cudaGraphInstantiate(exec, graph, 0), 99);
   if (graph) cudaGraphDestroy(graph);
   if (!ok) {
     note_cuda_error(1000 + log.step);   // 1000 + 10 * group + index of the capture step that failed
-    h->exec = nullptr;
+    *exec = nullptr;
     return false;
   }
-  h->graph_pdl = pdl;
-  h->graph_bounds = n_bounds;
+  if (!host_wrap) {
+    h->graph_pdl = pdl;
+    h->graph_bounds = n_bounds;
+  }
   return true;
+}
+
+// Tries the capture with programmatic dependent launches and nested IF nodes first, then with a
+// single IF node, then as a plain stream-ordered sequence.
+bool capture_with_fallbacks(ddd_handle* h, const DraftIO& io, cudaStream_t st, bool host_wrap) {
+  const int one = h->n_bounds < 1 ? h->n_bounds : 1;
+  return (h->use_pdl && capture_graph(h, io, true, h->n_bounds, st, host_wrap)) ||
+         (h->use_pdl && one != h->n_bounds && capture_graph(h, io, true, one, st, host_wrap)) ||
+         capture_graph(h, io, false, one, st, host_wrap);
 }
 
 bool aligned16(const void* q) { return (reinterpret_cast<uintptr_t>(q) & 15u) == 0; }
@@ -305,6 +335,8 @@ int ddd_create(const ddd_config* cfg, const void* W, const void* E, const float*
   h->use_pdl = cfg->launch_mode != DDD_LAUNCH_PLAIN;
   h->graph_pdl = false;
   h->exec = nullptr;
+  h->exec_host = nullptr;
+  h->host_stream = nullptr;
   h->bounce = nullptr;
   h->bounce_bytes = 0;
 
@@ -384,14 +416,7 @@ int ddd_draft(ddd_handle* h, const void* root_hidden, const int32_t* root_token,
     if (!h->have_graph || std::memcmp(&key, &h->key, sizeof key) != 0) {
       if (h->exec) { cudaGraphExecDestroy(h->exec); h->exec = nullptr; }
       h->have_graph = false;
-      // capture with programmatic dependent launches; if this driver cannot capture or
-      // instantiate them, capture the plain stream-ordered sequence instead; likewise fall back
-      // from nested IF nodes to a single one
-      const int one = h->n_bounds < 1 ? h->n_bounds : 1;
-      if (!(h->use_pdl && capture_graph(h, io, true, h->n_bounds, st)) &&
-          !(h->use_pdl && one != h->n_bounds && capture_graph(h, io, true, one, st)) &&
-          !capture_graph(h, io, false, one, st))
-        return DDD_ERR_CUDA;
+      if (!capture_with_fallbacks(h, io, st, false)) return DDD_ERR_CUDA;
       h->key = key;
       h->have_graph = true;
     }
@@ -403,7 +428,7 @@ int ddd_draft(ddd_handle* h, const void* root_hidden, const int32_t* root_token,
     return DDD_OK;
   }
   if (launch_init(h->p, io, root_hidden, root_token, root_pos, st) != cudaSuccess ||
-      enqueue_passes(h, io, h->use_pdl, 1, h->p.n, 0, 0, st) != cudaSuccess) {
+      enqueue_passes(h, io, h->use_pdl, 1, h->p.n, 0, 0, st, true) != cudaSuccess) {
     note_cuda_error(__LINE__);
     return DDD_ERR_CUDA;
   }
@@ -463,10 +488,6 @@ int ddd_draft_host(ddd_handle* h, const void* root_hidden, const int32_t* root_t
   std::memcpy(h->bounce, root_hidden, B * p.Hd * elt);
   std::memcpy(h->bounce + (L.in_token - L.in_hidden), root_token, B * 4);
   std::memcpy(h->bounce + (L.in_pos - L.in_hidden), root_pos, B * 4);
-  if (cudaMemcpyAsync(h->ws + L.in_hidden, h->bounce, L.in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) {
-    note_cuda_error(__LINE__);
-    return DDD_ERR_CUDA;
-  }
   unsigned char* ob = h->ws + L.out_block;
   ddd_output dev;
   dev.n_out = reinterpret_cast<int32_t*>(ob + L.o_n_out);
@@ -479,15 +500,36 @@ int ddd_draft_host(ddd_handle* h, const void* root_hidden, const int32_t* root_t
   dev.mask = reinterpret_cast<uint32_t*>(ob + L.o_mask);
   dev.H_trace = reinterpret_cast<float*>(ob + L.o_H);
   dev.status = reinterpret_cast<int32_t*>(ob + L.o_status);
-  const int rc = ddd_draft(h, h->ws + L.in_hidden, reinterpret_cast<const int32_t*>(h->ws + L.in_token),
-                           reinterpret_cast<const int32_t*>(h->ws + L.in_pos), &dev, nullptr, cuda_stream);
-  if (rc != DDD_OK) return rc;
-  // one device-to-host copy of the packed results, then scatter to the caller's arrays
-  if (cudaMemcpyAsync(h->bounce, ob, L.out_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
-      cudaStreamSynchronize(st) != cudaSuccess) {
-    note_cuda_error(__LINE__);
-    return DDD_ERR_CUDA;
+  if (h->cfg.launch_mode == DDD_LAUNCH_GRAPH && st != nullptr) {
+    // the whole call is one graph launch: input copy, init kernel, the passes, output copy
+    if (!h->exec_host || h->host_stream != st) {
+      if (h->exec_host) { cudaGraphExecDestroy(h->exec_host); h->exec_host = nullptr; }
+      DraftIO io;
+      io.out = dev;
+      std::memset(&io.trace, 0, sizeof io.trace);
+      if (!capture_with_fallbacks(h, io, st, true)) return DDD_ERR_CUDA;
+      h->host_stream = st;
+    }
+    if (cudaGraphLaunch(h->exec_host, st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess) {
+      note_cuda_error(__LINE__);
+      return DDD_ERR_CUDA;
+    }
+  } else {
+    if (cudaMemcpyAsync(h->ws + L.in_hidden, h->bounce, L.in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+      note_cuda_error(__LINE__);
+      return DDD_ERR_CUDA;
+    }
+    const int rc = ddd_draft(h, h->ws + L.in_hidden, reinterpret_cast<const int32_t*>(h->ws + L.in_token),
+                             reinterpret_cast<const int32_t*>(h->ws + L.in_pos), &dev, nullptr, cuda_stream);
+    if (rc != DDD_OK) return rc;
+    // one device-to-host copy of the packed results
+    if (cudaMemcpyAsync(h->bounce, ob, L.out_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) {
+      note_cuda_error(__LINE__);
+      return DDD_ERR_CUDA;
+    }
   }
+  // scatter the packed results to the caller's arrays
   const unsigned char* hb = h->bounce;
   std::memcpy(out->n_out, hb + L.o_n_out, B * 4);
   std::memcpy(out->stop_depth, hb + L.o_stop, B * 4);
@@ -532,6 +574,7 @@ int ddd_lm_head_blocks(const ddd_handle* h) {
 int ddd_destroy(ddd_handle* h) {
   if (!h) return DDD_ERR_INVALID_ARG;
   if (h->exec) cudaGraphExecDestroy(h->exec);
+  if (h->exec_host) cudaGraphExecDestroy(h->exec_host);
   if (h->bounce) cudaFreeHost(h->bounce);
   delete h;
   return DDD_OK;

@@ -188,6 +188,14 @@ def test_graph_mode_host_variant_and_determinism():
                      roots["root_pos"].pin_memory(), host_out)
     for name in host_out:
         np.testing.assert_array_equal(host_out[name].numpy(), a[name], err_msg=name)
+    # in graph mode the host-buffer call is one graph launch (copies and init kernel included)
+    with torch.cuda.stream(torch.cuda.Stream()):
+        for r, want in ((roots, a), (other, c), (roots, a)):
+            host_g = eng_g.make_host_out()
+            eng_g.draft_host(r["root_hidden"].pin_memory(), r["root_token"].pin_memory(),
+                             r["root_pos"].pin_memory(), host_g)
+            for name in host_g:
+                np.testing.assert_array_equal(host_g[name].numpy(), want[name], err_msg=name)
     assert P.ddd_launches_per_draft(eng_s.handle, 1) == 1 + 2 * cfg.max_depth
     # captured drafts end early after passes 3, 5 and 8 (every step checked, n = 12)
     assert cfg.max_depth == 12 and cfg.check_mask & 0xFFF == 0xFFF
