@@ -160,6 +160,45 @@ def test_edge_shapes_match_oracle(case, kernel):
     eng.close()
 
 
+# ----------------------------------------------------------------------------- seeded random shapes
+def random_shapes():
+    """Sixteen seeded configurations spread over the legal ranges: beam rows 1..256 (so every
+    epilogue grouping and stage size of the tensor-core kernel occurs), ragged vocabularies,
+    sparse and dense check schedules, planted rows, Zipf bias, both launch modes."""
+    rng = np.random.default_rng(20240900)
+    out = []
+    while len(out) < 16:
+        k = int(rng.choice([1, 2, 3, 5, 8, 10, 13, 16, 17, 24, 31, 32]))
+        batch = int(rng.choice([1, 1, 2, 3, 5, 8]))
+        if batch * k > 256:
+            continue
+        n = int(rng.integers(1, 9))
+        if 1 + k + (n - 1) * k * k > 6000:
+            continue
+        hidden = 64 * int(rng.integers(1, 9))
+        vocab = int(rng.integers(k + 1, 5000))
+        m = int(rng.integers(1, 200))
+        mask = int(rng.integers(0, 1 << n)) if rng.random() < 0.5 else 0xFFFFFFFF
+        base = S.CONFIGS[str(rng.choice(["llama2_7b", "vicuna_13b", "llama3_8b_128k"]))]
+        out.append(S.scaled_down(base, hidden, vocab, batch=batch, k=k, max_depth=n, total_tokens=m,
+                                 check_mask=mask, threshold=float(rng.choice([-1.0, -3.0, -6.0, -12.0])),
+                                 seed=int(rng.integers(1 << 30))))
+    return out
+
+
+@pytest.mark.parametrize("index", range(16))
+def test_random_shapes_match_oracle(index):
+    cfg = random_shapes()[index]
+    mode = P.DDD_LAUNCH_GRAPH if index % 2 else P.DDD_LAUNCH_STREAM
+    eng = engine_for(cfg, TC, mode)
+    with torch.cuda.stream(torch.cuda.Stream()):
+        for i in range(2):
+            roots = S.make_roots(cfg, i)
+            g = parity.run_gpu(eng, roots)
+            parity.compare_with_oracle(cfg, weights_for(cfg), roots, g)
+    eng.close()
+
+
 # ----------------------------------------------------------------------------- launch modes
 def test_graph_mode_host_variant_and_determinism():
     cfg = small_cases()["7b"]
