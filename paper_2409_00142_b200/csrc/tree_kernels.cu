@@ -258,9 +258,13 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
   unsigned long long* keys_s = reinterpret_cast<unsigned long long*>(smem_raw);              // [rows_max][nc][kl]
   float2* ms_s = reinterpret_cast<float2*>(keys_s + (size_t)rows_max * nc * kl);              // [rows_max][nc]
   int* plant_s = reinterpret_cast<int*>(ms_s + (size_t)rows_max * nc);                        // [rows_max]
-  __shared__ unsigned long long cand_key[DDD_MAX_K * DDD_MAX_K];   // used in block 0
-  __shared__ float cand_val[DDD_MAX_K * DDD_MAX_K];                // used in block 0
-  __shared__ int cand_tok[DDD_MAX_K * DDD_MAX_K];                  // used in block 0
+  // candidate (p, c) of this pass at [p * k + c]: score bits in the upper word, token (-1 = none)
+  // in the lower; one 8-byte store per block of the cluster carries it there
+  __shared__ unsigned long long cand_rec[DDD_MAX_K * DDD_MAX_K];
+  auto cand_key_of = [&](int idx) -> unsigned long long {     // selection key: score, ties to the lower index
+    const unsigned long long rec = cand_rec[idx];
+    return (int)(uint32_t)rec >= 0 ? make_key(__uint_as_float((uint32_t)(rec >> 32)), (uint32_t)idx) : 0ull;
+  };
   __shared__ int sel_flat[DDD_MAX_K];
   __shared__ int sel_tok[DDD_MAX_K];
   __shared__ double row_part[DDD_MAX_K * 64];
@@ -379,12 +383,8 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
       p.tree_parent[node] = beam_node_s[warp];
       p.tree_cum[node] = cand;
       // every block of the cluster gets the candidates of all rows
-      const unsigned long long ckey = (res != 0ull) ? make_key(cand, (uint32_t)flat) : 0ull;
-      for (int rk = 0; rk < kSelCluster; ++rk) {
-        cluster.map_shared_rank(cand_key, rk)[flat] = ckey;
-        cluster.map_shared_rank(cand_val, rk)[flat] = cand;
-        cluster.map_shared_rank(cand_tok, rk)[flat] = tok;
-      }
+      const unsigned long long rec = ((unsigned long long)__float_as_uint(cand) << 32) | (uint32_t)tok;
+      for (int rk = 0; rk < kSelCluster; ++rk) cluster.map_shared_rank(cand_rec, rk)[flat] = rec;
     }
     if (lane == 0 && io.trace.row_lse) io.trace.row_lse[((size_t)b * p.n + (d - 1)) * k + pr] = lse;
   }
@@ -398,7 +398,7 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
     if (n_cand <= 128) {
       unsigned long long ck[4];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) ck[i] = lane + 32 * i < n_cand ? cand_key[lane + 32 * i] : 0ull;
+      for (int i = 0; i < 4; ++i) ck[i] = lane + 32 * i < n_cand ? cand_key_of(lane + 32 * i) : 0ull;
       for (int j = 0; j < k; ++j) {
         unsigned long long best = ck[0];
 #pragma unroll
@@ -411,27 +411,30 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
           if (ck[i] == wk) ck[i] = 0ull;
       }
     } else {
-      unsigned long long prev = ~0ull;
+      // more candidates than fit four per lane: the k candidates of a beam row are already in
+      // descending key order (same parent score, log-probabilities descending, ties by lower
+      // index), so lane p walks row p and the beam is a k-way merge of the P <= 32 rows
+      int pos = 0;
+      unsigned long long head = lane < P ? cand_key_of(lane * k) : 0ull;
       for (int j = 0; j < k; ++j) {
-        unsigned long long best = 0ull;
-        for (int c = lane; c < n_cand; c += 32) {
-          const unsigned long long key = cand_key[c];
-          if (key < prev && key > best) best = key;
-        }
-        const unsigned long long wk = warp_max_key(best);
+        const unsigned long long wk = warp_max_key(head);
         if (lane == j) mine = wk;
-        prev = wk;
+        if (wk == 0ull) break;
+        if (head == wk) {                   // keys are unique: exactly one lane
+          ++pos;
+          head = pos < k ? cand_key_of(lane * k + pos) : 0ull;
+        }
       }
     }
     const bool have = lane < k && mine != 0ull;
     const int flat = have ? (int)key_index(mine) : 0;
-    const float cum = have ? cand_val[flat] : neg_inf();
+    const float cum = have ? __uint_as_float((uint32_t)(cand_rec[flat] >> 32)) : neg_inf();
     const float M = __shfl_sync(kFullMask, cum, 0);           // sorted descending: entry 0 is the max
     const float sum = warp_sum(have ? expf(cum - M) : 0.f);
     const float H = M + logf(sum);
     bool stop = (d == p.n);
     if (!stop && ((p.check_mask >> (d - 1)) & 1u)) stop = H < p.x;
-    const int tok = lane < k ? cand_tok[flat] : -1;
+    const int tok = lane < k ? (int)(uint32_t)cand_rec[flat] : -1;
     if (lane < k) {
       sel_flat[lane] = flat;
       sel_tok[lane] = tok;
