@@ -225,6 +225,12 @@ __device__ void draft_step(const Params& p, int b, int d, const int* sel_flat, c
     draft_step_warp<T>(p, b, d, sel_flat, sel_tok);
 }
 
+// 8-byte asynchronous copy global -> shared (both 8-byte aligned); completes at cp.async.wait_group.
+__device__ __forceinline__ void async_copy_8(void* dst_shared, const void* src_global) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 8;"
+               ::"r"((uint32_t)__cvta_generic_to_shared(dst_shared)), "l"(src_global) : "memory");
+}
+
 // One cluster of kSelCluster blocks per sequence.  Beam row pr is merged by block pr % 8
 // (warp pr / 8), which first copies that row's partial lists into its shared memory; the
 // candidates go to block 0 through distributed shared memory, block 0 picks the new beam and
@@ -274,50 +280,30 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
   __shared__ float beam_cum_s[DDD_MAX_K / kSelCluster];
   __shared__ int beam_node_s[DDD_MAX_K / kSelCluster];
 
-  // ---- phase 0: the block fetches everything phase 1 needs for its rows in one round trip
-  // (a warp copies one LM-head block's list per step: lane q takes the q-th key)
-  // All loads of all rows are issued before the first value is used: a round trip to memory
-  // costs this lone block a microsecond or two, so they must not queue up behind each other.
+  // ---- phase 0: the block fetches everything phase 1 needs for its rows in one round trip.
+  // The copies go from global to shared memory asynchronously (a warp copies one LM-head block's
+  // list per step: lane q takes the q-th key), so all of them are in flight together however
+  // many rows the block owns: a round trip to memory costs this lone block a microsecond or
+  // two, and loads through registers would have to go in several batches.
   {
-    constexpr int kW = kSelThreads / 32, kPre = 5, kRows = 2;   // two rows x five lists per warp and batch
-    for (int j0 = 0; j0 < n_mine; j0 += kRows)
-    for (int c0 = warp; c0 < nc; c0 += kW * kPre) {
-      unsigned long long key[kRows][kPre];
-      float2 ms[kRows][kPre];
-#pragma unroll
-      for (int j = 0; j < kRows; ++j) {
-        if (j0 + j >= n_mine) continue;
-        const int r = b * k + crank + kSelCluster * (j0 + j);
-#pragma unroll
-        for (int i = 0; i < kPre; ++i) {
-          const int c = c0 + kW * i;
-          if (c < nc) {
-            const size_t slot = (size_t)c * R + r;
-            if (lane < kl) key[j][i] = p.part_key[slot * k + lane];
-            if (lane == 31) ms[j][i] = p.part_ms[slot];
-          }
-        }
-      }
-      // the few scalars phase 1 needs ride along with the first batch
-      if (j0 == 0 && c0 == warp && warp == 0 && lane < n_mine) {
-        const int r = b * k + crank + kSelCluster * lane;
-        plant_s[lane] = p.row_plant[r];
-        beam_cum_s[lane] = p.beam_cum[r];
-        beam_node_s[lane] = p.beam_node[r];
-      }
-#pragma unroll
-      for (int j = 0; j < kRows; ++j) {
-        if (j0 + j >= n_mine) continue;
-#pragma unroll
-        for (int i = 0; i < kPre; ++i) {
-          const int c = c0 + kW * i;
-          if (c < nc) {
-            if (lane < kl) keys_s[((size_t)(j0 + j) * nc + c) * kl + lane] = key[j][i];
-            if (lane == 31) ms_s[(size_t)(j0 + j) * nc + c] = ms[j][i];
-          }
-        }
+    constexpr int kW = kSelThreads / 32;
+    for (int j = 0; j < n_mine; ++j) {
+      const int r = b * k + crank + kSelCluster * j;
+      for (int c = warp; c < nc; c += kW) {
+        const size_t slot = (size_t)c * R + r;
+        if (lane < kl) async_copy_8(&keys_s[((size_t)j * nc + c) * kl + lane], &p.part_key[slot * k + lane]);
+        if (lane == 31) async_copy_8(&ms_s[(size_t)j * nc + c], &p.part_ms[slot]);
       }
     }
+    // the few scalars phase 1 needs ride along
+    if (warp == 0 && lane < n_mine) {
+      const int r = b * k + crank + kSelCluster * lane;
+      plant_s[lane] = p.row_plant[r];
+      beam_cum_s[lane] = p.beam_cum[r];
+      beam_node_s[lane] = p.beam_node[r];
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
   }
   __syncthreads();
 
