@@ -146,34 +146,36 @@ __device__ __forceinline__ void row_tile_update(const float* zrow, int tok0, int
   const uint32_t tile_best = max(max(o[0], o[1]), max(o[2], o[3]));
   if (!__any_sync(kFullMask, tile_best > kth)) return;
 
-  uint32_t new_o = 0u, new_tok = 0u;
+  // Insert the tile's entries that beat the k-th best, best first.  An entry goes behind every
+  // list entry with a score at least as high (the older, lower token wins ties) and pushes the
+  // rest down one lane; the loop ends when the best entry left in the tile no longer beats the
+  // k-th best, after at most k insertions.
+  uint32_t kth_now = kth;
   for (int j = 0; j < k; ++j) {
-    const uint32_t best = max(carry_o, max(max(o[0], o[1]), max(o[2], o[3])));
+    const uint32_t best = max(max(o[0], o[1]), max(o[2], o[3]));
     const uint32_t top = __reduce_max_sync(kFullMask, best);
-    if (top == 0u) break;                       // pool exhausted (uniform)
-    uint32_t win_tok;
-    const unsigned in_list = __ballot_sync(kFullMask, carry_o == top);
-    if (in_list) {                              // uniform: an old entry wins ties
-      const int src = __ffs(in_list) - 1;
-      win_tok = __shfl_sync(kFullMask, carry_tok, src);
-      if (lane == src) carry_o = 0u;
-    } else {
-      const unsigned in_tile = __ballot_sync(kFullMask, best == top);
-      const int src = __ffs(in_tile) - 1;
-      int slot = 3;
-      if (o[2] == top) slot = 2;
-      if (o[1] == top) slot = 1;
-      if (o[0] == top) slot = 0;
-      win_tok = __shfl_sync(kFullMask, (uint32_t)(tok0 + 4 * lane + slot), src);
-      if (lane == src) {
+    if (top <= kth_now) break;                  // uniform; top > 0 here
+    const unsigned in_tile = __ballot_sync(kFullMask, best == top);
+    const int src = __ffs(in_tile) - 1;         // lowest lane, then lowest slot: the lowest token
+    int slot = 3;
+    if (o[2] == top) slot = 2;
+    if (o[1] == top) slot = 1;
+    if (o[0] == top) slot = 0;
+    const uint32_t win_tok = __shfl_sync(kFullMask, (uint32_t)(tok0 + 4 * lane + slot), src);
+    if (lane == src) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i)
-          if (i == slot) o[i] = 0u;
-      }
+      for (int i = 0; i < 4; ++i)
+        if (i == slot) o[i] = 0u;
     }
-    if (lane == j) { new_o = top; new_tok = win_tok; }
+    const int ins = __popc(__ballot_sync(kFullMask, lane < k && carry_o >= top));
+    const uint32_t up_o = __shfl_up_sync(kFullMask, carry_o, 1);
+    const uint32_t up_tok = __shfl_up_sync(kFullMask, carry_tok, 1);
+    if (lane == ins) { carry_o = top; carry_tok = win_tok; }
+    else if (lane > ins) { carry_o = up_o; carry_tok = up_tok; }
+    kth_now = __shfl_sync(kFullMask, carry_o, k - 1);
   }
-  list_key = new_o ? (((unsigned long long)new_o << 32) | (unsigned long long)(0xFFFFFFFFu - new_tok)) : 0ull;
+  list_key = (lane < k && carry_o) ? (((unsigned long long)carry_o << 32) | (unsigned long long)(0xFFFFFFFFu - carry_tok))
+                                   : 0ull;
 }
 
 // ---------------------------------------------------------------------------- launchers (host)
