@@ -35,7 +35,7 @@ NEG = -1e30
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes (read + write) of one LM-head launch from the ncu capture summarised under
 # profiles/, valid only while the kernel source is the one that was profiled.
-NCU_TRAFFIC = {"llama2_7b": {"bytes": 265.6e6, "source_sha256_16": "9270d077708fda9d",
+NCU_TRAFFIC = {"llama2_7b": {"bytes": 267.5e6, "source_sha256_16": "0b876d8fed98b331",
                              "profile": "profiles/lm_head_tc_llama2_7b.md"}}
 CLOCK_QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
                "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
@@ -67,13 +67,15 @@ def ncu_traffic(workload: str):
     ent = NCU_TRAFFIC.get(workload)
     if not ent:
         return None
-    src = os.path.join(ROOT, "paper_2409_00142_b200", "csrc", "lm_head_tc.cu")
+    digest = hashlib.sha256()
     try:
-        with open(src, "rb") as f:
-            if hashlib.sha256(f.read()).hexdigest()[:16] != ent["source_sha256_16"]:
-                return None          # kernel changed since the counters were taken
+        for name in ("lm_head_tc.cu", "ddd_common.cuh"):      # the kernel and the row update it inlines
+            with open(os.path.join(ROOT, "paper_2409_00142_b200", "csrc", name), "rb") as f:
+                digest.update(f.read())
     except OSError:
         return None
+    if digest.hexdigest()[:16] != ent["source_sha256_16"]:
+        return None                  # kernel changed since the counters were taken
     return ent["bytes"]
 
 
