@@ -348,6 +348,9 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
     }
   }
   __syncthreads();
+  unsigned long long node_rec = 0ull;
+  int node_flat = -1;
+  float node_lse = 0.f;
   if (warp < n_mine) {
     const int pr = crank + kSelCluster * warp;
     const float lse = lse_s[warp];
@@ -364,17 +367,25 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
       const int tok = (res != 0ull) ? (int)key_index(res) : -1;
       const float cand = beam_cum_s[warp] + lp;
       const int flat = pr * k + lane;
-      const size_t node = (size_t)b * p.Nn + base + flat;
-      p.tree_token[node] = tok;
-      p.tree_parent[node] = beam_node_s[warp];
-      p.tree_cum[node] = cand;
       // every block of the cluster gets the candidates of all rows
-      const unsigned long long rec = ((unsigned long long)__float_as_uint(cand) << 32) | (uint32_t)tok;
-      for (int rk = 0; rk < kSelCluster; ++rk) cluster.map_shared_rank(cand_rec, rk)[flat] = rec;
+      node_rec = ((unsigned long long)__float_as_uint(cand) << 32) | (uint32_t)tok;
+      for (int rk = 0; rk < kSelCluster; ++rk) cluster.map_shared_rank(cand_rec, rk)[flat] = node_rec;
+      node_flat = flat;
     }
-    if (lane == 0 && io.trace.row_lse) io.trace.row_lse[((size_t)b * p.n + (d - 1)) * k + pr] = lse;
+    node_lse = lse;
   }
   cluster.sync();       // the last time a block touches another block's shared memory before the draft step
+  // The new tree nodes go to global memory only now: the barrier above has release semantics,
+  // and with these stores ahead of it every block waited for them to reach L2 under the next
+  // pass's W burst.  (A sequence that stops meets at one more barrier before its rerank.)
+  if (node_flat >= 0) {
+    const size_t node = (size_t)b * p.Nn + base + node_flat;
+    p.tree_token[node] = (int)(uint32_t)node_rec;
+    p.tree_parent[node] = beam_node_s[warp];
+    p.tree_cum[node] = __uint_as_float((uint32_t)(node_rec >> 32));
+  }
+  if (warp < n_mine && lane == 0 && io.trace.row_lse)
+    io.trace.row_lse[((size_t)b * p.n + (d - 1)) * k + crank + kSelCluster * warp] = node_lse;
 
   // ---- phase 2: warp 0 of every block picks the new beam, evaluates Eq. 1 and takes the stop
   //      decision (same inputs, same result everywhere; block 0 records it)
@@ -451,8 +462,9 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
   // a sequence that goes on switches them on.
   if (set_cond && !s_stop && crank == 0 && threadIdx.x == 0) cudaGraphSetConditional(cond, 1);
   if (s_stop) {             // every block takes this branch alike
-    // the sequence is finished: block 0 goes straight on to the rerank and the mask (the nodes the
-    // other blocks appended in this pass are visible since the cluster barrier above)
+    // the sequence is finished: block 0 goes on to the rerank and the mask once the nodes the other
+    // blocks appended in this pass are visible to it
+    cluster.sync();
     if (crank == 0) rerank_mask_block<kSelThreads>(p, io, b, d, s_last, smem_raw);
     return;
   }
