@@ -189,7 +189,7 @@ int ddd_draft(ddd_handle *h, const void *root_hidden, const int32_t *root_token,
  * The same draft the way the paper runs it (Section 2, Section 3.4 "Strict"): after every
  * LM-head pass the HOST synchronises the stream, reads how many sequences are still drafting
  * and only then launches the next pass.  Arguments and results are those of ddd_draft (DEVICE
- * buffers); the call returns after the rerank has been enqueued, with *passes_run (HOST, may be
+ * buffers); the call returns after the last pass has been enqueued, with *passes_run (HOST, may be
  * NULL) = number of passes launched.  It exists to measure what the device-resident gate of
  * ddd_draft saves; results are identical.  Errors: INVALID_ARG, ALIGNMENT, CUDA.
  */

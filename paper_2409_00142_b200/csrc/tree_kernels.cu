@@ -1,5 +1,6 @@
-// Kernels around the LM head: draft initialisation, the per-pass select / gate / draft
-// step, and the final rerank with the bit-packed tree mask.  One thread block per sequence.
+// Kernels around the LM head: draft initialisation and the per-pass select / gate / draft step,
+// which for a sequence that stops at that pass ends with the rerank and the bit-packed tree
+// mask (tree_device.cuh).  One cluster of eight thread blocks per sequence.
 #include <cooperative_groups.h>
 
 #include "ddd_common.cuh"
