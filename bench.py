@@ -37,6 +37,8 @@ FALLBACK_HBM_GBS = 6650.0
 # profiles/, valid only while the kernel source is the one that was profiled.
 NCU_TRAFFIC = {"llama2_7b": {"bytes": 267.5e6, "source_sha256_16": "0b876d8fed98b331",
                              "profile": "profiles/lm_head_tc_llama2_7b.md"}}
+BEAM_WIDTHS = (5, 10, 20, 32)      # fixed-depth-6 sweep (the paper's appendix table goes on to 50, 75, 100)
+OTHER_WORKLOADS = ("vicuna_13b", "llama2_70b_b16", "llama3_8b_128k")
 CLOCK_QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
                "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
                "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
@@ -50,13 +52,18 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama2_7b", choices=list(S.CONFIGS))
     ap.add_argument("--threshold", type=float, default=None, help="override the workload's threshold x")
-    ap.add_argument("--drafts-per-step", type=int, default=32)
+    ap.add_argument("--drafts-per-step", type=int, default=1000,
+                    help="distinct seeded roots drafted per step and rank (the 7B workload is stated on 1000 drafts)")
     ap.add_argument("--lm-head-reps", type=int, default=200)
     ap.add_argument("--cpu-sample", type=int, default=None, help="drafts the CPU baseline times")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true")
-    ap.add_argument("--width-sweep", action="store_true",
-                    help="also time fixed-depth-6 drafts at beam widths 5, 10, 20, 32 (cf. the paper's appendix)")
+    ap.add_argument("--no-width-sweep", action="store_true",
+                    help="skip the fixed-depth-6 drafts at the beam widths of the paper's appendix table")
+    ap.add_argument("--no-other-workloads", action="store_true",
+                    help="skip the short runs of the other bf16 workloads (13B-, 70B-shaped, 128k vocabulary)")
+    ap.add_argument("--dist-backend", default="nccl", choices=["nccl", "gloo"],
+                    help="process-group backend of a multi-rank run (gloo: host-side tests of the rank logic)")
     ap.add_argument("--launch-mode", default="graph", choices=["graph", "stream", "plain"],
                     help="plain: ordinary stream-ordered launches, the mode profilers can follow")
     return ap.parse_args()
@@ -137,15 +144,33 @@ class ClockSampler:
         return out
 
 
-def dist_setup(n_gpus: int):
+def dist_setup(n_gpus: int, backend: str = "nccl"):
+    """Joins the process group torchrun describes in the environment (none for a single process)."""
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if world > 1:
         import torch.distributed as dist
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        if backend == "nccl":
+            dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        else:
+            dist.init_process_group(backend)
     return rank, world, local
+
+
+def dist_teardown(world: int):
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def emit(line: dict, rank: int) -> bool:
+    """Rank 0 prints the one JSON line of the run; the other ranks print nothing."""
+    if rank != 0:
+        return False
+    print(json.dumps(line), flush=True)
+    return True
 
 
 def barrier(world):
@@ -191,6 +216,8 @@ def timed_drafts(eng, roots_dev, steps: int, warmup: int, world: int, device):
         one_step()
     e1.record(stream)
     torch.cuda.synchronize(device)
+    # a draft that recorded an error (a bounded wait that ran out) publishes nothing and would look fast
+    assert int(eng.out["status"].item()) == 0, "device reported an error status during the timed drafts"
     barrier(world)
     ms = e0.elapsed_time(e1) / steps
     return max_over_ranks(ms, world, device), ms
@@ -247,7 +274,45 @@ def run_reference(args):
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
-    print(json.dumps(line))
+    emit(line, rank)
+
+
+def stack_roots(cfg, indices):
+    """The seeded roots of the given draft indices as three host tensors [n][B][Hd], [n][B], [n][B]."""
+    roots = [S.make_roots(cfg, i) for i in indices]
+    return {k: torch.stack([r[k] for r in roots]).contiguous() for k in ("root_hidden", "root_token", "root_pos")}
+
+
+def rows_of(stacked):
+    """Per-draft views (no copies) of stacked roots."""
+    n = stacked["root_token"].shape[0]
+    return [{k: v[i] for k, v in stacked.items()} for i in range(n)]
+
+
+def time_lm_head(eng, reps: int, stream, device, flush):
+    """The LM-head kernel alone, two ways.  Back to back: `reps` launches in a row, the period between
+    them (each launch's set-up and first loads overlap the tail of the one before, as they overlap the
+    select kernel inside a draft).  Isolated: one launch at a time behind a write of a buffer larger
+    than L2, timed by its own pair of events (nothing to overlap with, cold L2)."""
+    for _ in range(5):
+        eng.lm_head_pass()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(reps):
+        eng.lm_head_pass()
+    e1.record(stream)
+    torch.cuda.synchronize(device)
+    period_us = 1e3 * e0.elapsed_time(e1) / reps
+    n_iso = max(5, min(40, reps // 5))
+    pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_iso)]
+    for a, b in pairs:
+        flush.zero_()                  # evicts W from L2 and keeps the queue busy until the launch is enqueued
+        a.record(stream)
+        eng.lm_head_pass()
+        b.record(stream)
+    torch.cuda.synchronize(device)
+    iso_us = statistics.median(1e3 * a.elapsed_time(b) for a, b in pairs)
+    return period_us, iso_us
 
 
 def main():
@@ -257,7 +322,7 @@ def main():
         return
     import paper_2409_00142_b200 as P
 
-    rank, world, local = dist_setup(args.gpus)
+    rank, world, local = dist_setup(args.gpus, args.dist_backend)
     device = torch.device("cuda", local)
     torch.cuda.set_device(device)
     cfg = S.CONFIGS[args.workload]
@@ -266,13 +331,19 @@ def main():
     weights = S.make_weights(cfg)
     n_per_rank = args.drafts_per_step
     my_indices = S.shard_draft_indices(n_per_rank * world, rank, world)
-    roots_host = [S.make_roots(cfg, i) for i in my_indices]
+    roots_host = stack_roots(cfg, my_indices)
     stream = torch.cuda.Stream(device)
+    mode = {"graph": P.DDD_LAUNCH_GRAPH, "stream": P.DDD_LAUNCH_STREAM, "plain": P.DDD_LAUNCH_PLAIN}[args.launch_mode]
+    peak, peak_kind = measured_peak()
+    elt = 4 if cfg.dtype == "fp32" else 2
+    w_bytes = cfg.vocab * cfg.hidden * elt
+    sub_steps = max(3, args.steps // 4)
 
     with torch.cuda.stream(stream):
-        mode = {"graph": P.DDD_LAUNCH_GRAPH, "stream": P.DDD_LAUNCH_STREAM, "plain": P.DDD_LAUNCH_PLAIN}[args.launch_mode]
         eng = P.DraftEngine(cfg, weights, device=local, launch_mode=mode, with_trace=False)
-        roots_dev = [{k: v.to(device) for k, v in r.items()} for r in roots_host]
+        dev_weights = {"W": eng.W, "E": eng.E, "bias": eng.bias, "plant_next": eng.plant_next}
+        roots_dev = rows_of({k: v.to(device) for k, v in roots_host.items()})
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)      # larger than the 126 MB L2
         torch.cuda.synchronize(device)
         depth_lists = mean_stop_depth(eng, roots_dev, device)
         depth_mean = _mean(depth_lists)
@@ -284,95 +355,93 @@ def main():
         clocks = sampler.stop()
         drafts_total = n_per_rank * world * cfg.batch
         value = drafts_total / (ms_step / 1e3)
+        us_per_draft = 1e3 * ms_step / n_per_rank
+        passes_mean = _mean([[d] for d in stop_depths])
 
         # ---- the LM-head kernel alone: CUDA events on the launching stream, W (> L2) streamed each launch
-        for _ in range(5):
-            eng.lm_head_pass()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for _ in range(args.lm_head_reps):
-            eng.lm_head_pass()
-        e1.record(stream)
-        torch.cuda.synchronize(device)
-        lm_us = 1e3 * e0.elapsed_time(e1) / args.lm_head_reps
-        elt = 4 if cfg.dtype == "fp32" else 2
-        w_bytes = cfg.vocab * cfg.hidden * elt
+        lm_us, lm_iso_us = time_lm_head(eng, args.lm_head_reps, stream, device, flush)
         achieved = w_bytes / (lm_us * 1e-6) / 1e9
-        peak, peak_kind = measured_peak()
+
+        def variant(c, launch=P.DDD_LAUNCH_GRAPH, w=None):
+            return P.DraftEngine(c, w or dev_weights, device=local, launch_mode=launch, with_trace=False)
 
         # ---- fixed full depth (x = -inf): per-expansion-step time independent of where drafts stop
         extra = {}
+        step_us = None
         if not args.no_sweep:
-            full_cfg = cfg.replace(threshold=NEG)
-            eng_full = P.DraftEngine(full_cfg, {"W": eng.W, "E": eng.E, "bias": eng.bias,
-                                                "plant_next": eng.plant_next}, device=local,
-                                     launch_mode=P.DDD_LAUNCH_GRAPH, with_trace=False)
-            ms_full, _ = timed_drafts(eng_full, roots_dev, max(3, args.steps // 4), args.warmup, world, device)
-            per_draft_us = 1e3 * ms_full / n_per_rank
-            extra["full_depth"] = {"drafts_per_sec": drafts_total / (ms_full / 1e3),
-                                   "us_per_draft": per_draft_us,
-                                   "us_per_expansion_step": per_draft_us / cfg.max_depth,
-                                   "passes": cfg.max_depth}
+            full_roots = roots_dev[:max(1, min(len(roots_dev), 64))]
+            eng_full = variant(cfg.replace(threshold=NEG))
+            ms_full, _ = timed_drafts(eng_full, full_roots, sub_steps, args.warmup, world, device)
+            per_draft_us = 1e3 * ms_full / len(full_roots)
+            step_us = per_draft_us / cfg.max_depth
+            extra["full_depth"] = {"drafts_per_sec": len(full_roots) * world * cfg.batch / (ms_full / 1e3),
+                                   "us_per_draft": per_draft_us, "us_per_expansion_step": step_us,
+                                   "passes": cfg.max_depth, "drafts_per_step": len(full_roots) * world}
             eng_full.close()
             if cfg.name == "llama2_7b" and args.threshold is None:
                 sweep = {}
                 for x in S.LLAMA2_7B_THRESHOLDS:
-                    cx = cfg.replace(threshold=x)
-                    ex = P.DraftEngine(cx, {"W": eng.W, "E": eng.E, "bias": eng.bias,
-                                            "plant_next": eng.plant_next}, device=local,
-                                       launch_mode=P.DDD_LAUNCH_GRAPH, with_trace=False)
+                    ex = variant(cfg.replace(threshold=x))
                     dm = _mean(mean_stop_depth(ex, roots_dev, device))
-                    msx, _ = timed_drafts(ex, roots_dev, max(3, args.steps // 4), args.warmup, world, device)
-                    sweep[str(x)] = {"drafts_per_sec": drafts_total / (msx / 1e3), "mean_stop_depth": dm}
+                    msx, _ = timed_drafts(ex, roots_dev, sub_steps, args.warmup, world, device)
+                    sweep[str(x)] = {"drafts_per_sec": drafts_total / (msx / 1e3), "mean_stop_depth": dm,
+                                     "drafts": n_per_rank * world}
                     ex.close()
                 extra["threshold_sweep"] = sweep
 
         # ---- where the gate lives: the paper checks the heuristic on the host after a synchronisation
         # (Section 2; its "Strict" variants of Section 3.4 do so after every draft call); here the check
         # is on the device.  Same drafts, same results, host-gated: launch pass, synchronise, read, decide.
-        if not args.no_sweep:
+        if not args.no_sweep and world == 1:
+            gate_roots = roots_dev[:min(len(roots_dev), 128)]
+
             def host_gated_rate(engine, reps):
-                for r in roots_dev[:4]:
+                for r in gate_roots[:4]:
                     engine.draft_host_gated(r["root_hidden"], r["root_token"], r["root_pos"])
                 torch.cuda.synchronize(device)
                 t0 = time.perf_counter()
                 for _ in range(reps):
-                    for r in roots_dev:
+                    for r in gate_roots:
                         engine.draft_host_gated(r["root_hidden"], r["root_token"], r["root_pos"])
                 torch.cuda.synchronize(device)
-                return reps * n_per_rank * cfg.batch / (time.perf_counter() - t0)
+                return reps * len(gate_roots) * cfg.batch / (time.perf_counter() - t0)
 
-            reps = max(2, args.steps // 20)
-            extra["gate_placement"] = {"device_gate_drafts_per_sec": value,
+            def device_gated_rate(engine):
+                ms, _ = timed_drafts(engine, gate_roots, sub_steps, args.warmup, world, device)
+                return len(gate_roots) * cfg.batch / (ms / 1e3)
+
+            reps = max(2, args.steps // 10)
+            extra["gate_placement"] = {"device_gate_drafts_per_sec": device_gated_rate(eng),
                                        "host_gate_drafts_per_sec": host_gated_rate(eng, reps),
-                                       "note": "per rank; host gate = stream sync + 4-byte read after every pass"}
-            # the paper's own parameters (Section 3.2): n = 11, S = {5, 7, 9}, x = -0.3, w = 10
+                                       "note": "host gate = stream sync + 4-byte read after every pass"}
+            # the paper's own parameters (Section 3.2): n = 11, S = {5, 7, 9}, x = -0.3, w = 10, beside
+            # EAGLE-2's fixed depth 6 at the same width
             pmask = sum(1 << (s_ - 1) for s_ in (5, 7, 9))
-            pcfg = cfg.replace(max_depth=11, check_mask=pmask, threshold=-0.3, k=10)
-            pe = P.DraftEngine(pcfg, {"W": eng.W, "E": eng.E, "bias": eng.bias, "plant_next": eng.plant_next},
-                               device=local, launch_mode=mode, with_trace=False)
-            pdm = _mean(mean_stop_depth(pe, roots_dev, device))
-            pms, _ = timed_drafts(pe, roots_dev, max(3, args.steps // 4), args.warmup, world, device)
+            pe = variant(cfg.replace(max_depth=11, check_mask=pmask, threshold=-0.3, k=10), mode)
+            pdm = _mean(mean_stop_depth(pe, gate_roots, device))
+            fixed6 = variant(cfg.replace(max_depth=6, threshold=NEG, k=10), mode)
             extra["paper_parameters"] = {"n": 11, "S": [5, 7, 9], "x": -0.3, "w": 10, "mean_stop_depth": pdm,
-                                         "device_gate_drafts_per_sec": drafts_total / (pms / 1e3),
-                                         "host_gate_drafts_per_sec": host_gated_rate(pe, reps)}
+                                         "device_gate_drafts_per_sec": device_gated_rate(pe),
+                                         "host_gate_drafts_per_sec": host_gated_rate(pe, reps),
+                                         "eagle2_fixed_depth6_drafts_per_sec": device_gated_rate(fixed6)}
             pe.close()
+            fixed6.close()
 
         # ---- beam width vs run time at fixed depth 6 (the paper's appendix reports an almost flat curve)
-        if args.width_sweep:
+        if not args.no_width_sweep and not args.no_sweep and world == 1:
             sweep_w = {}
-            for kw in (5, 10, 20, 32):
-                wc = cfg.replace(k=kw, max_depth=6, threshold=NEG, total_tokens=60)
-                we = P.DraftEngine(wc, {"W": eng.W, "E": eng.E, "bias": eng.bias, "plant_next": eng.plant_next},
-                                   device=local, launch_mode=mode, with_trace=False)
-                wms, _ = timed_drafts(we, roots_dev, max(3, args.steps // 8), args.warmup, world, device)
-                sweep_w[str(kw)] = {"us_per_draft": 1e3 * wms / n_per_rank, "us_per_expansion_step": 1e3 * wms / n_per_rank / 6}
+            wide_roots = roots_dev[:min(len(roots_dev), 32)]
+            for kw in BEAM_WIDTHS:
+                we = variant(cfg.replace(k=kw, max_depth=6, threshold=NEG, total_tokens=60), mode)
+                wms, _ = timed_drafts(we, wide_roots, sub_steps, args.warmup, world, device)
+                sweep_w[str(kw)] = {"us_per_draft": 1e3 * wms / len(wide_roots),
+                                    "us_per_expansion_step": 1e3 * wms / len(wide_roots) / 6}
                 we.close()
             extra["beam_width_sweep_depth6"] = sweep_w
 
         # ---- end to end through the host-buffer entry point (pinned host memory, copies inside)
         host_out = eng.make_host_out(pinned=True)
-        pinned = [{k: v.pin_memory() for k, v in r.items()} for r in roots_host]
+        pinned = rows_of({k: v.pin_memory() for k, v in roots_host.items()})
         for r in pinned[:4]:
             eng.draft_host(r["root_hidden"], r["root_token"], r["root_pos"], host_out)
         torch.cuda.synchronize(device)
@@ -381,7 +450,7 @@ def main():
         e2e_steps = max(2, args.steps // 4)
         for _ in range(e2e_steps):
             for r in pinned:
-                eng.draft_host(r["root_hidden"], r["root_token"], r["root_pos"], host_out)
+                eng.draft_host(r["root_hidden"], r["root_token"], r["root_pos"], host_out)    # raises on a bad status
         torch.cuda.synchronize(device)
         e2e_ms = 1e3 * (time.perf_counter() - t0) / e2e_steps
         e2e_ms = max_over_ranks(e2e_ms, world, device)
@@ -391,12 +460,56 @@ def main():
         blocks = P.ddd_lm_head_blocks(eng.handle)
         eng.close()
 
+        # ---- the other bf16 workloads, briefly: LM-head bandwidth, drafts/s at the workload's own
+        # threshold, time per expansion step at full depth
+        if not args.no_other_workloads and not args.no_sweep and world == 1 and args.workload == "llama2_7b":
+            del eng, dev_weights, roots_dev
+            others = {}
+            for name in OTHER_WORKLOADS:
+                oc = S.CONFIGS[name]
+                ow = S.make_weights(oc)
+                oe = variant(oc, mode, ow)
+                odw = {"W": oe.W, "E": oe.E, "bias": oe.bias, "plant_next": oe.plant_next}
+                n_o = max(4, 64 // oc.batch)
+                oroots = rows_of({k: v.to(device) for k, v in stack_roots(oc, range(n_o)).items()})
+                odepth = _mean(mean_stop_depth(oe, oroots, device))
+                oms, _ = timed_drafts(oe, oroots, sub_steps, args.warmup, world, device)
+                o_period, o_iso = time_lm_head(oe, max(20, args.lm_head_reps // 4), stream, device, flush)
+                of = variant(oc.replace(threshold=NEG), mode, odw)
+                ofms, _ = timed_drafts(of, oroots[:8], 3, args.warmup, world, device)
+                o_bytes = oc.vocab * oc.hidden * 2
+                o_step = 1e3 * ofms / len(oroots[:8]) / oc.max_depth
+                others[name] = {
+                    "threshold": oc.threshold, "beam_rows": oc.batch * oc.k, "mean_stop_depth": odepth,
+                    "drafts_per_sec": n_o * oc.batch / (oms / 1e3),
+                    "lm_head_us_back_to_back": o_period, "lm_head_us_isolated": o_iso,
+                    "lm_head_gbs": o_bytes / (o_period * 1e-6) / 1e9, "lm_head_frac": o_bytes / (o_period * 1e-6) / 1e9 / peak,
+                    "us_per_expansion_step_full_depth": o_step,
+                    "step_frac": o_bytes / (o_step * 1e-6) / 1e9 / peak}
+                of.close()
+                oe.close()
+                del oe, of, ow, odw, oroots
+                torch.cuda.empty_cache()
+            extra["other_workloads"] = others
+
     if rank != 0:
-        if world > 1:
-            import torch.distributed as dist
-            dist.destroy_process_group()
+        dist_teardown(world)
         return
 
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "traffic": ncu_traffic(cfg.name), "peak_kind": f"of {peak_kind}",
+                "kernel": "lm_head", "us_per_launch": lm_us,
+                "us_per_launch_kind": "period of back-to-back launches (set-up and first loads overlap the predecessor)",
+                "us_per_launch_isolated": lm_iso_us, "frac_isolated": w_bytes / (lm_iso_us * 1e-6) / 1e9 / peak,
+                "algorithmic_bytes_per_launch": w_bytes,
+                "frac_of_8TBs_nominal": achieved / 8000.0, "blocks": blocks,
+                # the whole draft against the same peak: W bytes of the passes a draft needs / time per draft
+                "draft_frac": passes_mean * w_bytes / (us_per_draft * 1e-6) / 1e9 / peak}
+    if step_us is not None:
+        # the expansion step (LM head + select / gate / draft step) at full depth: the figure the
+        # 70-%-of-HBM-bandwidth target is stated on
+        roofline["step_frac"] = w_bytes / (step_us * 1e-6) / 1e9 / peak
+        roofline["step_frac_of_8TBs_nominal"] = w_bytes / (step_us * 1e-6) / 1e9 / 8000.0
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
@@ -411,18 +524,18 @@ def main():
         "e2e": {"value": n_per_rank * world * cfg.batch / (e2e_ms / 1e3), "unit": UNIT,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": launches,
-        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak, "traffic": ncu_traffic(cfg.name), "peak_kind": f"of {peak_kind}",
-                     "kernel": "lm_head", "us_per_launch": lm_us, "algorithmic_bytes_per_launch": w_bytes,
-                     "frac_of_8TBs_nominal": achieved / 8000.0, "blocks": blocks},
+        "gpu_launches_kind": "computed: ddd_launches_per_draft(stop depth) summed over the timed drafts",
+        "us_per_draft": us_per_draft,
+        "roofline": roofline,
     }
     line.update(extra)
     if not args.no_cpu_baseline and world == 1:
         from oracle import ddd_oracle as O
         # a bounded sample of the same workload: drafts until about 12 s of CPU work (or --cpu-sample drafts)
+        cpu_roots = rows_of(roots_host)
         sample, t0 = 0, time.perf_counter()
         while True:
-            O.draft(cfg, weights, **roots_host[sample % len(roots_host)])
+            O.draft(cfg, weights, **cpu_roots[sample % len(cpu_roots)])
             sample += 1
             dt = time.perf_counter() - t0
             if (args.cpu_sample and sample >= args.cpu_sample) or (not args.cpu_sample and (dt > 12.0 or sample >= 400)):
@@ -430,10 +543,8 @@ def main():
         line["cpu_baseline"] = {"value": sample * cfg.batch / dt, "unit": UNIT, "cores": O.num_threads(),
                                 "kind": "oracle",
                                 "sample": f"{sample} draft(s) of {cfg.name}, x={cfg.threshold}, {dt:.1f} s"}
-    print(json.dumps(line))
-    if world > 1:
-        import torch.distributed as dist
-        dist.destroy_process_group()
+    emit(line, rank)
+    dist_teardown(world)
 
 
 if __name__ == "__main__":

@@ -31,6 +31,9 @@
  *     has been synchronised.  Problems found on the device (a bounded wait that ran out)
  *     are reported through ddd_output.status, never as a fault.
  *   - One draft in flight per handle; a handle is not thread-safe.
+ *   - The library reads one environment variable, DDD_DEBUG: if it is set (to anything), a
+ *     failed CUDA call is described on stderr before DDD_ERR_CUDA is returned.  Nothing else
+ *     about its behaviour depends on the environment.
  */
 #ifndef DDD_H_
 #define DDD_H_

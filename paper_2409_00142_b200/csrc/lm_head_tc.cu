@@ -38,7 +38,7 @@ constexpr int kABytes = kBlockM * kBlockK * 2;        // 16384
 constexpr int kChunkCols = 16;          // accumulator columns (beam rows) per epilogue chunk
 constexpr int kSmemLimit = 232448;      // 227 KB opt-in limit per block
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
-constexpr int kL2PrefetchBytes = 128 * 1024;   // per block, ahead of the dependency wait (about 64 MB in all)
+constexpr int kL2PrefetchBytes = 128 * 1024;   // per block, ahead of the dependency wait (at most 148 blocks: about 19 MB in all)
 
 // Accumulator chunks (of kChunkCols beam rows) the epilogue can take out of tensor memory at a
 // time: one per group of four epilogue warps, each of which reads one lane quarter.

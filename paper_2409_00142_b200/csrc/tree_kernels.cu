@@ -259,6 +259,11 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
   const int crank = (int)cluster.block_rank();
   const int b = blockIdx.x / kSelCluster;
   if (p.active[b] == 0) return;                               // same decision in the whole cluster
+  // First half of a split cluster barrier: a block may only write into another block's shared
+  // memory once that block is known to have started.  Everyone arrives here, at once; the wait
+  // sits just before the first remote store (phase 1), by which time all arrivals are long in,
+  // so it costs next to nothing.
+  asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int k = p.k, nc = p.lm_ctas, R = p.R;
   const int P = (d == 1) ? 1 : k;                            // beam rows of this sequence in pass d
@@ -355,6 +360,7 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
     }
   }
   __syncthreads();
+  asm volatile("barrier.cluster.wait.aligned;" ::: "memory");   // every block of the cluster is running
   unsigned long long node_rec = 0ull;
   int node_flat = -1;
   float node_lse = 0.f;

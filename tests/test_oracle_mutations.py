@@ -1,5 +1,6 @@
 """The pins must notice plausible mistakes: each case below plants one mistake in the CPU
 oracle (never in the CUDA path) and expects a named pin from test_oracle_pins.py to fail."""
+import inspect
 import math
 
 import numpy as np
@@ -140,3 +141,61 @@ def test_gate_strictness_mistake_is_caught(monkeypatch):
     with pytest.raises(AssertionError):
         pins.test_stop_depth_against_hand_thresholds()
     assert O.draft.__code__ is src
+
+
+# ----------------------------------------------------------------------------- the replay checker
+# The checks that police another implementation's decisions live inside O.draft itself, so the
+# mistake is planted in its source text: one edit, recompiled in the oracle's own namespace.
+def _draft_with(monkeypatch, old: str, new: str):
+    src = inspect.getsource(O.draft)
+    assert src.count(old) == 1, f"the oracle's replay code no longer reads {old!r}"
+    scope = dict(vars(O))
+    exec(compile(src.replace(old, new), "<mutated oracle draft>", "exec"), scope)
+    monkeypatch.setattr(O, "draft", scope["draft"])
+
+
+REPLAY_MUTANTS = [
+    # the gate check never fires: any stop depth is adopted
+    ("if theirs != stop and abs(H - cfg.threshold) >= tol:", "if False:",
+     pins.test_replay_rejects_a_stop_decision_outside_the_tolerance_band),
+    # the band is ignored: a decision inside it is rejected too
+    ("if theirs != stop and abs(H - cfg.threshold) >= tol:", "if theirs != stop:",
+     pins.test_replay_rejects_a_stop_decision_outside_the_tolerance_band),
+    # a stop at an unchecked step goes unnoticed
+    ("elif follow is not None and follow[b].stop_depth == d:", "elif False:",
+     pins.test_replay_rejects_a_stop_at_an_unchecked_step),
+    # the rerank set is adopted without its admissibility check
+    ("for msg in admissible_topk(cum, ids - 1, min(m, N), tol, ordered=False):", "for msg in []:",
+     pins.test_replay_rejects_an_inadmissible_rerank_set),
+    # ... or without the order check
+    ("if (np.diff(ids) <= 0).any():", "if False:", pins.test_replay_rejects_an_inadmissible_rerank_set),
+    # ... or without the ancestor check
+    ("if (r.parent == -2).any():", "if False:",
+     pins.test_replay_accepts_a_swap_inside_the_band_and_wants_an_ancestor_closed_set),
+    # the beam choice is adopted unchecked
+    ("for msg in admissible_topk(cand, sel, k, tol):", "for msg in []:",
+     pins.test_replay_of_own_decisions_is_clean_and_detects_mistakes),
+    # the rows' token lists are adopted unchecked
+    ("for msg in admissible_topk(lp, top, k, tol):", "for msg in []:",
+     pins.test_replay_of_own_decisions_is_clean_and_detects_mistakes),
+]
+
+
+@pytest.mark.parametrize("old,new,pin", REPLAY_MUTANTS,
+                         ids=[f"{i}:{m[2].__name__}" for i, m in enumerate(REPLAY_MUTANTS)])
+def test_replay_checker_pins_catch_planted_mistakes(monkeypatch, old, new, pin):
+    pin()
+    _draft_with(monkeypatch, old, new)
+    with pytest.raises(AssertionError):
+        pin()
+
+
+def test_admissible_topk_mistakes_are_caught(monkeypatch):
+    real = O.admissible_topk
+    pins.test_admissible_topk_bands()
+    for broken in (lambda *a, **kw: [],                                             # accepts anything
+                   lambda s, c, k, tol, ordered=True: real(s, c, k, 0.0, ordered),   # no band at all
+                   lambda s, c, k, tol, ordered=True: real(s, c, k, tol, False)):    # order never checked
+        monkeypatch.setattr(O, "admissible_topk", broken)
+        with pytest.raises(AssertionError):
+            pins.test_admissible_topk_bands()

@@ -198,18 +198,17 @@ def test_tree_scores_equal_brute_force_path_table(V, k, depth, dtype):
         beam_paths = got
 
 
-def test_exhaustive_beam_equals_global_topk():
-    # (iii) with k >= V^(d-1) nothing is pruned before depth d, so the beam after
-    # pass d is the exact top-k of all V^d paths.
-    V, depth = 3, 3
-    k = V ** (depth - 1)
-    cfg = small_cfg(vocab=V, k=k, hidden=8, max_depth=depth, total_tokens=5, seed=5, logit_scale=2.0)
-    # per-beam top-k needs k <= V; with k > V the per-row list would be short, so
-    # emulate "keep everything" by running depth d with k=V beams only where valid:
-    cfg = cfg.replace(k=V, max_depth=2)
+@pytest.mark.parametrize("V,seed", [(3, 5), (4, 6), (6, 7)])
+def test_exhaustive_beam_equals_global_topk(V, seed):
+    # (iii) Beam search is a heuristic, but when nothing has been pruned before depth d the beam
+    # after pass d is the exact top-k of all V^d paths.  That needs k >= V^(d-1), and a row keeps
+    # k <= V tokens, so depth 2 with k = V is the one instance there is: the first beam holds every
+    # token, and the second is the best k of all V^2 two-token paths.
+    cfg = small_cfg(vocab=V, k=V, hidden=8, max_depth=2, total_tokens=5, seed=seed, logit_scale=2.0)
     w = S.make_weights(cfg)
     r = S.make_roots(cfg, 0)
     res = O.draft(cfg, w, **r)[0]
+    assert sorted(res.tree_token[1:V + 1].tolist()) == list(range(V))
     table = brute_force_paths(cfg, w, r["root_hidden"], 2)
     want = sorted((p for p in table if len(p) == 2), key=lambda p: -table[p])[:V]
     base = O.first_node_of_pass(2, V)
@@ -402,12 +401,27 @@ def _follow_from(res):
                             beam_sel=[list(s) for s in res.beam_sel], node_id=res.node_id.copy())
 
 
-def test_replay_of_own_decisions_is_clean_and_detects_mistakes():
+REPLAY_H = (-0.17074681981286077, -0.8118013902899263, -1.4596241337374665, -2.2107429074698577)
+
+
+def _replay_case(threshold=-1.0, **kw):
+    """A draft whose heuristic falls through -0.17, -0.81, -1.46, -2.21 (REPLAY_H, checked below):
+    with x = -1 it stops after the third of at most four calls, so a stop one step early and one
+    step late both exist."""
     cfg = small_cfg(vocab=60, k=3, hidden=16, max_depth=4, total_tokens=12, logit_scale=2.0,
-                    threshold=-6.0, seed=13)
-    w = S.make_weights(cfg)
-    r = S.make_roots(cfg, 0)
+                    threshold=threshold, seed=13, **kw)
+    return cfg, S.make_weights(cfg), S.make_roots(cfg, 0)
+
+
+def _gate_violations(res):
+    return [v for v in res.violations if "gate" in v]
+
+
+def test_replay_of_own_decisions_is_clean_and_detects_mistakes():
+    cfg, w, r = _replay_case()
     res = O.draft(cfg, w, **r)[0]
+    assert res.stop_depth == 3 and not res.ambiguities
+    np.testing.assert_allclose(res.H_trace, REPLAY_H[:3], rtol=0, atol=1e-12)
     again = O.draft(cfg, w, **r, follow=[_follow_from(res)])[0]
     assert not again.violations
     np.testing.assert_array_equal(again.tree_cum, res.tree_cum)
@@ -416,15 +430,135 @@ def test_replay_of_own_decisions_is_clean_and_detects_mistakes():
     worst = int(np.argmin(O.log_softmax_row(O.lm_head_logits(
         w["W"], O.to_f64(r["root_hidden"]), cfg.logit_scale, None)[0])))
     f.tree_token[2] = worst
-    assert O.draft(cfg, w, **r, follow=[f])[0].violations
-    # a wrong stop depth is flagged
-    if res.stop_depth < cfg.max_depth:
+    assert any("token top-k" in v for v in O.draft(cfg, w, **r, follow=[f])[0].violations)
+    # a wrong member of the new beam is flagged: the worst of the k*k candidates of pass 2
+    f = _follow_from(res)
+    base = O.first_node_of_pass(2, cfg.k)
+    cand = res.tree_cum[base:base + cfg.k * cfg.k]
+    f.beam_sel[1][cfg.k - 1] = int(np.argmin(cand))
+    assert int(np.argmin(cand)) not in res.beam_sel[1]
+    assert any("beam top-k" in v for v in O.draft(cfg, w, **r, follow=[f])[0].violations)
+
+
+def test_replay_rejects_a_stop_decision_outside_the_tolerance_band():
+    """Algorithm 1 stops iff H < x at a checked step.  A replayed stop that differs from that is a
+    violation unless |H - x| < tol; the heuristic values are fixed numbers here (REPLAY_H), so
+    which side of the band each case lies on is known without asking the oracle."""
+    tol = 2e-3
+    cfg, w, r = _replay_case(-1.0)
+    full = O.draft(cfg.replace(threshold=NEG_INF), w, **r)[0]          # the search itself does not depend on x
+    np.testing.assert_allclose(full.H_trace, REPLAY_H, rtol=0, atol=1e-12)
+    own = O.draft(cfg, w, **r)[0]
+    assert own.stop_depth == 3
+
+    def follow_stopping_at(depth):
+        return O.FollowSequence(stop_depth=depth, tree_token=full.tree_token.copy(),
+                                beam_sel=[list(s) for s in full.beam_sel[:depth]], node_id=None)
+
+    # x = -1: H_2 = -0.81 >= x and H_3 = -1.46 < x, both far outside the band
+    early = O.draft(cfg, w, **r, follow=[follow_stopping_at(2)])[0]
+    assert _gate_violations(early) and "pass 2" in _gate_violations(early)[0]
+    assert early.stop_depth == 2                                     # the decision is adopted after the check
+    late = O.draft(cfg, w, **r, follow=[follow_stopping_at(4)])[0]
+    assert _gate_violations(late) and "pass 3" in _gate_violations(late)[0]
+    right = O.draft(cfg, w, **r, follow=[follow_stopping_at(3)])[0]
+    assert not right.violations and right.stop_depth == 3
+    # the same two shifts with x moved to within half the tolerance of H_3: either decision passes
+    for x, own_depth in ((REPLAY_H[2] + 0.5 * tol, 3), (REPLAY_H[2] - 0.5 * tol, 4)):
+        c2 = cfg.replace(threshold=x)
+        assert O.draft(c2, w, **r)[0].stop_depth == own_depth
+        for depth in (3, 4):
+            res = O.draft(c2, w, **r, follow=[follow_stopping_at(depth)], tol=tol)[0]
+            assert not res.violations, (x, depth, res.violations)
+            assert res.stop_depth == depth
+            assert any("gate" in a for a in res.ambiguities)
+    # ... and just outside the band the shifted decision is rejected again
+    for x, wrong in ((REPLAY_H[2] + 1.5 * tol, 4), (REPLAY_H[2] - 1.5 * tol, 3)):
+        res = O.draft(cfg.replace(threshold=x), w, **r, follow=[follow_stopping_at(wrong)], tol=tol)[0]
+        assert _gate_violations(res), (x, wrong)
+
+
+def test_replay_rejects_a_stop_at_an_unchecked_step():
+    # S = {3}: nothing may stop after step 2, whatever H is
+    cfg, w, r = _replay_case(-0.5, check_mask=1 << 2)
+    own = O.draft(cfg, w, **r)[0]
+    assert own.stop_depth == 3                                       # H_1, H_2 are below x but unchecked
+    # the search decisions of every pass stay available: having noted the violation the replay goes on
+    f = _follow_from(O.draft(cfg.replace(threshold=NEG_INF), w, **r)[0])
+    f.stop_depth, f.node_id = 2, None
+    res = O.draft(cfg, w, **r, follow=[f])[0]
+    assert any("pass 2" in v and "outside S" in v for v in res.violations)
+
+
+def test_replay_rejects_an_inadmissible_rerank_set():
+    cfg, w, r = _replay_case()
+    res = O.draft(cfg, w, **r)[0]
+    N = cfg.k + (res.stop_depth - 1) * cfg.k ** 2
+    m = cfg.total_tokens
+    cum = res.tree_cum[1:N + 1]
+    order = np.argsort(-cum, kind="stable") + 1                      # node ids, best first
+    kept, dropped = order[:m], order[m:]
+    assert cum[kept[-1] - 1] - cum[dropped[0] - 1] > 0.05            # no near-tie at the boundary
+    assert sorted(kept.tolist()) == res.node_id[1:].tolist()
+
+    def replay(ids):
         f = _follow_from(res)
-        f.stop_depth = res.stop_depth  # unchanged decisions up to here
-        g = O.draft(cfg.replace(threshold=-5.0), w, **r)[0]
-        if g.stop_depth != res.stop_depth:
-            bad = O.draft(cfg.replace(threshold=-5.0), w, **r, follow=[f])[0]
-            assert bad.violations
+        f.node_id = np.concatenate([[0], np.asarray(ids, dtype=np.int64)])
+        return [v for v in O.draft(cfg, w, **r, follow=[f])[0].violations if "rerank" in v]
+
+    assert not replay(sorted(kept.tolist()))
+    # the best node dropped for the best of the rest: something clearly above the m-th is missing
+    assert any("not chosen" in v for v in replay(sorted(kept[1:].tolist() + [int(dropped[0])])))
+    # the m-th swapped for the worst node of the tree: a member clearly below the m-th
+    assert any("below" in v for v in replay(sorted(kept[:-1].tolist() + [int(dropped[-1])])))
+    # right set, wrong order
+    ids = sorted(kept.tolist())
+    ids[3], ids[4] = ids[4], ids[3]
+    assert any("ascending" in v for v in replay(ids))
+
+
+def _one_hot_bias_case():
+    """W = 0 and one token with a logit 60 above the rest: every row's best token has logprob
+    -(V-1) e^-60 (about -1e-25, far inside any tolerance) and every other token -60, so the chain root ->
+    a -> b -> c of best tokens has three nodes whose scores agree to 1e-24."""
+    cfg = small_cfg(vocab=9, k=2, hidden=8, max_depth=3, total_tokens=2)
+    bias = torch.zeros(cfg.vocab)
+    bias[4] = 60.0
+    return cfg, uniform_weights(cfg, bias=bias), S.make_roots(cfg, 0)
+
+
+def test_replay_accepts_a_swap_inside_the_band_and_wants_an_ancestor_closed_set():
+    cfg, w, r = _one_hot_bias_case()
+    res = O.draft(cfg, w, **r)[0]
+    k = cfg.k
+    a, b, c = 1, O.first_node_of_pass(2, k), O.first_node_of_pass(3, k)
+    assert res.tree_token[[a, b, c]].tolist() == [4, 4, 4]
+    assert res.tree_parent[[a, b, c]].tolist() == [0, a, b]
+    assert abs(res.tree_cum[c]) < 1e-20 and res.tree_cum[2] < -59
+    assert res.node_id.tolist() == [0, a, b]                          # ties go to the lower node id
+
+    def replay(ids):
+        f = _follow_from(res)
+        f.node_id = np.array([0] + ids, dtype=np.int64)
+        return O.draft(cfg, w, **r, follow=[f])[0]
+
+    # b and c score the same to 1e-24: by score alone {a, c} is as good as {a, b} ...
+    assert not O.admissible_topk(res.tree_cum[1:], [a - 1, c - 1], 2, 2e-3, ordered=False)
+    # ... but c's parent b would be missing from the emitted tree
+    swapped = replay([a, c])
+    assert any("ancestor-closed" in v for v in swapped.violations)
+    # with room for three nodes a swap among equal scores that keeps every parent is accepted:
+    # uniform logits, all nine depth-2 nodes tie, any of them may fill the last places
+    cfg2 = small_cfg(vocab=7, k=3, hidden=8, max_depth=2, total_tokens=6)
+    w2, r2 = uniform_weights(cfg2), S.make_roots(cfg2, 0)
+    res2 = O.draft(cfg2, w2, **r2)[0]
+    assert res2.node_id.tolist() == [0, 1, 2, 3, 4, 5, 6]
+    f = _follow_from(res2)
+    f.node_id = np.array([0, 1, 2, 3, 4, 5, 12], dtype=np.int64)
+    out = O.draft(cfg2, w2, **r2, follow=[f])[0]
+    assert not out.violations and out.node_id.tolist() == [0, 1, 2, 3, 4, 5, 12]
+    assert out.parent.tolist() == [-1, 0, 0, 0, 1, 1, 3]
+    assert any("rerank" in a_ for a_ in out.ambiguities)
 
 
 def test_admissible_topk_bands():

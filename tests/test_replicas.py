@@ -49,6 +49,44 @@ def test_two_rank_replica_sharding(tmp_path):
     assert [len(p) for p in res["gathered"]] == [4, 3]
 
 
+def _bench_rank_worker(rank, world, port, out_dir):
+    # what torchrun puts in the environment of each rank
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world),
+                      LOCAL_RANK=str(rank))
+    import contextlib
+    import io
+    import bench
+    got_rank, got_world, local = bench.dist_setup(world, backend="gloo")
+    cpu = torch.device("cpu")
+    bench.barrier(got_world)
+    slowest = bench.max_over_ranks(3.0 + 2.0 * got_rank, got_world, cpu)      # ms per step of this rank
+    total = bench.sum_over_ranks(5.0, got_world, cpu)
+    mine = list(S.shard_draft_indices(7 * got_world, got_rank, got_world))
+    buf = io.StringIO()
+    with contextlib.redirect_stdout(buf):
+        printed = bench.emit({"value": 7 * got_world / (slowest / 1e3), "n_gpus": got_world}, got_rank)
+    bench.barrier(got_world)
+    bench.dist_teardown(got_world)
+    torch.save({"rank": got_rank, "world": got_world, "local": local, "slowest": slowest, "total": total,
+                "mine": mine, "printed": printed, "stdout": buf.getvalue()}, os.path.join(out_dir, f"b{rank}.pt"))
+
+
+def test_bench_rank_logic_over_two_gloo_ranks(tmp_path):
+    """bench.py's own multi-rank code: group set-up from the torchrun environment, barrier, the
+    max-over-ranks time, and that rank 0 alone prints the line."""
+    import json
+    world = 2
+    mp.spawn(_bench_rank_worker, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True)
+    recs = [torch.load(os.path.join(tmp_path, f"b{r}.pt")) for r in range(world)]
+    assert [r["rank"] for r in recs] == [0, 1] and all(r["world"] == 2 for r in recs)
+    assert all(r["slowest"] == 5.0 for r in recs)            # every rank reports the slowest rank's time
+    assert all(r["total"] == 10.0 for r in recs)
+    assert sorted(recs[0]["mine"] + recs[1]["mine"]) == list(range(14))
+    assert recs[0]["printed"] and not recs[1]["printed"] and recs[1]["stdout"] == ""
+    line = json.loads(recs[0]["stdout"])
+    assert line["n_gpus"] == 2 and abs(line["value"] - 14 / 5e-3) < 1e-6
+
+
 def test_shard_is_a_partition_for_any_world_size():
     for n in (0, 1, 5, 32, 1000):
         for world in (1, 2, 3, 8):
