@@ -37,7 +37,7 @@ FALLBACK_HBM_GBS = 6650.0
 # profiles/, valid only while the kernel source is the one that was profiled.
 NCU_TRAFFIC = {"llama2_7b": {"bytes": 267.5e6, "source_sha256_16": "0b876d8fed98b331",
                              "profile": "profiles/lm_head_tc_llama2_7b.md"}}
-BEAM_WIDTHS = (5, 10, 20, 32)      # fixed-depth-6 sweep (the paper's appendix table goes on to 50, 75, 100)
+BEAM_WIDTHS = (5, 10, 20, 50, 75, 100)      # fixed-depth-6 sweep: the widths of the paper's appendix table
 OTHER_WORKLOADS = ("vicuna_13b", "llama2_70b_b16", "llama3_8b_128k")
 CLOCK_QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
                "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"

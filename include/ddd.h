@@ -72,11 +72,11 @@ enum { DDD_LM_HEAD_AUTO = 0, DDD_LM_HEAD_SIMT = 1, DDD_LM_HEAD_TCGEN05 = 2 };
  * profilers can follow. */
 enum { DDD_LAUNCH_STREAM = 0, DDD_LAUNCH_GRAPH = 1, DDD_LAUNCH_PLAIN = 2 };
 
-#define DDD_MAX_K 32          /* beam width limit                                  */
+#define DDD_MAX_K 128         /* beam width limit (the paper's appendix table goes to 100) */
 #define DDD_MAX_DEPTH 32      /* check_mask has one bit per step                   */
 #define DDD_MAX_TOTAL 1023    /* m limit (output rows = m + 1)                     */
 #define DDD_MAX_ROWS 256      /* B * k limit                                       */
-#define DDD_MAX_NODES 24576   /* 1 + k + (n-1) k^2 limit                           */
+#define DDD_MAX_NODES 98304   /* 1 + k + (n-1) k^2 limit                           */
 #define DDD_CHECK_EVERY_STEP 0xFFFFFFFFu
 
 /* Parameters of Algorithm 1 (n, w, S, x) and the tensor shapes. */
@@ -84,7 +84,9 @@ typedef struct {
   int32_t batch;        /* B >= 1 independent sequences                                           */
   int32_t hidden;       /* Hd, multiple of 8 (multiple of 64 for the TCGEN05 kernel)              */
   int32_t vocab;        /* V > k                                                                  */
-  int32_t k;            /* beam width w, 1..DDD_MAX_K                                             */
+  int32_t k;            /* beam width w, 1..DDD_MAX_K (beams wider than 32 take a slower, sort-based path;
+                           a configuration whose per-row lists do not fit on chip, e.g. 256 rows of
+                           width 128, is refused with DDD_ERR_UNSUPPORTED)                        */
   int32_t max_depth;    /* n: maximum number of draft-model calls, 1..DDD_MAX_DEPTH               */
   int32_t total_tokens; /* m: draft nodes kept by the rerank (the root is extra), 1..DDD_MAX_TOTAL */
   int32_t dtype;        /* DDD_DTYPE_*: storage type of W, E and every hidden state               */
@@ -251,7 +253,7 @@ int ddd_lm_head_blocks(const ddd_handle *h);
  *   out_token    DEVICE [rows][k] int32, best first (ties: lower token id)
  *   out_logprob  DEVICE [rows][k] fp32, clamped to <= 0
  *   out_lse      DEVICE [rows] fp32 logsumexp of the row's logits
- * Limits: 1 <= rows <= 32, 1 <= k <= DDD_MAX_K, hidden a multiple of 8, vocab > k.  Sizes
+ * Limits: 1 <= rows <= 32, 1 <= k <= 32, hidden a multiple of 8, vocab > k.  Sizes
  * beyond these do not fit the fixed scratch and return DDD_ERR_INVALID_ARG; misaligned W or
  * hidden_rows return DDD_ERR_ALIGNMENT.  Works on the device that is current in the calling
  * thread and only enqueues two kernels on `cuda_stream`; it calls no allocating routine.

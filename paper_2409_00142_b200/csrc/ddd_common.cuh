@@ -178,6 +178,116 @@ __device__ __forceinline__ void row_tile_update(const float* zrow, int tok0, int
                                    : 0ull;
 }
 
+// ---------------------------------------------------------------------------- wide lists (beam width 33..128)
+// A warp holds a list of 128 keys, four per lane: element e sits in lane e / 4, register e % 4.
+// Lists are kept sorted descending (position e = e-th best, 0 = empty at the end).  Everything a
+// wide beam needs - a row's running top-k, the merge of the thread blocks' partial lists, the
+// choice of the new beam among k sorted candidate rows - is built from two operations on such
+// lists: sort 128 keys, and merge two sorted lists keeping the best 128.
+constexpr int kWideK = 128;        // capacity of a wide list
+constexpr int kNarrowK = 32;       // beams up to this width keep one key per lane
+
+__device__ __forceinline__ unsigned long long shfl_xor_key(unsigned long long v, int mask) {
+  return __shfl_xor_sync(kFullMask, v, mask);
+}
+// One compare-exchange step of a bitonic network at distance j (a power of two, 1..64) inside
+// blocks of size k2 (descending where bit k2 of the element index is clear).
+__device__ __forceinline__ void bitonic_step(unsigned long long (&v)[4], int j, int k2) {
+  const int lane = threadIdx.x & 31;
+  if (j >= 4) {
+    const int lm = j >> 2;
+    const bool lower = (lane & lm) == 0;
+#pragma unroll
+    for (int s = 0; s < 4; ++s) {
+      const unsigned long long o = shfl_xor_key(v[s], lm);
+      const bool desc = ((4 * lane + s) & k2) == 0;
+      const bool keep_max = lower == desc;
+      v[s] = keep_max ? (v[s] > o ? v[s] : o) : (v[s] < o ? v[s] : o);
+    }
+  } else {
+#pragma unroll
+    for (int s = 0; s < 4; ++s) {
+      if ((s & j) == 0) {
+        const int t = s | j;
+        const bool desc = ((4 * lane + s) & k2) == 0;
+        const unsigned long long a = v[s], b = v[t];
+        const unsigned long long hi = a > b ? a : b, lo = a > b ? b : a;
+        v[s] = desc ? hi : lo;
+        v[t] = desc ? lo : hi;
+      }
+    }
+  }
+}
+// Sorts the warp's 128 keys descending.
+__device__ __forceinline__ void wide_sort(unsigned long long (&v)[4]) {
+  for (int k2 = 2; k2 <= kWideK; k2 <<= 1)
+    for (int j = k2 >> 1; j > 0; j >>= 1) bitonic_step(v, j, k2);
+}
+// a, b sorted descending -> a = the best 128 of both, sorted descending.
+__device__ __forceinline__ void wide_merge(unsigned long long (&a)[4], const unsigned long long (&b)[4]) {
+  const int lane = threadIdx.x & 31;
+#pragma unroll
+  for (int s = 0; s < 4; ++s) {
+    // element e of the reversed b is element 127 - e: lane 31 - lane, register 3 - s
+    const unsigned long long r = __shfl_sync(kFullMask, b[3 - s], 31 - lane);
+    a[s] = a[s] > r ? a[s] : r;                 // bitonic: first rising part of one, falling part of the other
+  }
+  for (int j = kWideK >> 1; j > 0; j >>= 1) bitonic_step(a, j, kWideK);
+}
+// Element e of a wide list (uniform e): broadcast from its lane.
+__device__ __forceinline__ unsigned long long wide_element(const unsigned long long (&v)[4], int e) {
+  unsigned long long x = v[0];
+  const int s = e & 3;
+  if (s == 1) x = v[1];
+  if (s == 2) x = v[2];
+  if (s == 3) x = v[3];
+  return __shfl_sync(kFullMask, x, e >> 2);
+}
+// Loads / stores the first `count` elements of a list laid out densely in memory (8-byte aligned).
+__device__ __forceinline__ void wide_load(unsigned long long (&v)[4], const unsigned long long* src, int count) {
+  const int lane = threadIdx.x & 31;
+#pragma unroll
+  for (int s = 0; s < 4; ++s) v[s] = (4 * lane + s < count) ? src[4 * lane + s] : 0ull;
+}
+__device__ __forceinline__ void wide_store(const unsigned long long (&v)[4], unsigned long long* dst, int count) {
+  const int lane = threadIdx.x & 31;
+#pragma unroll
+  for (int s = 0; s < 4; ++s)
+    if (4 * lane + s < count) dst[4 * lane + s] = v[s];
+}
+
+// The per-row tile update for wide beams: same contract as row_tile_update, with the row's list
+// held as a wide list.  A tile's 128 logits arrive four per lane in token order, which is the
+// list layout, so the tile is sorted as it stands and merged in.
+__device__ __forceinline__ void row_tile_update_wide(const float* zrow, int tok0, int k, float& m, float& s,
+                                                     unsigned long long (&list)[4]) {
+  const int lane = threadIdx.x & 31;
+  const float4 z4 = *reinterpret_cast<const float4*>(zrow + 4 * lane);
+  const float z[4] = {z4.x, z4.y, z4.z, z4.w};
+  const float lm = fmaxf(fmaxf(z[0], z[1]), fmaxf(z[2], z[3]));
+  const float mt = ordered_to_float(__reduce_max_sync(kFullMask, float_to_ordered(lm)));
+  if (mt == neg_inf()) return;
+  float ls = 0.f;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) ls += __expf(z[i] - mt);
+  const float st = warp_sum(ls);
+  if (mt > m) {
+    s = s * __expf(m - mt) + st;
+    m = mt;
+  } else {
+    s += st * __expf(mt - m);
+  }
+  unsigned long long t[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) t[i] = (z[i] == neg_inf()) ? 0ull : make_key(z[i], (uint32_t)(tok0 + 4 * lane + i));
+  // nothing to do unless some entry beats the current k-th best (0 while the list is not full)
+  const unsigned long long kth = wide_element(list, k - 1);
+  const unsigned long long best = max(max(t[0], t[1]), max(t[2], t[3]));
+  if (!__any_sync(kFullMask, best > kth)) return;
+  wide_sort(t);
+  wide_merge(list, t);
+}
+
 // ---------------------------------------------------------------------------- launchers (host)
 // Lets a kernel use as much dynamic shared memory as the device allows.  The limit is a
 // property of the function, shared by every handle of the process, so it is set to the

@@ -19,7 +19,7 @@ namespace {
 using namespace ddd;
 
 constexpr int kNaMaxRows = 32;      // beam rows per call
-constexpr int kNaMaxK = DDD_MAX_K;  // 32
+constexpr int kNaMaxK = 32;         // list width per row (one key per lane)
 constexpr int kNaMaxBlocks = 256;   // thread blocks of the first kernel
 constexpr int kNaThreads = 256;
 constexpr int kNaWarps = kNaThreads / 32;

@@ -47,7 +47,8 @@ __global__ void __launch_bounds__(kThreads) lm_head_simt_kernel(const Params p, 
   extern __shared__ __align__(16) unsigned char smem_raw[];
   float* zt = reinterpret_cast<float*>(smem_raw);
   unsigned long long* st_key = reinterpret_cast<unsigned long long*>(zt + (size_t)p.R * kTile);
-  float2* st_ms = reinterpret_cast<float2*>(st_key + (size_t)p.R * 32);
+  const int kst = p.k <= kNarrowK ? 32 : kWideK;     // keys kept per row: one or four per lane
+  float2* st_ms = reinterpret_cast<float2*>(st_key + (size_t)p.R * kst);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   constexpr int VEC = Vec<T>::N;
@@ -56,7 +57,7 @@ __global__ void __launch_bounds__(kThreads) lm_head_simt_kernel(const Params p, 
   const int n_tiles = (p.V + kTile - 1) / kTile;
 
   for (int r = warp; r < p.R; r += kWarps) {
-    st_key[r * 32 + lane] = 0ull;
+    for (int e = lane; e < kst; e += 32) st_key[r * kst + e] = 0ull;
     if (lane == 0) st_ms[r] = make_float2(neg_inf(), 0.f);
   }
   __syncthreads();
@@ -111,9 +112,16 @@ __global__ void __launch_bounds__(kThreads) lm_head_simt_kernel(const Params p, 
     for (int r = warp; r < p.R; r += kWarps) {
       if (!row_live(p, r, d, force_all)) continue;
       float2 ms = st_ms[r];
-      unsigned long long key = st_key[r * 32 + lane];
-      row_tile_update(zt + (size_t)r * kTile, v0, p.k, ms.x, ms.y, key);
-      st_key[r * 32 + lane] = key;
+      if (p.k <= kNarrowK) {
+        unsigned long long key = st_key[r * 32 + lane];
+        row_tile_update(zt + (size_t)r * kTile, v0, p.k, ms.x, ms.y, key);
+        st_key[r * 32 + lane] = key;
+      } else {
+        unsigned long long list[4];
+        wide_load(list, st_key + (size_t)r * kWideK, kWideK);
+        row_tile_update_wide(zt + (size_t)r * kTile, v0, p.k, ms.x, ms.y, list);
+        wide_store(list, st_key + (size_t)r * kWideK, kWideK);
+      }
       if (lane == 0) st_ms[r] = ms;
     }
     __syncthreads();
@@ -123,13 +131,14 @@ __global__ void __launch_bounds__(kThreads) lm_head_simt_kernel(const Params p, 
   for (int r = warp; r < p.R; r += kWarps) {
     if (!row_live(p, r, d, force_all)) continue;
     const size_t slot = (size_t)blockIdx.x * p.R + r;
-    if (lane < p.k) p.part_key[slot * p.k + lane] = st_key[r * 32 + lane];
+    for (int e = lane; e < p.k; e += 32) p.part_key[slot * p.k + e] = st_key[r * kst + e];
     if (lane == 0) p.part_ms[slot] = st_ms[r];
   }
 }
 
 size_t simt_smem(const Params& p) {
-  return (size_t)p.R * kTile * sizeof(float) + (size_t)p.R * 32 * sizeof(unsigned long long) +
+  const size_t kst = p.k <= kNarrowK ? 32 : kWideK;
+  return (size_t)p.R * kTile * sizeof(float) + (size_t)p.R * kst * sizeof(unsigned long long) +
          (size_t)p.R * sizeof(float2);
 }
 

@@ -51,13 +51,17 @@ struct SmemPlan {
   int a, b, zt, key, ms, plant, live, bars, tmem_ptr, abort_flag, total;
 };
 
+// Keys kept per beam row in shared memory: k for beams of up to 32 (one key per lane), else k
+// rounded up to whole lanes of four (the wide-list layout).
+__host__ __device__ inline int key_stride(int k) { return k <= kNarrowK ? k : (k + 3) & ~3; }
+
 __host__ __device__ inline SmemPlan smem_plan(int stages, int ksub, int n_pad, int R, int k, int cpg) {
   SmemPlan s;
   int off = 0;
   s.a = off; off += stages * ksub * kABytes;
   s.b = off; off += stages * ksub * n_pad * kBlockK * 2;
   s.zt = off; off += cpg * kChunkCols * kTile * 4;
-  s.key = off; off += R * k * 8;
+  s.key = off; off += R * key_stride(k) * 8;
   s.ms = off; off += R * 8;
   s.plant = off; off += R * 4;
   s.live = off; off += R * 4;
@@ -346,7 +350,8 @@ lm_head_tc_kernel(const Params p, const unsigned char* __restrict__ w_packed,
     s_live[r] = row_live(p, r, d, force_all) ? 1 : 0;
     st_ms[r] = make_float2(neg_inf(), 0.f);
   }
-  for (int i = threadIdx.x; i < p.R * p.k; i += kTcThreads) st_key[i] = 0ull;
+  const int kst = key_stride(p.k);
+  for (int i = threadIdx.x; i < p.R * kst; i += kTcThreads) st_key[i] = 0ull;
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -465,9 +470,16 @@ lm_head_tc_kernel(const Params p, const unsigned char* __restrict__ w_packed,
           const int r = g0 * kChunkCols + rr;
           if (r >= p.R || !s_live[r]) continue;
           float2 ms = st_ms[r];
-          unsigned long long key = lane < p.k ? st_key[r * p.k + lane] : 0ull;
-          row_tile_update(zt + rr * kTile, row0, p.k, ms.x, ms.y, key);
-          if (lane < p.k) st_key[r * p.k + lane] = key;
+          if (p.k <= kNarrowK) {
+            unsigned long long key = lane < p.k ? st_key[r * p.k + lane] : 0ull;
+            row_tile_update(zt + rr * kTile, row0, p.k, ms.x, ms.y, key);
+            if (lane < p.k) st_key[r * p.k + lane] = key;
+          } else {
+            unsigned long long list[4];
+            wide_load(list, st_key + r * kst, kst);
+            row_tile_update_wide(zt + rr * kTile, row0, p.k, ms.x, ms.y, list);
+            wide_store(list, st_key + r * kst, kst);
+          }
           if (lane == 0) st_ms[r] = ms;
         }
         epilogue_barrier();
@@ -478,7 +490,7 @@ lm_head_tc_kernel(const Params p, const unsigned char* __restrict__ w_packed,
       for (int r = ew; r < p.R; r += kEpiWarps) {
         if (!s_live[r]) continue;
         const size_t slot = (size_t)bid * p.R + r;
-        if (lane < p.k) p.part_key[slot * p.k + lane] = st_key[r * p.k + lane];
+        for (int e = lane; e < p.k; e += 32) p.part_key[slot * p.k + e] = st_key[r * kst + e];
         if (lane == 0) p.part_ms[slot] = st_ms[r];
       }
     }

@@ -138,14 +138,17 @@ __device__ int block_exclusive_scan(int v, int* warp_tot /* [32] shared */, int*
 // which the sequence stopped (D): keep the m best nodes, emit the rows and the ancestor mask.
 // smem_raw: ordered cum keys [Nn] (32 bit), then selection flags / output rows [Nn] (16 bit).  `last` says that this
 // was the last sequence of the batch still drafting: that block also reports the device status.
-template <int THREADS>
+// KEYS_IN_SMEM false: the tree is too large to keep its keys in shared memory; they are formed from
+// the scores in global memory each time (smem_raw then holds only the 16-bit rows).
+template <int THREADS, bool KEYS_IN_SMEM>
 __device__ void rerank_mask_block(const Params& p, const DraftIO& io, const int b, const int D, const bool last,
                                   unsigned char* smem_raw) {
   const int tid = threadIdx.x;
   const int k = p.k, T = p.T;
   const int N = (D >= 1) ? k + (D - 1) * k * k : 0;     // generated non-root nodes
-  uint32_t* key = reinterpret_cast<uint32_t*>(smem_raw);           // key of node id i+1 at [i]
-  short* slot_of = reinterpret_cast<short*>(key + p.Nn);            // output row of node id (< 1024), -1 = dropped
+  uint32_t* key_s = reinterpret_cast<uint32_t*>(smem_raw);         // key of node id i+1 at [i]
+  short* slot_of = reinterpret_cast<short*>(KEYS_IN_SMEM ? smem_raw + (size_t)p.Nn * sizeof(uint32_t) : smem_raw);
+                                                                    // output row of node id (< 1024), -1 = dropped
   __shared__ int hist[256];
   __shared__ int warp_tot[32];
   __shared__ uint32_t s_prefix;
@@ -155,7 +158,9 @@ __device__ void rerank_mask_block(const Params& p, const DraftIO& io, const int 
   const float* cum = p.tree_cum + (size_t)b * p.Nn;
   const int* tparent = p.tree_parent + (size_t)b * p.Nn;
   const int* ttoken = p.tree_token + (size_t)b * p.Nn;
-  for (int i = tid; i < N; i += THREADS) key[i] = float_to_ordered(cum[i + 1]);
+  auto key = [&](int i) -> uint32_t { return KEYS_IN_SMEM ? key_s[i] : float_to_ordered(cum[i + 1]); };
+  if (KEYS_IN_SMEM)
+    for (int i = tid; i < N; i += THREADS) key_s[i] = float_to_ordered(cum[i + 1]);
   const int m_eff = min(p.m, N);
   if (tid == 0) { s_prefix = 0u; s_remaining = m_eff; }
   __syncthreads();
@@ -168,7 +173,7 @@ __device__ void rerank_mask_block(const Params& p, const DraftIO& io, const int 
     __syncthreads();
     const uint32_t prefix = s_prefix;
     for (int i = tid; i < N; i += THREADS) {
-      const uint32_t q = key[i];
+      const uint32_t q = key(i);
       if ((q & known_mask) == prefix) atomicAdd(&hist[(q >> shift) & 0xFF], 1);
     }
     __syncthreads();
@@ -205,12 +210,12 @@ __device__ void rerank_mask_block(const Params& p, const DraftIO& io, const int 
   const int chunk = (N + THREADS - 1) / THREADS;
   const int lo = min(N, tid * chunk), hi = min(N, lo + chunk);
   int n_eq = 0;
-  for (int i = lo; i < hi; ++i) n_eq += (key[i] == thr);
+  for (int i = lo; i < hi; ++i) n_eq += (key(i) == thr);
   int tot_unused;
   int eq_before = block_exclusive_scan<THREADS>(n_eq, warp_tot, &tot_unused);
   int n_sel = 0;
   for (int i = lo; i < hi; ++i) {
-    const uint32_t q = key[i];
+    const uint32_t q = key(i);
     bool sel = false;
     if (m_eff > 0) {
       if (q > thr) sel = true;

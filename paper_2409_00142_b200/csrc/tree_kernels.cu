@@ -278,19 +278,19 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
   int* plant_s = reinterpret_cast<int*>(ms_s + (size_t)rows_max * nc);                        // [rows_max]
   // candidate (p, c) of this pass at [p * k + c]: score bits in the upper word, token (-1 = none)
   // in the lower; one 8-byte store per block of the cluster carries it there
-  __shared__ unsigned long long cand_rec[DDD_MAX_K * DDD_MAX_K];
+  __shared__ unsigned long long cand_rec[kNarrowK * kNarrowK];
   auto cand_key_of = [&](int idx) -> unsigned long long {     // selection key: score, ties to the lower index
     const unsigned long long rec = cand_rec[idx];
     return (int)(uint32_t)rec >= 0 ? make_key(__uint_as_float((uint32_t)(rec >> 32)), (uint32_t)idx) : 0ull;
   };
-  __shared__ int sel_flat[DDD_MAX_K];
-  __shared__ int sel_tok[DDD_MAX_K];
-  __shared__ double row_part[DDD_MAX_K * 64];
-  __shared__ double row_inv[DDD_MAX_K];
+  __shared__ int sel_flat[kNarrowK];
+  __shared__ int sel_tok[kNarrowK];
+  __shared__ double row_part[kNarrowK * 64];
+  __shared__ double row_inv[kNarrowK];
   __shared__ int s_stop;
   __shared__ bool s_last;
-  __shared__ float beam_cum_s[DDD_MAX_K / kSelCluster];
-  __shared__ int beam_node_s[DDD_MAX_K / kSelCluster];
+  __shared__ float beam_cum_s[kNarrowK / kSelCluster];
+  __shared__ int beam_node_s[kNarrowK / kSelCluster];
 
   // ---- phase 0: the block fetches everything phase 1 needs for its rows in one round trip.
   // The copies go from global to shared memory asynchronously (a warp copies one LM-head block's
@@ -321,9 +321,9 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
 
   // ---- phase 1: per beam row of this block, warp j merges the top-k lists while warp j + 4
   //      adds up the log-sum-exp of the same row
-  __shared__ float lse_s[DDD_MAX_K / kSelCluster];
-  __shared__ unsigned long long plant_key_s[DDD_MAX_K / kSelCluster];
-  constexpr int kRowsPerBlock = DDD_MAX_K / kSelCluster;
+  __shared__ float lse_s[kNarrowK / kSelCluster];
+  __shared__ unsigned long long plant_key_s[kNarrowK / kSelCluster];
+  constexpr int kRowsPerBlock = kNarrowK / kSelCluster;
   unsigned long long res = 0ull;
   if (warp < n_mine) {
     const int r = b * k + crank + kSelCluster * warp;
@@ -478,11 +478,206 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
     // the sequence is finished: block 0 goes on to the rerank and the mask once the nodes the other
     // blocks appended in this pass are visible to it
     cluster.sync();
-    if (crank == 0) rerank_mask_block<kSelThreads>(p, io, b, d, s_last, smem_raw);
+    if (crank == 0) rerank_mask_block<kSelThreads, true>(p, io, b, d, s_last, smem_raw);
     return;
   }
 
   // ---- phase 3: synthetic draft step for the k new beam rows
+  if (p.dtype == DDD_DTYPE_BF16)
+    draft_step<__nv_bfloat16>(p, b, d, sel_flat, sel_tok, row_part, row_inv);
+  else
+    draft_step<float>(p, b, d, sel_flat, sel_tok, row_part, row_inv);
+}
+
+
+// ---------------------------------------------------------------------------- wide beams (width 33..128)
+// The same pass for beams too wide for one key per lane.  Every list here - a thread block's
+// partial top-k of a row, a row's k candidates, the new beam - is a sorted wide list (four keys
+// per lane, ddd_common.cuh), and every choice is a merge of sorted lists: the warps of a block
+// each fold a share of the lists into one, the 16 results meet in shared memory and are merged
+// pairwise in four rounds.
+constexpr int kWideThreads = 512;
+constexpr int kWideWarps = kWideThreads / 32;
+
+// Tree of pairwise merges over the warps' lists in buf [kWideWarps][kWideK]; the result ends up
+// in warp 0's registers (and in buf[0]).  All threads of the block call this.
+__device__ __forceinline__ void block_merge_lists(unsigned long long (&acc)[4], unsigned long long* buf) {
+  const int warp = threadIdx.x >> 5;
+  wide_store(acc, buf + warp * kWideK, kWideK);
+  __syncthreads();
+  for (int half = kWideWarps / 2; half >= 1; half >>= 1) {
+    if (warp < half) {
+      unsigned long long other[4];
+      wide_load(other, buf + (warp + half) * kWideK, kWideK);
+      wide_merge(acc, other);
+      wide_store(acc, buf + warp * kWideK, kWideK);
+    }
+    __syncthreads();
+  }
+}
+
+// Dynamic shared memory: candidate records [k*k], merge buffers [16][128], partial sums of squares
+// of the draft step [k][slots]; after a stop the same memory serves the rerank.
+__global__ void __launch_bounds__(kWideThreads) select_gate_step_wide_kernel(const Params p, const DraftIO io,
+                                                                             const int d, const int part_slots,
+                                                                             const cudaGraphConditionalHandle cond,
+                                                                             const int set_cond) {
+  griddep_wait();
+  griddep_launch_dependents();
+  cg::cluster_group cluster = cg::this_cluster();
+  const int crank = (int)cluster.block_rank();
+  const int b = blockIdx.x / kSelCluster;
+  if (p.active[b] == 0) return;                               // same decision in the whole cluster
+  // split cluster barrier: remote shared-memory stores below need every block of the cluster running
+  asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int k = p.k, nc = p.lm_ctas, R = p.R;
+  const int P = (d == 1) ? 1 : k;
+  const int base = (d == 1) ? 1 : 1 + k + (d - 2) * k * k;
+
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  unsigned long long* cand_rec = reinterpret_cast<unsigned long long*>(smem_raw);           // [k * k]
+  unsigned long long* buf = cand_rec + (size_t)k * k;                                       // [16][128]
+  double* row_part = reinterpret_cast<double*>(buf + kWideWarps * kWideK);                  // [k][part_slots]
+  __shared__ int sel_flat[kWideK];
+  __shared__ int sel_tok[kWideK];
+  __shared__ double row_inv[kWideK];
+  __shared__ int s_stop;
+  __shared__ bool s_last;
+  (void)part_slots;
+
+  // ---- phase 1: merge the partial lists of this block's beam rows, one row at a time
+  bool waited = false;
+  for (int pr = crank; pr < P; pr += kSelCluster) {
+    const int r = b * k + pr;
+    unsigned long long acc[4] = {0ull, 0ull, 0ull, 0ull};
+    for (int c = warp; c < nc; c += kWideWarps) {
+      unsigned long long t[4];
+      wide_load(t, p.part_key + ((size_t)c * R + r) * k, k);
+      wide_merge(acc, t);
+    }
+    block_merge_lists(acc, buf);
+    if (!waited) {
+      asm volatile("barrier.cluster.wait.aligned;" ::: "memory");
+      waited = true;
+    }
+    if (warp == 0) {
+      float M = neg_inf();
+      for (int c = lane; c < nc; c += 32) M = fmaxf(M, p.part_ms[(size_t)c * R + r].x);
+      M = ordered_to_float(__reduce_max_sync(kFullMask, float_to_ordered(M)));
+      float S = 0.f;
+      for (int c = lane; c < nc; c += 32) {
+        const float2 ms = p.part_ms[(size_t)c * R + r];
+        if (ms.y > 0.f) S += ms.y * expf(ms.x - M);
+      }
+      S = warp_sum(S);
+      const int pc = p.row_plant[r];
+      if (pc >= 0) {          // planted column: (max of the others) + delta; it was left out of the partials
+        const float zc = M + p.plant_delta;
+        const float M2 = fmaxf(M, zc);
+        S = S * expf(M - M2) + expf(zc - M2);
+        M = M2;
+        unsigned long long one[4] = {lane == 0 ? make_key(zc, (uint32_t)pc) : 0ull, 0ull, 0ull, 0ull};
+        wide_merge(acc, one);
+      }
+      const float lse = M + logf(S);
+      const float cum0 = p.beam_cum[r];
+      const int parent_node = p.beam_node[r];
+#pragma unroll
+      for (int s4 = 0; s4 < 4; ++s4) {
+        const int e = 4 * lane + s4;
+        if (e >= k) continue;
+        const unsigned long long key = acc[s4];
+        const float lp = key != 0ull ? fminf(key_value(key) - lse, 0.f) : neg_inf();
+        const int tok = key != 0ull ? (int)key_index(key) : -1;
+        const float cand = cum0 + lp;
+        const int flat = pr * k + e;
+        const unsigned long long rec = ((unsigned long long)__float_as_uint(cand) << 32) | (uint32_t)tok;
+        for (int rk = 0; rk < kSelCluster; ++rk) cluster.map_shared_rank(cand_rec, rk)[flat] = rec;
+        const size_t node = (size_t)b * p.Nn + base + flat;
+        p.tree_token[node] = tok;
+        p.tree_parent[node] = parent_node;
+        p.tree_cum[node] = cand;
+      }
+      if (lane == 0 && io.trace.row_lse) io.trace.row_lse[((size_t)b * p.n + (d - 1)) * k + pr] = lse;
+    }
+    __syncthreads();
+  }
+  if (!waited) asm volatile("barrier.cluster.wait.aligned;" ::: "memory");
+  cluster.sync();
+
+  // ---- phase 2: the new beam = best k of the P sorted candidate rows (every block, same result)
+  {
+    unsigned long long acc[4] = {0ull, 0ull, 0ull, 0ull};
+    for (int row = warp; row < P; row += kWideWarps) {
+      unsigned long long t[4];
+#pragma unroll
+      for (int s4 = 0; s4 < 4; ++s4) {
+        const int e = 4 * lane + s4;
+        t[s4] = 0ull;
+        if (e < k) {
+          const unsigned long long rec = cand_rec[row * k + e];
+          if ((int)(uint32_t)rec >= 0) t[s4] = make_key(__uint_as_float((uint32_t)(rec >> 32)), (uint32_t)(row * k + e));
+        }
+      }
+      wide_merge(acc, t);
+    }
+    block_merge_lists(acc, buf);
+    if (warp == 0) {
+      float cum[4];
+      int flat[4], tok[4];
+      float part = 0.f;
+      const float M = key_value(wide_element(acc, 0));          // sorted descending: entry 0 is the maximum
+#pragma unroll
+      for (int s4 = 0; s4 < 4; ++s4) {
+        const int e = 4 * lane + s4;
+        const bool have = e < k && acc[s4] != 0ull;
+        flat[s4] = have ? (int)key_index(acc[s4]) : 0;
+        cum[s4] = have ? key_value(acc[s4]) : neg_inf();
+        tok[s4] = e < k ? (int)(uint32_t)cand_rec[flat[s4]] : -1;
+        if (have) part += expf(cum[s4] - M);
+        if (e < k) {
+          sel_flat[e] = flat[s4];
+          sel_tok[e] = tok[s4];
+        }
+      }
+      const float H = M + logf(warp_sum(part));
+      bool stop = (d == p.n);
+      if (!stop && ((p.check_mask >> (d - 1)) & 1u)) stop = H < p.x;
+      if (lane == 0) s_stop = stop ? 1 : 0;
+      __syncwarp();
+      if (crank == 0) {
+#pragma unroll
+        for (int s4 = 0; s4 < 4; ++s4) {
+          const int e = 4 * lane + s4;
+          if (e >= k) continue;
+          p.beam_node[b * k + e] = base + flat[s4];
+          p.beam_tok[b * k + e] = tok[s4];
+          p.beam_cum[b * k + e] = cum[s4];
+          p.row_plant[b * k + e] = (p.plant_next && tok[s4] >= 0 && tok[s4] < p.V) ? p.plant_next[tok[s4]] : -1;
+          if (io.trace.beam_sel) io.trace.beam_sel[((size_t)b * p.n + (d - 1)) * k + e] = flat[s4];
+        }
+        if (lane == 0) {
+          io.out.H_trace[(size_t)b * p.n + (d - 1)] = H;
+          if (stop) {
+            p.stop_depth[b] = d;
+            p.active[b] = 0;
+            s_last = atomicSub(p.n_active, 1) == 1;
+          }
+        }
+      }
+    }
+  }
+  __syncthreads();
+  if (set_cond && !s_stop && crank == 0 && threadIdx.x == 0) cudaGraphSetConditional(cond, 1);
+  if (s_stop) {
+    cluster.sync();          // the nodes the other blocks appended in this pass are visible to block 0
+    if (crank == 0) {
+      if (p.Nn * 6 <= 160 * 1024) rerank_mask_block<kWideThreads, true>(p, io, b, d, s_last, smem_raw);
+      else rerank_mask_block<kWideThreads, false>(p, io, b, d, s_last, smem_raw);
+    }
+    return;
+  }
   if (p.dtype == DDD_DTYPE_BF16)
     draft_step<__nv_bfloat16>(p, b, d, sel_flat, sel_tok, row_part, row_inv);
   else
@@ -499,10 +694,24 @@ size_t select_smem_bytes(const Params& p, bool lists) {
 bool select_lists_in_smem(const Params& p) {
   return p.lm_ctas <= 320 && select_smem_bytes(p, true) <= 160 * 1024;
 }
-size_t rerank_smem(const Params& p) { return (size_t)p.Nn * (sizeof(uint32_t) + sizeof(short)); }
+bool is_wide(const Params& p) { return p.k > kNarrowK; }
+// the rerank keeps 32-bit keys and 16-bit row numbers of all tree nodes in shared memory; trees too
+// large for that (wide beams) keep only the row numbers there and read the scores from global memory
+size_t rerank_smem(const Params& p) {
+  const size_t both = (size_t)p.Nn * (sizeof(uint32_t) + sizeof(short));
+  return (!is_wide(p) || both <= 160 * 1024) ? both : (size_t)p.Nn * sizeof(short);
+}
+int wide_part_slots(const Params& p) {
+  const int cpr = p.Hd / (p.dtype == DDD_DTYPE_BF16 ? 8 : 4);
+  return (cpr % 32 == 0 && cpr / 32 <= 64) ? cpr / 32 : 0;
+}
+size_t wide_select_smem(const Params& p) {
+  return ((size_t)p.k * p.k + kWideWarps * kWideK) * sizeof(unsigned long long) +
+         (size_t)p.k * wide_part_slots(p) * sizeof(double);
+}
 // the select kernel's dynamic shared memory also serves the rerank that follows a stop
 size_t select_smem(const Params& p) {
-  const size_t a = select_smem_bytes(p, select_lists_in_smem(p)), b = rerank_smem(p);
+  const size_t a = is_wide(p) ? wide_select_smem(p) : select_smem_bytes(p, select_lists_in_smem(p)), b = rerank_smem(p);
   return a > b ? a : b;
 }
 
@@ -513,13 +722,15 @@ cudaError_t prepare_tree(const Params& p) {
   // static + dynamic shared memory of the select kernel must fit one block's limit
   cudaFuncAttributes fa;
   const bool wide = p.k >= kSelWideFromK;
-  cudaError_t e = wide ? cudaFuncGetAttributes(&fa, select_gate_step_kernel<kSelThreadsWide>)
-                       : cudaFuncGetAttributes(&fa, select_gate_step_kernel<kSelThreadsNarrow>);
+  cudaError_t e = is_wide(p) ? cudaFuncGetAttributes(&fa, select_gate_step_wide_kernel)
+                  : wide     ? cudaFuncGetAttributes(&fa, select_gate_step_kernel<kSelThreadsWide>)
+                             : cudaFuncGetAttributes(&fa, select_gate_step_kernel<kSelThreadsNarrow>);
   if (e != cudaSuccess) return e;
   int dev = 0, limit = 0;
   if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
   if ((e = cudaDeviceGetAttribute(&limit, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev)) != cudaSuccess) return e;
   if (fa.sharedSizeBytes + select_smem(p) > (size_t)limit) return cudaErrorInvalidValue;
+  if (is_wide(p)) return allow_max_dynamic_smem(select_gate_step_wide_kernel);
   return wide ? allow_max_dynamic_smem(select_gate_step_kernel<kSelThreadsWide>)
               : allow_max_dynamic_smem(select_gate_step_kernel<kSelThreadsNarrow>);
 }
@@ -539,7 +750,7 @@ cudaError_t launch_select(const Params& p, const DraftIO& io, int d, bool pdl, c
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(p.B * kSelCluster), 1, 1);
   const bool wide = p.k >= kSelWideFromK;
-  cfg.blockDim = dim3(wide ? kSelThreadsWide : kSelThreadsNarrow, 1, 1);
+  cfg.blockDim = dim3(is_wide(p) ? kWideThreads : wide ? kSelThreadsWide : kSelThreadsNarrow, 1, 1);
   cfg.dynamicSmemBytes = select_smem(p);
   cfg.stream = st;
   cudaLaunchAttribute attr[2];
@@ -552,6 +763,8 @@ cudaError_t launch_select(const Params& p, const DraftIO& io, int d, bool pdl, c
   cfg.attrs = attr;
   cfg.numAttrs = pdl ? 2 : 1;
   const int lists = select_lists_in_smem(p) ? 1 : 0, sc = set_cond ? 1 : 0;
+  if (is_wide(p))
+    return cudaLaunchKernelEx(&cfg, select_gate_step_wide_kernel, p, io, d, wide_part_slots(p), cond, sc);
   if (wide) return cudaLaunchKernelEx(&cfg, select_gate_step_kernel<kSelThreadsWide>, p, io, d, lists, cond, sc);
   return cudaLaunchKernelEx(&cfg, select_gate_step_kernel<kSelThreadsNarrow>, p, io, d, lists, cond, sc);
 }

@@ -32,9 +32,9 @@ def test_library_exports_every_declared_symbol():
 
 def test_workspace_bytes_and_config_validation():
     assert P.ddd_workspace_bytes(good_config()) > 0
-    for bad in (dict(batch=0), dict(hidden=100), dict(k=0), dict(k=33), dict(vocab=4), dict(max_depth=0),
+    for bad in (dict(batch=0), dict(hidden=100), dict(k=0), dict(k=129), dict(vocab=4), dict(max_depth=0),
                 dict(max_depth=33), dict(total_tokens=0), dict(total_tokens=1024), dict(dtype=7),
-                dict(batch=100, k=4), dict(k=32, max_depth=32), dict(lm_head_kernel=9), dict(launch_mode=5),
+                dict(batch=100, k=4), dict(k=64, max_depth=32, vocab=4096), dict(lm_head_kernel=9), dict(launch_mode=5),
                 dict(logit_scale=float("nan")), dict(device=-1)):
         assert P.ddd_workspace_bytes(good_config(**bad)) == 0, bad
     big = P.ddd_workspace_bytes(good_config(batch=16, hidden=8192, vocab=32000, k=10, max_depth=10,

@@ -138,6 +138,50 @@ def test_k1_greedy_chain_and_k_equal_to_limit():
             eng.close()
 
 
+# ----------------------------------------------------------------------------- wide beams (the paper's appendix: up to 100)
+def wide_cases():
+    base = S.scaled_down(S.CONFIGS["llama2_7b"], 256, 3000 + 24, threshold=NEG, max_depth=3, total_tokens=200)
+    zipf = S.scaled_down(S.CONFIGS["llama3_8b_128k"], 128, 9000 + 5, threshold=-6.0, max_depth=4, total_tokens=300)
+    return {
+        "k33": base.replace(k=33),                                   # first width past one key per lane
+        "k50": base.replace(k=50),
+        "k75_two_sequences": base.replace(k=75, batch=2, max_depth=2, threshold=-9.0),   # 150 rows in a pass
+        "k100": base.replace(k=100),
+        "k128": base.replace(k=128, max_depth=2),                    # the limit
+        "k100_zipf": zipf.replace(k=100, batch=1),                   # winners cluster in the first vocab tiles
+        # 28,737 tree nodes: more than the rerank keeps keys for in shared memory
+        "k64_large_tree": S.scaled_down(S.CONFIGS["vicuna_13b"], 128, 2000, threshold=NEG, k=64, max_depth=8,
+                                        total_tokens=500, plant_frac=0.2),
+    }
+
+
+@pytest.mark.parametrize("kernel", [SIMT, TC], ids=["simt", "tcgen05"])
+@pytest.mark.parametrize("case", list(wide_cases()))
+def test_wide_beams_match_oracle(case, kernel):
+    cfg = wide_cases()[case]
+    if kernel == SIMT and cfg.batch * cfg.k > 128:
+        pytest.skip("the CUDA-core kernel keeps at most 128 wide rows in shared memory")
+    eng = engine_for(cfg, kernel, P.DDD_LAUNCH_GRAPH if case == "k50" else P.DDD_LAUNCH_STREAM)
+    with torch.cuda.stream(torch.cuda.Stream()):
+        for i in range(2):
+            roots = S.make_roots(cfg, i)
+            g = parity.run_gpu(eng, roots)
+            parity.compare_with_oracle(cfg, weights_for(cfg), roots, g)
+    eng.close()
+
+
+def test_full_size_7b_at_width_100_depth_6():
+    # the widest row of the paper's appendix table, in the configuration the benchmark's sweep times
+    cfg = S.CONFIGS["llama2_7b"].replace(k=100, max_depth=6, threshold=NEG, total_tokens=60)
+    eng = engine_for(cfg, P.DDD_LM_HEAD_AUTO, P.DDD_LAUNCH_GRAPH)
+    with torch.cuda.stream(torch.cuda.Stream()):
+        roots = S.make_roots(cfg, 0)
+        g = parity.run_gpu(eng, roots)
+    parity.compare_with_oracle(cfg, weights_for(cfg), roots, g)
+    assert int(g["stop_depth"][0]) == 6 and int(g["n_out"][0]) == 61
+    eng.close()
+
+
 def edge_cases():
     base = S.scaled_down(S.CONFIGS["llama2_7b"], 128, 1000, threshold=NEG)
     return {
