@@ -77,6 +77,7 @@ enum { DDD_LAUNCH_STREAM = 0, DDD_LAUNCH_GRAPH = 1, DDD_LAUNCH_PLAIN = 2 };
 #define DDD_MAX_TOTAL 1023    /* m limit (output rows = m + 1)                     */
 #define DDD_MAX_ROWS 256      /* B * k limit                                       */
 #define DDD_MAX_NODES 98304   /* 1 + k + (n-1) k^2 limit                           */
+#define DDD_MAX_SHARDS 16      /* slices of a vocabulary-parallel LM head           */
 #define DDD_CHECK_EVERY_STEP 0xFFFFFFFFu
 
 /* Parameters of Algorithm 1 (n, w, S, x) and the tensor shapes. */
@@ -98,6 +99,8 @@ typedef struct {
   int32_t device;       /* CUDA device ordinal                                                    */
   int32_t lm_head_kernel; /* DDD_LM_HEAD_*                                                        */
   int32_t launch_mode;    /* DDD_LAUNCH_*                                                         */
+  int32_t vocab_begin;    /* first token id of the slice of W this handle owns, and                      */
+  int32_t vocab_count;    /* its number of rows; 0, 0 = the whole vocabulary (see ddd_shard_* below)      */
 } ddd_config;
 
 /*
@@ -266,6 +269,51 @@ int ddd_lm_head_blocks(const ddd_handle *h);
 int ddd_lm_head_topk_noalloc(const void *W, const float *bias, const void *hidden_rows, int32_t dtype,
                              int32_t rows, int32_t hidden, int32_t vocab, int32_t k, float logit_scale,
                              int32_t *out_token, float *out_logprob, float *out_lse, void *cuda_stream);
+
+/*
+ * Vocabulary-parallel LM head.  (The paper runs on one GPU - Section 3.1, Setup - and has no
+ * counterpart; this splits the one step of Algorithm 1 that streams the LM-head matrix.)
+ * G ranks, one handle each, created with vocab_begin / vocab_count set: such a handle takes as W
+ * only the rows [vocab_begin, vocab_begin + vocab_count) of the LM head (DEVICE
+ * [vocab_count][Hd]) and as bias the matching slice ([vocab_count] or NULL); E, plant_next and
+ * cfg->vocab stay those of the whole vocabulary, and token ids everywhere are global.  Every rank
+ * keeps the whole tree state and runs the same select / gate / draft step; only the LM-head pass
+ * is split.  A pass d = 1..n is three steps on every rank:
+ *   ddd_shard_lm_head  streams the rank's slice and folds the result into one record per beam row:
+ *                      the slice's (max, sum-exp) and its k best (logit, token) pairs.  The record
+ *                      goes to slot `slot` of each of the n_dst record sets listed in records_dst:
+ *                      the rank's own and, through peer pointers, those of the other ranks (or
+ *                      only its own, if the caller moves records itself, e.g. with an all-gather).
+ *                      If flags_dst is given, flags_dst[i][slot] is set to a value that names this
+ *                      draft and pass once the records are on their way.
+ *   (exchange)         whatever carries the other ranks' records into this rank's record set
+ *   ddd_shard_select   merges the `slots` records of a record set, in slot order, and runs the
+ *                      ordinary select / gate / draft step of pass d; with `flags` given it first
+ *                      waits, bounded, until all of them name this draft and pass (a wait that
+ *                      runs out sets status to DDD_ERR_TIMEOUT; nothing hangs).
+ * A record set is ddd_shard_records_bytes(cfg, slots) bytes, 16-byte aligned; flags are `slots`
+ * int32 words, zero before the first draft.  Use two record sets and flag arrays, alternating by
+ * the parity of d: a rank may already be writing pass d + 1 while a slower peer still reads pass d.
+ * ddd_shard_begin starts a draft (resets the state, loads the root; every rank passes the same
+ * inputs) and must be called the same number of times on every rank, since the flag values count
+ * drafts.  After a sequence has stopped, the calls of later passes do nothing for it; once all have
+ * stopped they do nothing at all but still raise their flags, so the simplest caller enqueues all
+ * n passes.  Results land in `out` / `trace` of ddd_shard_begin on every rank alike.  Per-slice
+ * sums are added up per rank and then across ranks, so scores may differ from an unsharded draft
+ * in the last bits (not in the tokens, unless two scores tie to within those bits).
+ * ddd_draft* on a handle that owns a slice return DDD_ERR_INVALID_ARG.  A handle that owns the
+ * whole vocabulary may use these calls with slots = 1: a one-slice run.
+ * Errors: INVALID_ARG (d, slot, slots, n_dst out of range, NULL pointers), ALIGNMENT, CUDA.
+ */
+size_t ddd_shard_records_bytes(const ddd_config *cfg /* HOST */, int32_t slots);
+int ddd_shard_begin(ddd_handle *h, const void *root_hidden, const int32_t *root_token, const int32_t *root_pos,
+                    const ddd_output *out, const ddd_trace *trace, void *cuda_stream);
+int ddd_shard_lm_head(ddd_handle *h, int32_t d, int32_t slot, int32_t slots,
+                      void *const *records_dst /* HOST array of n_dst DEVICE pointers */,
+                      int32_t *const *flags_dst /* HOST array of n_dst DEVICE pointers, or NULL */,
+                      int32_t n_dst, void *cuda_stream);
+int ddd_shard_select(ddd_handle *h, int32_t d, const void *records /* DEVICE */, int32_t slots,
+                     const int32_t *flags /* DEVICE [slots] or NULL */, void *cuda_stream);
 
 /*
  * What the verification step needs from a finished tree.  With T = t_rows and L = max_depth + 1,

@@ -28,6 +28,7 @@ class DddConfig(ctypes.Structure):
         ("dtype", ctypes.c_int32), ("threshold", ctypes.c_float), ("check_mask", ctypes.c_uint32),
         ("logit_scale", ctypes.c_float), ("rms_eps", ctypes.c_float), ("plant_delta", ctypes.c_float),
         ("device", ctypes.c_int32), ("lm_head_kernel", ctypes.c_int32), ("launch_mode", ctypes.c_int32),
+        ("vocab_begin", ctypes.c_int32), ("vocab_count", ctypes.c_int32),
     ]
 
 
@@ -83,6 +84,16 @@ def load_library():
     lib.ddd_lm_head_topk_noalloc.restype = ctypes.c_int
     lib.ddd_lm_head_topk_noalloc.argtypes = [vp, vp, vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
                                              ctypes.c_int32, ctypes.c_int32, ctypes.c_float, vp, vp, vp, vp]
+    lib.ddd_shard_records_bytes.restype = ctypes.c_size_t
+    lib.ddd_shard_records_bytes.argtypes = [ctypes.POINTER(DddConfig), ctypes.c_int32]
+    lib.ddd_shard_begin.restype = ctypes.c_int
+    lib.ddd_shard_begin.argtypes = [vp, vp, i32p, i32p, ctypes.POINTER(DddOutput), ctypes.POINTER(DddTrace), vp]
+    lib.ddd_shard_lm_head.restype = ctypes.c_int
+    lib.ddd_shard_lm_head.argtypes = [vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
+                                      ctypes.POINTER(ctypes.c_void_p), ctypes.POINTER(ctypes.c_void_p),
+                                      ctypes.c_int32, vp]
+    lib.ddd_shard_select.restype = ctypes.c_int
+    lib.ddd_shard_select.argtypes = [vp, ctypes.c_int32, vp, ctypes.c_int32, vp, vp]
     lib.ddd_verify_greedy.restype = ctypes.c_int
     lib.ddd_verify_greedy.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, i32p, i32p, i32p, i32p,
                                       ctypes.POINTER(DddVerifyOutput), vp]
@@ -98,6 +109,7 @@ def exported_symbols():
     """Names this binding expects the library to export (all of include/ddd.h)."""
     return ["ddd_workspace_bytes", "ddd_create", "ddd_draft", "ddd_draft_host", "ddd_draft_host_gated", "ddd_lm_head_pass",
             "ddd_launches_per_draft", "ddd_lm_head_blocks", "ddd_lm_head_topk_noalloc", "ddd_verify_greedy",
+            "ddd_shard_records_bytes", "ddd_shard_begin", "ddd_shard_lm_head", "ddd_shard_select",
             "ddd_destroy", "ddd_strerror"]
 
 
@@ -183,6 +195,49 @@ def ddd_verify_greedy(batch: int, t_rows: int, max_depth: int, n_out: int, token
         raise DddError(rc, "ddd_verify_greedy")
 
 
+def ddd_shard_records_bytes(cfg: DddConfig, slots: int) -> int:
+    return int(load_library().ddd_shard_records_bytes(ctypes.byref(cfg), int(slots)))
+
+
+def ddd_shard_begin(handle: int, root_hidden: int, root_token: int, root_pos: int, out: DddOutput,
+                    trace: Optional[DddTrace], stream: int) -> None:
+    rc = load_library().ddd_shard_begin(handle, root_hidden, root_token, root_pos, ctypes.byref(out),
+                                        ctypes.byref(trace) if trace is not None else None, stream)
+    if rc != 0:
+        raise DddError(rc, "ddd_shard_begin")
+
+
+def ddd_shard_lm_head(handle: int, d: int, slot: int, slots: int, records_dst, flags_dst, stream: int) -> None:
+    """records_dst / flags_dst: sequences of device addresses, one per destination record set
+    (flags_dst may be None)."""
+    n = len(records_dst)
+    rec = (ctypes.c_void_p * n)(*records_dst)
+    flg = None if flags_dst is None else (ctypes.c_void_p * n)(*flags_dst)
+    rc = load_library().ddd_shard_lm_head(handle, d, slot, slots, rec, flg, n, stream)
+    if rc != 0:
+        raise DddError(rc, "ddd_shard_lm_head")
+
+
+def ddd_shard_select(handle: int, d: int, records: int, slots: int, flags: Optional[int], stream: int) -> None:
+    rc = load_library().ddd_shard_select(handle, d, records, slots, flags, stream)
+    if rc != 0:
+        raise DddError(rc, "ddd_shard_select")
+
+
+def vocab_slice(vocab: int, world: int, rank: int):
+    """(first token id, number of rows) of rank's slice of a vocabulary split over `world` ranks:
+    whole 32-row units (the granule the tensor-core kernel streams), as even as they go, the
+    ragged end with the last rank that has rows."""
+    if not (0 <= rank < world):
+        raise ValueError("rank out of range")
+    units = (vocab + 31) // 32
+    base, extra = divmod(units, world)
+    first = rank * base + min(rank, extra)
+    mine = base + (1 if rank < extra else 0)
+    begin = min(first * 32, vocab)
+    return begin, max(0, min((first + mine) * 32, vocab) - begin)
+
+
 def ddd_destroy(handle: int) -> None:
     rc = load_library().ddd_destroy(handle)
     if rc != 0:
@@ -195,7 +250,9 @@ class DraftEngine:
     and one set of output / trace tensors.  All computation happens inside the library."""
 
     def __init__(self, cfg, weights: Dict, device: int = 0, lm_head_kernel: int = DDD_LM_HEAD_AUTO,
-                 launch_mode: int = DDD_LAUNCH_STREAM, with_trace: bool = True):
+                 launch_mode: int = DDD_LAUNCH_STREAM, with_trace: bool = True, vocab_slice=None):
+        """vocab_slice = (begin, count): this engine owns only those rows of the LM head (one rank
+        of a vocabulary-parallel head); it then drafts through the shard_* methods."""
         import torch
         load_library()
         if not torch.cuda.is_available():
@@ -205,9 +262,13 @@ class DraftEngine:
         self.device = torch.device("cuda", device)
         self.dtype = torch.float32 if cfg.dtype == "fp32" else torch.bfloat16
         dev = self.device
-        self.W = weights["W"].to(dev, self.dtype).contiguous()
+        v_begin, v_count = vocab_slice if vocab_slice is not None else (0, 0)
+        if vocab_slice is not None and v_count < 1:
+            raise ValueError("an empty vocabulary slice cannot have a handle")
+        rows = slice(v_begin, v_begin + v_count) if v_count else slice(None)
+        self.W = weights["W"][rows].to(dev, self.dtype).contiguous()
         self.E = weights["E"].to(dev, self.dtype).contiguous()
-        self.bias = None if weights.get("bias") is None else weights["bias"].to(dev, torch.float32).contiguous()
+        self.bias = None if weights.get("bias") is None else weights["bias"][rows].to(dev, torch.float32).contiguous()
         pn = weights.get("plant_next")
         self.plant_next = None if pn is None else pn.to(dev, torch.int32).contiguous()
         self.c = DddConfig(
@@ -215,7 +276,7 @@ class DraftEngine:
             total_tokens=cfg.total_tokens, dtype=DDD_DTYPE_FP32 if cfg.dtype == "fp32" else DDD_DTYPE_BF16,
             threshold=max(cfg.threshold, -3.0e38), check_mask=cfg.check_mask & 0xFFFFFFFF,
             logit_scale=cfg.logit_scale, rms_eps=cfg.rms_eps, plant_delta=cfg.plant_delta, device=device,
-            lm_head_kernel=lm_head_kernel, launch_mode=launch_mode)
+            lm_head_kernel=lm_head_kernel, launch_mode=launch_mode, vocab_begin=v_begin, vocab_count=v_count)
         nbytes = ddd_workspace_bytes(self.c)
         if nbytes == 0:
             raise DddError(-1, "ddd_workspace_bytes")
@@ -302,6 +363,19 @@ class DraftEngine:
                           self.out["parent"].data_ptr(), target_argmax.data_ptr(), self.c_verify_out,
                           self.stream_ptr())
         return self.verify_out
+
+    def shard_begin(self, root_hidden, root_token, root_pos) -> None:
+        ddd_shard_begin(self.handle, root_hidden.data_ptr(), root_token.data_ptr(), root_pos.data_ptr(),
+                        self.c_out, self.c_trace, self.stream_ptr())
+
+    def shard_lm_head(self, d: int, slot: int, slots: int, records_dst, flags_dst=None) -> None:
+        """records_dst / flags_dst: device tensors (record sets and flag arrays) to publish into."""
+        ddd_shard_lm_head(self.handle, d, slot, slots, [t.data_ptr() for t in records_dst],
+                          None if flags_dst is None else [t.data_ptr() for t in flags_dst], self.stream_ptr())
+
+    def shard_select(self, d: int, records, slots: int, flags=None) -> None:
+        ddd_shard_select(self.handle, d, records.data_ptr(), slots,
+                         None if flags is None else flags.data_ptr(), self.stream_ptr())
 
     def lm_head_pass(self) -> None:
         ddd_lm_head_pass(self.handle, self.stream_ptr())

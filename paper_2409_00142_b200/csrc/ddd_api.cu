@@ -26,7 +26,7 @@ size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
   size_t hbuf[2], part_key, part_ms, tree_token, tree_parent, tree_cum, beam_node, beam_tok, beam_cum,
-      row_plant, active, stop_depth, root_pos, n_active, dev_status, lm_ticket, w_packed;
+      row_plant, active, stop_depth, root_pos, n_active, dev_status, lm_ticket, shard_counter, w_packed;
   // staging for ddd_draft_host: inputs, then the packed output block
   size_t in_hidden, in_token, in_pos, out_block;
   size_t o_n_out, o_stop, o_token, o_parent, o_depth, o_position, o_cum, o_mask, o_H, o_status, out_bytes;
@@ -50,6 +50,10 @@ int validate(const ddd_config* c) {
   if (c->device < 0) return DDD_ERR_INVALID_ARG;
   if (c->lm_head_kernel < DDD_LM_HEAD_AUTO || c->lm_head_kernel > DDD_LM_HEAD_TCGEN05) return DDD_ERR_INVALID_ARG;
   if (c->launch_mode < DDD_LAUNCH_STREAM || c->launch_mode > DDD_LAUNCH_PLAIN) return DDD_ERR_INVALID_ARG;
+  if (c->vocab_count == 0 ? c->vocab_begin != 0
+                          : (c->vocab_begin < 0 || c->vocab_count < 1 ||
+                             (long long)c->vocab_begin + c->vocab_count > c->vocab))
+    return DDD_ERR_INVALID_ARG;
   if (c->lm_head_kernel == DDD_LM_HEAD_TCGEN05 && (c->dtype != DDD_DTYPE_BF16 || c->hidden % 64 != 0))
     return DDD_ERR_UNSUPPORTED;
   return DDD_OK;
@@ -79,10 +83,11 @@ Layout make_layout(const ddd_config* c) {
   L.n_active = take(4);
   L.dev_status = take(4);
   L.lm_ticket = take(8);
+  L.shard_counter = take(8);
   // packed copy of W for the tensor-core kernel (kept 1024-byte aligned relative to the base)
   off = (off + 1023) / 1024 * 1024;
   const bool tc_possible = c->dtype == DDD_DTYPE_BF16 && c->hidden % 64 == 0 && c->lm_head_kernel != DDD_LM_HEAD_SIMT;
-  L.w_packed = take(tc_possible ? tc_packed_bytes(c->vocab, c->hidden) : 0);
+  L.w_packed = take(tc_possible ? tc_packed_bytes(c->vocab_count ? c->vocab_count : c->vocab, c->hidden) : 0);
   // host-variant staging: inputs packed back to back (each 16-byte aligned), one output block
   L.in_hidden = take(0);
   size_t in = 0;
@@ -145,6 +150,11 @@ struct ddd_handle {
   // pinned host bounce buffer for ddd_draft_host
   unsigned char* bounce;
   size_t bounce_bytes;
+  // vocabulary-parallel drafting: output pointers of the draft in progress, drafts begun so far
+  DraftIO shard_io;
+  bool shard_open;
+  int shard_epoch;
+  int* shard_counter;
 };
 
 namespace {
@@ -339,10 +349,15 @@ int ddd_create(const ddd_config* cfg, const void* W, const void* E, const float*
   h->host_stream = nullptr;
   h->bounce = nullptr;
   h->bounce_bytes = 0;
+  h->shard_open = false;
+  h->shard_epoch = 0;
+  h->shard_counter = reinterpret_cast<int*>(h->ws + L.shard_counter);
 
   Params& p = h->p;
   p.B = cfg->batch; p.Hd = cfg->hidden; p.V = cfg->vocab; p.k = cfg->k; p.n = cfg->max_depth;
   p.m = cfg->total_tokens; p.dtype = cfg->dtype;
+  p.Vl = cfg->vocab_count ? cfg->vocab_count : cfg->vocab;
+  p.v0 = cfg->vocab_count ? cfg->vocab_begin : 0;
   p.R = p.B * p.k;
   p.Nn = 1 + p.k + (p.n - 1) * p.k * p.k;
   p.T = p.m + 1;
@@ -380,7 +395,7 @@ int ddd_create(const ddd_config* cfg, const void* W, const void* E, const float*
     if (rc == DDD_OK) rc = tc_plan_create(p, h->sm_count, ws + L.w_packed, &h->tc);
     if (rc == DDD_OK) p.lm_ctas = h->tc.ctas;
   } else if (rc == DDD_OK) {
-    const int n_tiles = (p.V + kTile - 1) / kTile;
+    const int n_tiles = (p.Vl + kTile - 1) / kTile;
     int ctas = 2 * h->sm_count;
     if (ctas > n_tiles) ctas = n_tiles;
     if (ctas > kMaxLmCtas) ctas = kMaxLmCtas;
@@ -404,6 +419,7 @@ int ddd_draft(ddd_handle* h, const void* root_hidden, const int32_t* root_token,
       !out->cum || !out->mask || !out->H_trace || !out->status)
     return DDD_ERR_INVALID_ARG;
   if (!aligned16(root_hidden)) return DDD_ERR_ALIGNMENT;
+  if (h->cfg.vocab_count != 0) return DDD_ERR_INVALID_ARG;     // a slice cannot draft alone: ddd_shard_*
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   DraftIO io;
   io.out = *out;
@@ -443,6 +459,7 @@ int ddd_draft_host_gated(ddd_handle* h, const void* root_hidden, const int32_t* 
       !out->cum || !out->mask || !out->H_trace || !out->status)
     return DDD_ERR_INVALID_ARG;
   if (!aligned16(root_hidden)) return DDD_ERR_ALIGNMENT;
+  if (h->cfg.vocab_count != 0) return DDD_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   DraftIO io;
   io.out = *out;
@@ -471,6 +488,7 @@ int ddd_draft_host(ddd_handle* h, const void* root_hidden, const int32_t* root_t
   if (!out->n_out || !out->stop_depth || !out->token || !out->parent || !out->depth || !out->position ||
       !out->cum || !out->mask || !out->H_trace || !out->status)
     return DDD_ERR_INVALID_ARG;
+  if (h->cfg.vocab_count != 0) return DDD_ERR_INVALID_ARG;
   const Layout& L = h->L;
   const Params& p = h->p;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
@@ -542,6 +560,74 @@ int ddd_draft_host(ddd_handle* h, const void* root_hidden, const int32_t* root_t
   std::memcpy(out->H_trace, hb + L.o_H, B * p.n * 4);
   std::memcpy(out->status, hb + L.o_status, 4);
   return out->status[0];
+}
+
+size_t ddd_shard_records_bytes(const ddd_config* cfg, int32_t slots) {
+  if (validate(cfg) != DDD_OK || slots < 1 || slots > DDD_MAX_SHARDS) return 0;
+  const size_t R = (size_t)cfg->batch * cfg->k;
+  return (size_t)slots * R * ((size_t)cfg->k + 1) * 8;
+}
+
+int ddd_shard_begin(ddd_handle* h, const void* root_hidden, const int32_t* root_token, const int32_t* root_pos,
+                    const ddd_output* out, const ddd_trace* trace, void* cuda_stream) {
+  if (!h || !root_hidden || !root_token || !root_pos || !out) return DDD_ERR_INVALID_ARG;
+  if (!out->n_out || !out->stop_depth || !out->token || !out->parent || !out->depth || !out->position ||
+      !out->cum || !out->mask || !out->H_trace || !out->status)
+    return DDD_ERR_INVALID_ARG;
+  if (!aligned16(root_hidden)) return DDD_ERR_ALIGNMENT;
+  h->shard_io.out = *out;
+  if (trace) h->shard_io.trace = *trace; else std::memset(&h->shard_io.trace, 0, sizeof h->shard_io.trace);
+  if (launch_init(h->p, h->shard_io, root_hidden, root_token, root_pos, static_cast<cudaStream_t>(cuda_stream)) !=
+      cudaSuccess) {
+    note_cuda_error(__LINE__);
+    return DDD_ERR_CUDA;
+  }
+  h->shard_open = true;
+  h->shard_epoch = (h->shard_epoch + 1) & 0xFFFFFF;
+  return DDD_OK;
+}
+
+static int shard_flag_value(const ddd_handle* h, int d) { return h->shard_epoch * (DDD_MAX_DEPTH + 1) + d; }
+
+int ddd_shard_lm_head(ddd_handle* h, int32_t d, int32_t slot, int32_t slots, void* const* records_dst,
+                      int32_t* const* flags_dst, int32_t n_dst, void* cuda_stream) {
+  if (!h || !h->shard_open || !records_dst) return DDD_ERR_INVALID_ARG;
+  if (d < 1 || d > h->p.n || slots < 1 || slots > DDD_MAX_SHARDS || slot < 0 || slot >= slots) return DDD_ERR_INVALID_ARG;
+  if (n_dst < 1 || n_dst > DDD_MAX_SHARDS) return DDD_ERR_INVALID_ARG;
+  for (int i = 0; i < n_dst; ++i) {
+    if (!records_dst[i] || (flags_dst && !flags_dst[i])) return DDD_ERR_INVALID_ARG;
+    if (!aligned16(records_dst[i])) return DDD_ERR_ALIGNMENT;
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (launch_lm_head(h, d, 0, false, st) != cudaSuccess ||
+      launch_shard_reduce(h->p, d, slot, slots, records_dst, flags_dst, n_dst, shard_flag_value(h, d),
+                          h->shard_counter, st) != cudaSuccess) {
+    note_cuda_error(__LINE__);
+    return DDD_ERR_CUDA;
+  }
+  return DDD_OK;
+}
+
+int ddd_shard_select(ddd_handle* h, int32_t d, const void* records, int32_t slots, const int32_t* flags,
+                     void* cuda_stream) {
+  if (!h || !h->shard_open || !records) return DDD_ERR_INVALID_ARG;
+  if (d < 1 || d > h->p.n || slots < 1 || slots > DDD_MAX_SHARDS) return DDD_ERR_INVALID_ARG;
+  if (!aligned16(records)) return DDD_ERR_ALIGNMENT;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  cudaError_t e = cudaSuccess;
+  if (flags) e = launch_shard_wait(flags, slots, shard_flag_value(h, d), h->p.dev_status, st);
+  // the select kernel merges `slots` partials per row from the record set instead of one per thread block
+  Params q = h->p;
+  unsigned char* base = static_cast<unsigned char*>(const_cast<void*>(records));
+  q.part_key = reinterpret_cast<unsigned long long*>(base);
+  q.part_ms = reinterpret_cast<float2*>(base + (size_t)slots * q.R * q.k * sizeof(unsigned long long));
+  q.lm_ctas = slots;
+  if (e == cudaSuccess) e = launch_select(q, h->shard_io, d, false, 0, false, st);
+  if (e != cudaSuccess) {
+    note_cuda_error(__LINE__);
+    return DDD_ERR_CUDA;
+  }
+  return DDD_OK;
 }
 
 int ddd_lm_head_pass(ddd_handle* h, void* cuda_stream) {

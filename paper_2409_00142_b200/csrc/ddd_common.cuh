@@ -18,6 +18,8 @@ constexpr unsigned kFullMask = 0xFFFFFFFFu;
 // Everything a kernel needs that does not change between drafts.
 struct Params {
   int B, Hd, V, k, n, m, dtype;
+  int Vl, v0;         // rows of W this handle streams and the token id of its first row (V, 0 unless
+                      // the handle owns a slice of a vocabulary-parallel LM head)
   int R;              // B * k beam rows
   int Nn;             // node slots per sequence: 1 + k + (n-1) k^2
   int T, W32;         // output rows per sequence (m + 1) and mask words per row
@@ -315,5 +317,12 @@ cudaError_t launch_lm_head_simt(const Params& p, int d, int force_all, int ctas,
 // set_cond: a sequence that continues after pass d sets the graph conditional `cond` to 1.
 cudaError_t launch_select(const Params& p, const DraftIO& io, int d, bool pdl, cudaGraphConditionalHandle cond,
                           bool set_cond, cudaStream_t st);
+
+// Vocabulary-parallel pieces (shard.cu): fold this rank's per-block partials of pass d into one
+// record per row, stored into slot `slot` of each of the n_dst record sets (flags raised beside
+// them if given); wait for the flags of all slots.
+cudaError_t launch_shard_reduce(const Params& p, int d, int slot, int slots, void* const* records,
+                                int32_t* const* flags, int n_dst, int flag_value, int* done_counter, cudaStream_t st);
+cudaError_t launch_shard_wait(const int* flags, int slots, int flag_value, int* dev_status, cudaStream_t st);
 
 }  // namespace ddd

@@ -54,7 +54,7 @@ __global__ void __launch_bounds__(kThreads) lm_head_simt_kernel(const Params p, 
   constexpr int VEC = Vec<T>::N;
   const T* W = static_cast<const T*>(p.W);
   const T* H = static_cast<const T*>(p.hbuf[(d - 1) & 1]);
-  const int n_tiles = (p.V + kTile - 1) / kTile;
+  const int n_tiles = (p.Vl + kTile - 1) / kTile;   // W, bias: local rows; tokens: v0 + local row
 
   for (int r = warp; r < p.R; r += kWarps) {
     for (int e = lane; e < kst; e += 32) st_key[r * kst + e] = 0ull;
@@ -67,7 +67,7 @@ __global__ void __launch_bounds__(kThreads) lm_head_simt_kernel(const Params p, 
     // ---- logits of this tile
     for (int vl = warp; vl < kTile; vl += kWarps) {
       const int v = v0 + vl;
-      const bool v_ok = v < p.V;
+      const bool v_ok = v < p.Vl;
       const float bias = (v_ok && p.bias) ? p.bias[v] : 0.f;
       for (int r0 = 0; r0 < p.R; r0 += kRowChunk) {
         float acc[kRowChunk];
@@ -101,7 +101,7 @@ __global__ void __launch_bounds__(kThreads) lm_head_simt_kernel(const Params p, 
           if (lane == rc) {
             const int r = r0 + rc;
             float z = neg_inf();
-            if (v_ok && live[rc] && p.row_plant[r] != v) z = fmaf(sum, p.s, bias);
+            if (v_ok && live[rc] && p.row_plant[r] != v + p.v0) z = fmaf(sum, p.s, bias);
             zt[(size_t)r * kTile + vl] = z;
           }
         }
@@ -114,12 +114,12 @@ __global__ void __launch_bounds__(kThreads) lm_head_simt_kernel(const Params p, 
       float2 ms = st_ms[r];
       if (p.k <= kNarrowK) {
         unsigned long long key = st_key[r * 32 + lane];
-        row_tile_update(zt + (size_t)r * kTile, v0, p.k, ms.x, ms.y, key);
+        row_tile_update(zt + (size_t)r * kTile, v0 + p.v0, p.k, ms.x, ms.y, key);
         st_key[r * 32 + lane] = key;
       } else {
         unsigned long long list[4];
         wide_load(list, st_key + (size_t)r * kWideK, kWideK);
-        row_tile_update_wide(zt + (size_t)r * kTile, v0, p.k, ms.x, ms.y, list);
+        row_tile_update_wide(zt + (size_t)r * kTile, v0 + p.v0, p.k, ms.x, ms.y, list);
         wide_store(list, st_key + (size_t)r * kWideK, kWideK);
       }
       if (lane == 0) st_ms[r] = ms;

@@ -248,7 +248,7 @@ lm_head_tc_kernel(const Params p, const unsigned char* __restrict__ w_packed,
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   // this block's contiguous range of 32-row units
-  const int n_units = (p.V + kUnitRows - 1) / kUnitRows;
+  const int n_units = (p.Vl + kUnitRows - 1) / kUnitRows;    // W, bias: local rows; tokens: v0 + local row
   const int base_units = n_units / (int)gridDim.x, rem_units = n_units % (int)gridDim.x;
   // Vocab ranges are handed out in arrival order: the larger ranges go to the blocks that
   // start first, and the blocks that could only start after the previous select kernel left
@@ -444,7 +444,7 @@ lm_head_tc_kernel(const Params p, const unsigned char* __restrict__ w_packed,
       tc_fence_after();
       const int vrow = quarter * 32 + lane;
       const int v = row0 + vrow;
-      const bool v_ok = vrow < rows && v < p.V;
+      const bool v_ok = vrow < rows && v < p.Vl;
       const float bias = (v_ok && p.bias) ? p.bias[v] : 0.f;
       for (int g0 = 0; g0 < n_chunks; g0 += cpg) {
         const int ch = g0 + lw;
@@ -456,7 +456,7 @@ lm_head_tc_kernel(const Params p, const unsigned char* __restrict__ w_packed,
           for (int c = 0; c < kChunkCols; ++c) {
             const int r = c0 + c;
             float z = neg_inf();
-            if (v_ok && r < p.R && s_plant[r] != v) z = fmaf(accv[c], p.s, bias);
+            if (v_ok && r < p.R && s_plant[r] != v + p.v0) z = fmaf(accv[c], p.s, bias);
             zt[(lw * kChunkCols + c) * kTile + vrow] = z;
           }
           tc_fence_before();
@@ -472,12 +472,12 @@ lm_head_tc_kernel(const Params p, const unsigned char* __restrict__ w_packed,
           float2 ms = st_ms[r];
           if (p.k <= kNarrowK) {
             unsigned long long key = lane < p.k ? st_key[r * p.k + lane] : 0ull;
-            row_tile_update(zt + rr * kTile, row0, p.k, ms.x, ms.y, key);
+            row_tile_update(zt + rr * kTile, row0 + p.v0, p.k, ms.x, ms.y, key);
             if (lane < p.k) st_key[r * p.k + lane] = key;
           } else {
             unsigned long long list[4];
             wide_load(list, st_key + r * kst, kst);
-            row_tile_update_wide(zt + rr * kTile, row0, p.k, ms.x, ms.y, list);
+            row_tile_update_wide(zt + rr * kTile, row0 + p.v0, p.k, ms.x, ms.y, list);
             wide_store(list, st_key + r * kst, kst);
           }
           if (lane == 0) st_ms[r] = ms;
@@ -575,7 +575,7 @@ int tc_plan_create(const Params& p, int sm_count, void* w_packed, TcPlan* plan) 
   int cols = 32;
   while (cols < 2 * n_pad) cols *= 2;
   if (cols > 512) return DDD_ERR_UNSUPPORTED;
-  const int n_units = (p.V + kUnitRows - 1) / kUnitRows;
+  const int n_units = (p.Vl + kUnitRows - 1) / kUnitRows;
   int ctas = sm_count < n_units ? sm_count : n_units;
   if (ctas > kMaxLmCtas) ctas = kMaxLmCtas;
   // K-blocks per stage: as many as still leave a ring of two stages, at most 4.  A pipeline step
@@ -607,8 +607,8 @@ int tc_plan_create(const Params& p, int sm_count, void* w_packed, TcPlan* plan) 
   plan->smem = (size_t)smem_plan(stages, ksub, n_pad, p.R, p.k, cpg).total + 1024;
   plan->w_packed = static_cast<unsigned char*>(w_packed);
   {
-    const size_t chunks = tc_packed_bytes(p.V, p.Hd) / kUnitBytes;
-    pack_w_kernel<<<(unsigned)chunks, 256>>>(static_cast<const __nv_bfloat16*>(p.W), plan->w_packed, p.V, p.Hd,
+    const size_t chunks = tc_packed_bytes(p.Vl, p.Hd) / kUnitBytes;
+    pack_w_kernel<<<(unsigned)chunks, 256>>>(static_cast<const __nv_bfloat16*>(p.W), plan->w_packed, p.Vl, p.Hd,
                                              n_units);
     if (cudaGetLastError() != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) return DDD_ERR_CUDA;
   }

@@ -65,6 +65,28 @@ __device__ __forceinline__ unsigned long long merge_row_heads(int k, int nc, con
 }
 
 
+// Blocks that work on wide lists (ddd_common.cuh) have 16 warps.
+constexpr int kWideThreads = 512;
+constexpr int kWideWarps = kWideThreads / 32;
+
+// Tree of pairwise merges over the warps' lists in buf [kWideWarps][kWideK]; the result ends up
+// in warp 0's registers (and in buf[0]).  All threads of the block call this.
+__device__ __forceinline__ void block_merge_lists(unsigned long long (&acc)[4], unsigned long long* buf) {
+  const int warp = threadIdx.x >> 5;
+  wide_store(acc, buf + warp * kWideK, kWideK);
+  __syncthreads();
+  for (int half = kWideWarps / 2; half >= 1; half >>= 1) {
+    if (warp < half) {
+      unsigned long long other[4];
+      wide_load(other, buf + (warp + half) * kWideK, kWideK);
+      wide_merge(acc, other);
+      wide_store(acc, buf + warp * kWideK, kWideK);
+    }
+    __syncthreads();
+  }
+}
+
+
 // 8 (bf16) or 4 (fp32) consecutive elements of h_parent + E[token], formed in fp64.
 template <typename T>
 struct Chunk;

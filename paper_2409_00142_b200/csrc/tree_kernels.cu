@@ -496,26 +496,6 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
 // per lane, ddd_common.cuh), and every choice is a merge of sorted lists: the warps of a block
 // each fold a share of the lists into one, the 16 results meet in shared memory and are merged
 // pairwise in four rounds.
-constexpr int kWideThreads = 512;
-constexpr int kWideWarps = kWideThreads / 32;
-
-// Tree of pairwise merges over the warps' lists in buf [kWideWarps][kWideK]; the result ends up
-// in warp 0's registers (and in buf[0]).  All threads of the block call this.
-__device__ __forceinline__ void block_merge_lists(unsigned long long (&acc)[4], unsigned long long* buf) {
-  const int warp = threadIdx.x >> 5;
-  wide_store(acc, buf + warp * kWideK, kWideK);
-  __syncthreads();
-  for (int half = kWideWarps / 2; half >= 1; half >>= 1) {
-    if (warp < half) {
-      unsigned long long other[4];
-      wide_load(other, buf + (warp + half) * kWideK, kWideK);
-      wide_merge(acc, other);
-      wide_store(acc, buf + warp * kWideK, kWideK);
-    }
-    __syncthreads();
-  }
-}
-
 // Dynamic shared memory: candidate records [k*k], merge buffers [16][128], partial sums of squares
 // of the draft step [k][slots]; after a stop the same memory serves the rerank.
 __global__ void __launch_bounds__(kWideThreads) select_gate_step_wide_kernel(const Params p, const DraftIO io,
