@@ -69,8 +69,13 @@ enum { DDD_LM_HEAD_AUTO = 0, DDD_LM_HEAD_SIMT = 1, DDD_LM_HEAD_TCGEN05 = 2 };
  * but the first sits behind a conditional node that only a still-drafting sequence switches
  * on, so that a draft that stops early launches little that has nothing to do.  PLAIN launches
  * kernel by kernel in ordinary stream order, one after the other: the slowest, and the one
- * profilers can follow. */
-enum { DDD_LAUNCH_STREAM = 0, DDD_LAUNCH_GRAPH = 1, DDD_LAUNCH_PLAIN = 2 };
+ * profilers can follow.  FUSED runs the whole draft as ONE persistent kernel of one thread block
+ * per SM (a cooperative launch) that loops over the passes itself and hands over between them
+ * through counters in global memory, followed by one small kernel for the rerank and the mask:
+ * the fastest, for bf16 handles on the tensor-core kernel with a beam of at most 32
+ * (ddd_create returns DDD_ERR_UNSUPPORTED otherwise); nothing else should run on the device
+ * meanwhile, since its blocks occupy every SM until the draft ends. */
+enum { DDD_LAUNCH_STREAM = 0, DDD_LAUNCH_GRAPH = 1, DDD_LAUNCH_PLAIN = 2, DDD_LAUNCH_FUSED = 3 };
 
 #define DDD_MAX_K 128         /* beam width limit (the paper's appendix table goes to 100) */
 #define DDD_MAX_DEPTH 32      /* check_mask has one bit per step                   */

@@ -12,7 +12,7 @@ _lib = None
 
 DDD_DTYPE_FP32, DDD_DTYPE_BF16 = 0, 1
 DDD_LM_HEAD_AUTO, DDD_LM_HEAD_SIMT, DDD_LM_HEAD_TCGEN05 = 0, 1, 2
-DDD_LAUNCH_STREAM, DDD_LAUNCH_GRAPH, DDD_LAUNCH_PLAIN = 0, 1, 2
+DDD_LAUNCH_STREAM, DDD_LAUNCH_GRAPH, DDD_LAUNCH_PLAIN, DDD_LAUNCH_FUSED = 0, 1, 2, 3
 
 
 class DddError(RuntimeError):

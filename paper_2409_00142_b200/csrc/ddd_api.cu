@@ -8,6 +8,7 @@
 #include <new>
 
 #include "ddd_common.cuh"
+#include "draft_fused.cuh"
 #include "lm_head_tc.cuh"
 
 using namespace ddd;
@@ -26,7 +27,8 @@ size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
   size_t hbuf[2], part_key, part_ms, tree_token, tree_parent, tree_cum, beam_node, beam_tok, beam_cum,
-      row_plant, active, stop_depth, root_pos, n_active, dev_status, lm_ticket, shard_counter, w_packed;
+      row_plant, active, stop_depth, root_pos, n_active, dev_status, lm_ticket, shard_counter, fused_sync,
+      fused_beam_cum, fused_beam_node, fused_row_plant, w_packed;
   // staging for ddd_draft_host: inputs, then the packed output block
   size_t in_hidden, in_token, in_pos, out_block;
   size_t o_n_out, o_stop, o_token, o_parent, o_depth, o_position, o_cum, o_mask, o_H, o_status, out_bytes;
@@ -49,7 +51,7 @@ int validate(const ddd_config* c) {
   if (!(c->rms_eps >= 0.f)) return DDD_ERR_INVALID_ARG;
   if (c->device < 0) return DDD_ERR_INVALID_ARG;
   if (c->lm_head_kernel < DDD_LM_HEAD_AUTO || c->lm_head_kernel > DDD_LM_HEAD_TCGEN05) return DDD_ERR_INVALID_ARG;
-  if (c->launch_mode < DDD_LAUNCH_STREAM || c->launch_mode > DDD_LAUNCH_PLAIN) return DDD_ERR_INVALID_ARG;
+  if (c->launch_mode < DDD_LAUNCH_STREAM || c->launch_mode > DDD_LAUNCH_FUSED) return DDD_ERR_INVALID_ARG;
   if (c->vocab_count == 0 ? c->vocab_begin != 0
                           : (c->vocab_begin < 0 || c->vocab_count < 1 ||
                              (long long)c->vocab_begin + c->vocab_count > c->vocab))
@@ -84,6 +86,10 @@ Layout make_layout(const ddd_config* c) {
   L.dev_status = take(4);
   L.lm_ticket = take(8);
   L.shard_counter = take(8);
+  L.fused_sync = take(16);
+  L.fused_beam_cum = take(2 * R * 4);
+  L.fused_beam_node = take(2 * R * 4);
+  L.fused_row_plant = take(2 * R * 4);
   // packed copy of W for the tensor-core kernel (kept 1024-byte aligned relative to the base)
   off = (off + 1023) / 1024 * 1024;
   const bool tc_possible = c->dtype == DDD_DTYPE_BF16 && c->hidden % 64 == 0 && c->lm_head_kernel != DDD_LM_HEAD_SIMT;
@@ -392,8 +398,13 @@ int ddd_create(const ddd_config* cfg, const void* W, const void* E, const float*
     h->lm_kind = (cfg->dtype == DDD_DTYPE_BF16 && cfg->hidden % 64 == 0) ? DDD_LM_HEAD_TCGEN05 : DDD_LM_HEAD_SIMT;
   if (rc == DDD_OK && h->lm_kind == DDD_LM_HEAD_TCGEN05) {
     if (prop.major != 10) rc = DDD_ERR_UNSUPPORTED;
-    if (rc == DDD_OK) rc = tc_plan_create(p, h->sm_count, ws + L.w_packed, &h->tc);
+    const bool fused = cfg->launch_mode == DDD_LAUNCH_FUSED;
+    if (rc == DDD_OK && fused && cfg->k > 32) rc = DDD_ERR_UNSUPPORTED;
+    if (rc == DDD_OK) rc = tc_plan_create(p, h->sm_count, ws + L.w_packed, &h->tc, fused ? fused_extra_smem(cfg->k) : 0);
     if (rc == DDD_OK) p.lm_ctas = h->tc.ctas;
+    if (rc == DDD_OK && fused) rc = fused_prepare(p, h->tc);
+  } else if (rc == DDD_OK && cfg->launch_mode == DDD_LAUNCH_FUSED) {
+    rc = DDD_ERR_UNSUPPORTED;            // the one-kernel draft is built on the tensor-core LM head
   } else if (rc == DDD_OK) {
     const int n_tiles = (p.Vl + kTile - 1) / kTile;
     int ctas = 2 * h->sm_count;
@@ -425,6 +436,22 @@ int ddd_draft(ddd_handle* h, const void* root_hidden, const int32_t* root_token,
   io.out = *out;
   if (trace) io.trace = *trace; else std::memset(&io.trace, 0, sizeof io.trace);
 
+  if (h->cfg.launch_mode == DDD_LAUNCH_FUSED) {
+    FusedArgs fa = {};
+    fa.root_hidden = root_hidden;
+    fa.root_token = root_token;
+    fa.root_pos = root_pos;
+    fa.io = io;
+    fa.beam_cum = reinterpret_cast<float*>(h->ws + h->L.fused_beam_cum);
+    fa.beam_node = reinterpret_cast<int*>(h->ws + h->L.fused_beam_node);
+    fa.row_plant = reinterpret_cast<int*>(h->ws + h->L.fused_row_plant);
+    fa.sync = reinterpret_cast<int*>(h->ws + h->L.fused_sync);
+    if (launch_draft_fused(h->p, h->tc, fa, st) != cudaSuccess) {
+      note_cuda_error(__LINE__);
+      return DDD_ERR_CUDA;
+    }
+    return DDD_OK;
+  }
   if (h->cfg.launch_mode == DDD_LAUNCH_GRAPH && st != nullptr) {
     GraphKey key;
     std::memset(&key, 0, sizeof key);
@@ -644,6 +671,7 @@ int ddd_launches_per_draft(const ddd_handle* h, int32_t passes_needed) {
   if (!h) return DDD_ERR_INVALID_ARG;
   const int n = h->p.n;
   int passes = n;
+  if (h->cfg.launch_mode == DDD_LAUNCH_FUSED) return 2;     // the draft kernel and the rerank kernel
   if (h->cfg.launch_mode == DDD_LAUNCH_GRAPH) {
     const int nb = h->have_graph ? h->graph_bounds : h->n_bounds;
     for (int j = nb - 1; j >= 0; --j)

@@ -1,0 +1,771 @@
+// One persistent kernel per draft (launch mode DDD_LAUNCH_FUSED).
+//
+// Every pass of Algorithm 1 - LM head, log-softmax statistics, per-row top-k, merge, beam choice,
+// Eq. 1 and the gate, draft step - runs inside ONE cooperative launch of one thread block per SM.
+// The blocks never leave between passes, so the two kernel boundaries per pass of the other launch
+// modes become two grid-wide hand-overs through counters in global memory, and a draft that
+// stops after d passes has launched nothing for the passes it does not run:
+//
+//   warp 0      producer: streams this block's vocabulary range of the packed W through the
+//               shared-memory ring, pass after pass without a break; the W of the next pass goes
+//               into the ring while the tree work of this pass is still going on, only the hidden
+//               rows wait for it
+//   warp 1      issues tcgen05.mma into two tensor-memory accumulators
+//   warps 2-17  epilogue of every tile (scale, bias, online max / sum-exp, running top-k), then
+//               the tree work of the pass
+//
+// Tree work of pass d.  Once every block has published its partials (hand-over 1), the new beam
+// row i of sequence b belongs to block (b k + i) mod G.  Each of those blocks merges the partial
+// lists of the sequence's rows and picks the new beam by itself - the same inputs give the same
+// result everywhere, which saves a hand-over - and then runs the draft step of its own row: 512
+// threads, one 16-byte chunk each, fp64, one rounding.  The block of row 0 also keeps the books
+// (tree nodes, beam state, trace, stop).  Blocks without a row go straight to hand-over 2, after
+// which the producers fetch the new hidden rows and the next pass runs.  The beam state is kept
+// twice, by pass parity: a block may still read the old beam while the book-keeper writes the new.
+// The rerank and the mask run in a small kernel of their own afterwards.
+//
+// Every wait is bounded.  A wait that runs out records DDD_ERR_TIMEOUT, raises a grid-wide abort
+// word that ends every other wait, and each block drains its copies, frees its tensor memory and
+// returns; the last block out resets the counters.
+#include "draft_fused.cuh"
+#include "tc_ptx.cuh"
+#include "tree_device.cuh"
+
+namespace ddd {
+
+namespace {
+
+using namespace tc;
+
+constexpr int kListDepth = 8;     // keys of a partial list a lane keeps in registers during a merge
+
+struct TreeSmem {
+  int cand, lse, sel_flat, sel_tok, sel_cum, red, misc, bar, total;
+};
+__host__ __device__ inline TreeSmem tree_smem(int k) {
+  TreeSmem t;
+  int off = 0;
+  t.cand = off; off += k * k * 8;            // candidate records of one sequence
+  t.lse = off; off += kNarrowK * 4;
+  t.sel_flat = off; off += kNarrowK * 4;
+  t.sel_tok = off; off += kNarrowK * 4;
+  t.sel_cum = off; off += kNarrowK * 4;
+  off = (off + 7) / 8 * 8;
+  t.red = off; off += 64 * 8;                // partial sums of squares of one row
+  t.misc = off; off += 16;                   // stop flag, H
+  t.bar = off; off += 8;                     // spare mbarrier (end of the MMAs on a give-up)
+  t.total = off;
+  return t;
+}
+
+__device__ __forceinline__ int ld_acquire(const int* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.b32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ int ld_relaxed(const int* p) {
+  int v;
+  asm volatile("ld.relaxed.gpu.global.b32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+
+// Waits until *counter >= target (every block adds one per hand-over; the counters only grow
+// during a draft).  False if the wait ran out or another block gave up.
+__device__ __forceinline__ bool grid_wait(const int* counter, int target, int* abort_word, int* status) {
+  unsigned long long t0 = 0;
+  for (uint32_t it = 0;; ++it) {
+    if (ld_acquire(counter) >= target) return true;
+    if ((it & 15u) == 15u) {
+      if (ld_relaxed(abort_word) != 0) return false;
+      const unsigned long long now = global_timer();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > kWaitLimitNs) {
+        atomicCAS(status, DDD_OK, DDD_ERR_TIMEOUT);
+        atomicExch(abort_word, 1);
+        return false;
+      }
+    }
+  }
+}
+// One arrival of this block at a hand-over: the caller has synchronised the threads whose writes
+// the other blocks are to see.
+__device__ __forceinline__ void grid_arrive(int* counter) {
+  asm volatile("fence.proxy.async;" ::: "memory");     // the hidden rows are read by tensor copies elsewhere
+  __threadfence();
+  atomicAdd(counter, 1);
+}
+
+// Merge of one beam row's partial lists (part_key [nc][R][k], sorted descending) by one warp,
+// straight from global memory: the k lists with the best heads are the only ones that can
+// contribute; lane j walks the j-th of them with its next kListDepth keys in registers.  Lane j
+// returns the j-th best key, and (M, S) = the row's merged max and sum-exp (all lanes).
+constexpr int kFusedMaxCtas = 160;     // partial lists per row the merge keeps heads of (five per lane)
+
+__device__ __forceinline__ unsigned long long merge_row_global(const Params& p, int r, float& M, float& S) {
+  const int lane = threadIdx.x & 31;
+  const int k = p.k, nc = p.lm_ctas, R = p.R;
+  constexpr int NL = kFusedMaxCtas / 32;
+  // heads and (max, sum-exp) of every block: one round trip
+  unsigned long long best_left[NL];
+  float2 ms[NL];
+#pragma unroll
+  for (int q = 0; q < NL; ++q) {
+    const int c = lane + 32 * q;
+    best_left[q] = 0ull;
+    ms[q] = make_float2(neg_inf(), 0.f);
+    if (c < nc) {
+      best_left[q] = p.part_key[((size_t)c * R + r) * k];
+      ms[q] = p.part_ms[(size_t)c * R + r];
+    }
+  }
+  M = neg_inf();
+#pragma unroll
+  for (int q = 0; q < NL; ++q) M = fmaxf(M, ms[q].x);
+  M = ordered_to_float(__reduce_max_sync(kFullMask, float_to_ordered(M)));
+  S = 0.f;
+#pragma unroll
+  for (int q = 0; q < NL; ++q)
+    if (ms[q].y > 0.f) S += ms[q].y * expf(ms[q].x - M);
+  S = warp_sum(S);
+  // the k best heads: lane j takes the block that owns the j-th best
+  int my_c = -1;
+  for (int j = 0; j < k; ++j) {
+    unsigned long long best = 0ull;
+    int best_q = 0;
+#pragma unroll
+    for (int q = 0; q < NL; ++q)
+      if (best_left[q] > best) { best = best_left[q]; best_q = q; }
+    const unsigned long long wk = warp_max_key(best);
+    if (wk == 0ull) break;
+    const bool mine = best == wk;              // keys are unique: one lane
+    const int src = __ffs(__ballot_sync(kFullMask, mine)) - 1;
+    const int win_c = __shfl_sync(kFullMask, lane + 32 * best_q, src);
+    if (mine) {
+#pragma unroll
+      for (int q = 0; q < NL; ++q)
+        if (q == best_q) best_left[q] = 0ull;
+    }
+    if (lane == j) my_c = win_c;
+  }
+  // lane j's list: the first kListDepth keys in registers, refilled from global memory as it is consumed
+  const unsigned long long* list = my_c >= 0 ? p.part_key + ((size_t)my_c * R + r) * k : nullptr;
+  unsigned long long lk[kListDepth];
+#pragma unroll
+  for (int i = 0; i < kListDepth; ++i) lk[i] = (list && i < k) ? list[i] : 0ull;
+  int next = kListDepth;
+  unsigned long long res = 0ull;
+  for (int j = 0; j < k; ++j) {
+    const unsigned long long wk = warp_max_key(lk[0]);
+    if (wk == 0ull) break;
+    if (lane == j) res = wk;
+    if (lk[0] == wk) {
+#pragma unroll
+      for (int i = 0; i + 1 < kListDepth; ++i) lk[i] = lk[i + 1];
+      lk[kListDepth - 1] = (list && next < k) ? list[next] : 0ull;
+      ++next;
+    }
+  }
+  return res;
+}
+
+// ---------------------------------------------------------------------------- kernel
+__global__ void __launch_bounds__(kTcThreads, 1)
+draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ CUtensorMap map_h0,
+                   const __grid_constant__ CUtensorMap map_h1) {
+  extern __shared__ unsigned char smem_dyn[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>(
+      (reinterpret_cast<uintptr_t>(smem_dyn) + 1023u) & ~static_cast<uintptr_t>(1023u));
+  const int stages = fa.stages, ksub = fa.ksub, n_pad = fa.n_pad, cpg = fa.cpg;
+  const SmemPlan sp = smem_plan(stages, ksub, n_pad, p.R, p.k, cpg);
+  const TreeSmem ts = tree_smem(p.k);
+  unsigned char* tree_base = smem + ((sp.total + 7) / 8 * 8);
+  float* zt = reinterpret_cast<float*>(smem + sp.zt);
+  unsigned long long* st_key = reinterpret_cast<unsigned long long*>(smem + sp.key);
+  float2* st_ms = reinterpret_cast<float2*>(smem + sp.ms);
+  int* s_plant = reinterpret_cast<int*>(smem + sp.plant);
+  int* s_live = reinterpret_cast<int*>(smem + sp.live);
+  unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + sp.bars);
+  uint32_t* tmem_ptr = reinterpret_cast<uint32_t*>(smem + sp.tmem_ptr);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + sp.abort_flag);
+  unsigned long long* cand_s = reinterpret_cast<unsigned long long*>(tree_base + ts.cand);
+  float* lse_s = reinterpret_cast<float*>(tree_base + ts.lse);
+  int* sel_flat = reinterpret_cast<int*>(tree_base + ts.sel_flat);
+  int* sel_tok = reinterpret_cast<int*>(tree_base + ts.sel_tok);
+  float* sel_cum = reinterpret_cast<float*>(tree_base + ts.sel_cum);
+  double* red_s = reinterpret_cast<double*>(tree_base + ts.red);
+  volatile int* s_misc = reinterpret_cast<volatile int*>(tree_base + ts.misc);    // [0] stop, [1] H bits
+  __shared__ int s_pass_state[2];      // what the producer learnt at hand-over 2: pass number to run, or 0 = leave
+
+  const uint32_t a_base = smem_u32(smem + sp.a), b_base = smem_u32(smem + sp.b);
+  const uint32_t b_bytes = (uint32_t)n_pad * kBlockK * 2;
+  const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8u * stages;
+  const uint32_t bar_tfull = bar_empty + 8u * stages, bar_tempty = bar_tfull + 16u;
+  const uint32_t bar_pass = bar_tempty + 16u;      // the plan's fifth word: "the producer knows how the draft goes on"
+  const uint32_t bar_spare = smem_u32(tree_base + ts.bar);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int G = (int)gridDim.x, bid = (int)blockIdx.x;
+  const int k = p.k, R = p.R;
+  int* const cnt_partials = fa.sync + 0;     // hand-over 1: partials of a pass published
+  int* const cnt_hidden = fa.sync + 1;       // hand-over 2: state and hidden rows of the next pass written
+  int* const abort_word = fa.sync + 2;
+  int* const exit_ticket = fa.sync + 3;
+
+  // this block's contiguous range of 32-row units (fixed: block i always covers the same rows)
+  const int n_units = (p.Vl + kUnitRows - 1) / kUnitRows;
+  const int base_units = n_units / G, rem_units = n_units % G;
+  const int my_units = base_units + (bid < rem_units ? 1 : 0);
+  const int unit0 = bid * base_units + (bid < rem_units ? bid : rem_units);
+  const int n_tiles = (my_units + 3) / 4;
+  const int num_kb = p.Hd / (kBlockK * ksub);
+  const uint32_t a_stage = (uint32_t)ksub * kABytes, b_stage = (uint32_t)ksub * b_bytes;
+  const int total_iters = n_tiles * num_kb;                        // pipeline steps per pass
+  const int prefill = total_iters < stages ? total_iters : stages;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(bar_full + 8u * s, 1);
+      mbar_init(bar_empty + 8u * s, 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(bar_tfull + 8u * a, 1);
+      mbar_init(bar_tempty + 8u * a, 4);
+    }
+    mbar_init(bar_pass, 1);
+    mbar_init(bar_spare, 1);
+    *abort_flag = 0;
+    s_pass_state[0] = s_pass_state[1] = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(tmem_ptr)), "r"((uint32_t)fa.tmem_cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  // ---- start of a draft: per-sequence state and the root rows (version 0 of the beam state)
+  for (int b = bid; b < p.B; b += G) {
+    const uint4* src = reinterpret_cast<const uint4*>(static_cast<const unsigned char*>(fa.root_hidden) +
+                                                      (size_t)b * p.Hd * 2);
+    uint4* dst = reinterpret_cast<uint4*>(static_cast<unsigned char*>(p.hbuf[0]) + (size_t)b * k * p.Hd * 2);
+    for (int j = threadIdx.x; j < p.Hd / 8; j += kTcThreads) dst[j] = src[j];
+    if (threadIdx.x == 0) {
+      const int tok = fa.root_token[b];
+      p.tree_token[(size_t)b * p.Nn] = tok;
+      p.tree_parent[(size_t)b * p.Nn] = -1;
+      p.tree_cum[(size_t)b * p.Nn] = 0.f;
+      fa.beam_node[b * k] = 0;
+      fa.beam_cum[b * k] = 0.f;
+      fa.row_plant[b * k] = (p.plant_next && tok >= 0 && tok < p.V) ? p.plant_next[tok] : -1;
+      p.active[b] = 1;
+      p.stop_depth[b] = 0;
+      p.root_pos[b] = fa.root_pos[b];
+    }
+  }
+  if (bid == 0 && threadIdx.x == 0) {
+    *p.n_active = p.B;
+    *p.dev_status = DDD_OK;
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_ptr;
+  if (threadIdx.x == 0) grid_arrive(cnt_hidden);     // instance 0 of hand-over 2
+
+  if (warp == 0) {
+    // ======================================================================= producer
+    unsigned long long evict_first = 0ull;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(evict_first));
+    uint32_t itg = 0;                // pipeline steps issued since the start of the draft
+    bool ok = true;
+    auto issue_w = [&](int i, int stage) {
+      const int t = i / num_kb, kb = i - t * num_kb;
+      const int nu = min(4, my_units - 4 * t);
+      const uint32_t full = bar_full + 8u * stage;
+      if (lane == 0) mbar_expect_tx(full, (uint32_t)ksub * ((uint32_t)nu * kUnitBytes + b_bytes));
+      __syncwarp();
+      const unsigned char* src = fa.w_packed + ((size_t)(kb * ksub) * n_units + (size_t)(unit0 + 4 * t)) * kUnitBytes;
+      const uint32_t dst = a_base + (uint32_t)stage * a_stage;
+      if (lane < ksub)
+        bulk_load_hint(dst + (uint32_t)lane * kABytes, src + (size_t)lane * n_units * kUnitBytes,
+                       (uint32_t)nu * kUnitBytes, full, evict_first);
+    };
+    auto issue_h = [&](const CUtensorMap* map, int i, int stage) {
+      if (lane == ksub)
+        tma_load_3d(b_base + (uint32_t)stage * b_stage, map, bar_full + 8u * stage, 0, 0, (i % num_kb) * ksub);
+    };
+    auto wait_stage_free = [&](uint32_t it) -> bool {
+      const uint32_t fill = it / (uint32_t)stages;
+      if (fill == 0) return true;
+      return __all_sync(kFullMask, mbar_wait(bar_empty + 8u * (it % stages), (fill - 1u) & 1u, abort_flag, p.dev_status));
+    };
+    for (int d = 1; d <= p.n; ++d) {
+      const CUtensorMap* map = ((d - 1) & 1) ? &map_h1 : &map_h0;
+      const uint32_t it0 = itg;
+      // W of the first steps of this pass: it depends on nothing, so it is fetched while the tree
+      // work of the previous pass is still going on elsewhere
+      int issued_w = 0;
+      for (; issued_w < prefill && ok; ++issued_w) {
+        ok = wait_stage_free(itg);
+        if (!ok) break;
+        issue_w(issued_w, (int)(itg % stages));
+        ++itg;
+      }
+      // hand-over 2 of the previous pass: hidden rows and state of this pass are in place
+      int go = 0;
+      if (ok) {
+        if (lane == 0) {
+          go = grid_wait(cnt_hidden, d * G, abort_word, p.dev_status) ? 1 : -1;
+          if (go == 1 && d > 1 && *reinterpret_cast<volatile const int*>(p.n_active) == 0) go = 0;
+        }
+        go = __shfl_sync(kFullMask, go, 0);
+      } else {
+        go = -1;
+      }
+      if (lane == 0) {
+        if (go < 0) *abort_flag = 1;
+        s_pass_state[(d - 1) & 1] = go == 1 ? d : 0;
+        mbar_arrive(bar_pass);                       // tells the other warps of the block
+      }
+      __syncwarp();
+      asm volatile("fence.proxy.async;" ::: "memory");
+      // the hidden rows of the steps already holding W (on a stop they are fetched all the same:
+      // a stage's barrier only completes, and its copies only end, once both parts have landed)
+      for (int i = 0; i < issued_w; ++i) issue_h(map, i, (int)((it0 + i) % stages));
+      __syncwarp();
+      if (go != 1) {
+        for (int i = 0; i < issued_w; ++i) {
+          const uint32_t it = it0 + i;
+          mbar_wait(bar_full + 8u * (it % stages), (it / stages) & 1u, abort_flag, p.dev_status, false);
+        }
+        __syncwarp();
+        break;
+      }
+      for (int i = prefill; i < total_iters; ++i) {
+        ok = wait_stage_free(itg);
+        if (!ok) break;
+        issue_w(i, (int)(itg % stages));
+        issue_h(map, i, (int)(itg % stages));
+        __syncwarp();
+        ++itg;
+      }
+      if (!ok) {
+        // gave up in mid-pass: wait (bounded) until every copy already issued has landed
+        for (uint32_t it = (itg > (uint32_t)stages ? itg - stages : 0u); it < itg; ++it)
+          mbar_wait(bar_full + 8u * (it % stages), (it / stages) & 1u, abort_flag, p.dev_status, false);
+        __syncwarp();
+        break;
+      }
+    }
+  } else if (warp == 1) {
+    // ======================================================================= MMA issuer
+    const uint32_t idesc = make_instr_desc(n_pad);
+    uint32_t itg = 0, tg = 0;
+    bool ok = true;
+    for (int d = 1; d <= p.n && ok; ++d) {
+      ok = __all_sync(kFullMask, mbar_wait(bar_pass, (uint32_t)(d - 1) & 1u, abort_flag, p.dev_status));
+      if (!ok || s_pass_state[(d - 1) & 1] == 0) break;
+      for (int t = 0; t < n_tiles && ok; ++t, ++tg) {
+        const int acc = (int)(tg & 1u);
+        ok = __all_sync(kFullMask, mbar_wait(bar_tempty + 8u * acc, ((tg >> 1) & 1u) ^ 1u, abort_flag, p.dev_status));
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * n_pad);
+        for (int kb = 0; kb < num_kb; ++kb, ++itg) {
+          const int stage = (int)(itg % stages);
+          ok = __all_sync(kFullMask, mbar_wait(bar_full + 8u * stage, (itg / stages) & 1u, abort_flag, p.dev_status));
+          if (!ok) break;
+          tc_fence_after();
+          if (lane == 0) {
+            for (int kk = 0; kk < ksub; ++kk) {
+              const uint32_t a_addr = a_base + (uint32_t)stage * a_stage + (uint32_t)kk * kABytes;
+              const uint32_t b_addr = b_base + (uint32_t)stage * b_stage + (uint32_t)kk * b_bytes;
+#pragma unroll
+              for (int k4 = 0; k4 < kBlockK / kUmmaK; ++k4)
+                tc_mma_bf16(d_tmem, make_smem_desc(a_addr + k4 * kUmmaK * 2), make_smem_desc(b_addr + k4 * kUmmaK * 2),
+                            idesc, (kb | kk | k4) != 0 ? 1u : 0u);
+            }
+            tc_commit(bar_empty + 8u * stage);
+          }
+          __syncwarp();
+        }
+        if (ok && lane == 0) tc_commit(bar_tfull + 8u * acc);
+        __syncwarp();
+      }
+    }
+    if (!ok) {
+      // make sure no MMA is still running before tensor memory is released
+      if (lane == 0) tc_commit(bar_spare);
+      __syncwarp();
+      mbar_wait(bar_spare, 0u, abort_flag, p.dev_status, false);
+      __syncwarp();
+    }
+  } else {
+    // ======================================================================= epilogue, then tree work
+    const int quarter = warp & 3;
+    const int ew = warp - 2, et = (int)threadIdx.x - 64;
+    const int lw = ew >> 2;
+    const int n_chunks = (R + kChunkCols - 1) / kChunkCols;
+    const int cpr = p.Hd / 8;                      // 16-byte chunks per hidden row
+    const bool row_by_block = (cpr % 32 == 0) && (cpr / 32 <= 64);
+    uint32_t tg = 0;
+    bool ok = true;
+    for (int d = 1; d <= p.n; ++d) {
+      ok = epilogue_all(mbar_wait(bar_pass, (uint32_t)(d - 1) & 1u, abort_flag, p.dev_status, false));
+      if (!ok || s_pass_state[(d - 1) & 1] == 0) break;
+      const int par_in = (d - 1) & 1, par_out = d & 1;
+      // ---- per-row flags and running state of this pass
+      for (int r = et; r < R; r += kEpiThreads) {
+        s_plant[r] = fa.row_plant[par_in * R + r];
+        s_live[r] = row_live(p, r, d, 0) ? 1 : 0;
+        st_ms[r] = make_float2(neg_inf(), 0.f);
+      }
+      for (int i = et; i < R * k; i += kEpiThreads) st_key[i] = 0ull;
+      epilogue_barrier();
+      // ---- the tiles of this block's vocabulary range
+      for (int t = 0; t < n_tiles && ok; ++t, ++tg) {
+        const int acc = (int)(tg & 1u);
+        const int rows = min(4, my_units - 4 * t) * kUnitRows;
+        const int row0 = (unit0 + 4 * t) * kUnitRows;
+        ok = epilogue_all(mbar_wait(bar_tfull + 8u * acc, (tg >> 1) & 1u, abort_flag, p.dev_status, false));
+        if (!ok) break;
+        tc_fence_after();
+        const int vrow = quarter * 32 + lane;
+        const int v = row0 + vrow;
+        const bool v_ok = vrow < rows && v < p.Vl;
+        const float bias = (v_ok && p.bias) ? p.bias[v] : 0.f;
+        for (int g0 = 0; g0 < n_chunks; g0 += cpg) {
+          const int ch = g0 + lw;
+          if (lw < cpg && ch < n_chunks) {
+            const int c0 = ch * kChunkCols;
+            float accv[16];
+            tc_load_16cols(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * n_pad + c0), accv);
+#pragma unroll
+            for (int c = 0; c < kChunkCols; ++c) {
+              const int r = c0 + c;
+              float z = neg_inf();
+              if (v_ok && r < R && s_plant[r] != v + p.v0) z = fmaf(accv[c], p.s, bias);
+              zt[(lw * kChunkCols + c) * kTile + vrow] = z;
+            }
+            tc_fence_before();
+          }
+          epilogue_barrier();
+          if (g0 + cpg >= n_chunks && ew < 4 && lane == 0) mbar_arrive(bar_tempty + 8u * acc);
+          for (int rr = ew; rr < cpg * kChunkCols; rr += kEpiWarps) {
+            const int r = g0 * kChunkCols + rr;
+            if (r >= R || !s_live[r]) continue;
+            float2 ms = st_ms[r];
+            unsigned long long key = lane < k ? st_key[r * k + lane] : 0ull;
+            row_tile_update(zt + rr * kTile, row0 + p.v0, k, ms.x, ms.y, key);
+            if (lane < k) st_key[r * k + lane] = key;
+            if (lane == 0) st_ms[r] = ms;
+          }
+          epilogue_barrier();
+        }
+      }
+      if (!ok) break;
+      // ---- publish this block's partials: hand-over 1
+      for (int r = ew; r < R; r += kEpiWarps) {
+        if (!s_live[r]) continue;
+        const size_t slot = (size_t)bid * R + r;
+        if (lane < k) p.part_key[slot * k + lane] = st_key[r * k + lane];
+        if (lane == 0) p.part_ms[slot] = st_ms[r];
+      }
+      epilogue_barrier();
+      if (et == 0) grid_arrive(cnt_partials);
+
+      // ---- tree work: the new beam rows this block owns
+      const int P = (d == 1) ? 1 : k;
+      const int base = (d == 1) ? 1 : 1 + k + (d - 2) * k * k;
+      bool waited = false;
+      int cur_b = -1;
+      for (int r_new = bid; r_new < R && ok; r_new += G) {
+        const int b = r_new / k, i = r_new - b * k;
+        if (!s_live[b * k]) continue;                 // sequence not drafting in this pass
+        if (d == p.n && i != 0) continue;             // after the last pass there is no draft step
+        if (!waited) {
+          bool w_ok = true;
+          if (et == 0) w_ok = grid_wait(cnt_partials, d * G, abort_word, p.dev_status);
+          ok = epilogue_all(w_ok);
+          waited = true;
+          if (!ok) break;
+        }
+        if (b != cur_b) {
+          cur_b = b;
+          // merge the partial lists of the sequence's rows, one warp per row
+          for (int pr = ew; pr < P; pr += kEpiWarps) {
+            const int r = b * k + pr;
+            float M, S;
+            unsigned long long res = merge_row_global(p, r, M, S);
+            const int pc = s_plant[r];
+            if (pc >= 0) {      // planted column: (max of the others) + delta; it was left out of the partials
+              const float zc = M + p.plant_delta;
+              const float M2 = fmaxf(M, zc);
+              S = S * expf(M - M2) + expf(zc - M2);
+              M = M2;
+              const unsigned long long plant_key = make_key(zc, (uint32_t)pc);
+              const int ins = __popc(__ballot_sync(kFullMask, lane < k && res > plant_key));
+              const unsigned long long up = __shfl_up_sync(kFullMask, res, 1);
+              if (lane == ins) res = plant_key;
+              else if (lane > ins) res = up;
+            }
+            const float lse = M + logf(S);
+            if (lane < k) {
+              const float lp = (res != 0ull) ? fminf(key_value(res) - lse, 0.f) : neg_inf();
+              const int tok = (res != 0ull) ? (int)key_index(res) : -1;
+              const float cand = fa.beam_cum[par_in * R + r] + lp;
+              cand_s[pr * k + lane] = ((unsigned long long)__float_as_uint(cand) << 32) | (uint32_t)tok;
+            }
+            if (lane == 0) lse_s[pr] = lse;
+          }
+          epilogue_barrier();
+          // the new beam, Eq. 1 and the gate
+          if (ew == 0) {
+            auto cand_key_of = [&](int idx) -> unsigned long long {
+              const unsigned long long rec = cand_s[idx];
+              return (int)(uint32_t)rec >= 0 ? make_key(__uint_as_float((uint32_t)(rec >> 32)), (uint32_t)idx) : 0ull;
+            };
+            const int n_cand = P * k;
+            unsigned long long mine = 0ull;
+            if (n_cand <= 128) {
+              unsigned long long ck[4];
+#pragma unroll
+              for (int q = 0; q < 4; ++q) ck[q] = lane + 32 * q < n_cand ? cand_key_of(lane + 32 * q) : 0ull;
+              for (int j = 0; j < k; ++j) {
+                unsigned long long best = ck[0];
+#pragma unroll
+                for (int q = 1; q < 4; ++q) best = ck[q] > best ? ck[q] : best;
+                const unsigned long long wk = warp_max_key(best);
+                if (lane == j) mine = wk;
+                if (wk == 0ull) break;
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                  if (ck[q] == wk) ck[q] = 0ull;
+              }
+            } else {
+              int pos = 0;
+              unsigned long long head = lane < P ? cand_key_of(lane * k) : 0ull;
+              for (int j = 0; j < k; ++j) {
+                const unsigned long long wk = warp_max_key(head);
+                if (lane == j) mine = wk;
+                if (wk == 0ull) break;
+                if (head == wk) {
+                  ++pos;
+                  head = pos < k ? cand_key_of(lane * k + pos) : 0ull;
+                }
+              }
+            }
+            const bool have = lane < k && mine != 0ull;
+            const int flat = have ? (int)key_index(mine) : 0;
+            const float cum = have ? __uint_as_float((uint32_t)(cand_s[flat] >> 32)) : neg_inf();
+            const float M = __shfl_sync(kFullMask, cum, 0);
+            const float sum = warp_sum(have ? expf(cum - M) : 0.f);
+            const float H = M + logf(sum);
+            bool stop = (d == p.n);
+            if (!stop && ((p.check_mask >> (d - 1)) & 1u)) stop = H < p.x;
+            if (lane < k) {
+              sel_flat[lane] = flat;
+              sel_tok[lane] = (int)(uint32_t)cand_s[flat];
+              sel_cum[lane] = cum;
+            }
+            if (lane == 0) {
+              s_misc[0] = stop ? 1 : 0;
+              s_misc[1] = __float_as_int(H);
+            }
+          }
+          epilogue_barrier();
+          if (i == 0) {
+            // this block keeps the sequence's books
+            for (int flat = et; flat < P * k; flat += kEpiThreads) {
+              const unsigned long long rec = cand_s[flat];
+              const size_t node = (size_t)b * p.Nn + base + flat;
+              p.tree_token[node] = (int)(uint32_t)rec;
+              p.tree_parent[node] = fa.beam_node[par_in * R + b * k + flat / k];
+              p.tree_cum[node] = __uint_as_float((uint32_t)(rec >> 32));
+            }
+            if (et < k) {
+              const int tok = sel_tok[et];
+              fa.beam_node[par_out * R + b * k + et] = base + sel_flat[et];
+              fa.beam_cum[par_out * R + b * k + et] = sel_cum[et];
+              fa.row_plant[par_out * R + b * k + et] = (p.plant_next && tok >= 0 && tok < p.V) ? p.plant_next[tok] : -1;
+              if (fa.io.trace.beam_sel) fa.io.trace.beam_sel[((size_t)b * p.n + (d - 1)) * k + et] = sel_flat[et];
+            }
+            if (et < P && fa.io.trace.row_lse) fa.io.trace.row_lse[((size_t)b * p.n + (d - 1)) * k + et] = lse_s[et];
+            if (et == 0) {
+              fa.io.out.H_trace[(size_t)b * p.n + (d - 1)] = __int_as_float(s_misc[1]);
+              if (s_misc[0]) {
+                p.stop_depth[b] = d;
+                p.active[b] = 0;
+                atomicSub(p.n_active, 1);
+              }
+            }
+          }
+        }
+        if (s_misc[0]) continue;                       // the sequence stops here: no draft step
+        // ---- draft step of new beam row i: h = round(u / sqrt(mean(u^2) + eps)), u = h_parent + E[token]
+        {
+          const int tok = sel_tok[i];
+          const uint4* hp = reinterpret_cast<const uint4*>(p.hbuf[par_in]) + (size_t)(b * k + sel_flat[i] / k) * cpr;
+          const uint4* er = reinterpret_cast<const uint4*>(p.E) + (size_t)(tok >= 0 && tok < p.V ? tok : 0) * cpr;
+          uint4* out = reinterpret_cast<uint4*>(p.hbuf[par_out]) + (size_t)(b * k + i) * cpr;
+          if (row_by_block) {
+            // chunk q belongs to thread q mod 512; a warp's 32 chunks form one partial sum (slot q / 32)
+            const int slots = cpr / 32;
+            uint4 hv0 = make_uint4(0, 0, 0, 0), ev0 = hv0;
+            for (int q = et; q - lane < cpr; q += kEpiThreads) {
+              const uint4 hv = hp[q], ev = er[q];
+              if (q == et) { hv0 = hv; ev0 = ev; }
+              double u[8];
+              Chunk<__nv_bfloat16>::sum(hv, ev, u);
+              double ss = 0.0;
+#pragma unroll
+              for (int e = 0; e < 8; ++e) ss = fma(u[e], u[e], ss);
+              ss = warp_sum_f64(ss);
+              if (lane == 0) red_s[q / 32] = ss;
+            }
+            epilogue_barrier();
+            double ss = 0.0;
+            for (int j = 0; j < slots; ++j) ss += red_s[j];
+            const double inv = 1.0 / sqrt(ss / (double)p.Hd + (double)p.eps);
+            for (int q = et; q < cpr; q += kEpiThreads) {
+              uint4 hv = hv0, ev = ev0;
+              if (q != et) { hv = hp[q]; ev = er[q]; }
+              double u[8];
+              Chunk<__nv_bfloat16>::sum(hv, ev, u);
+#pragma unroll
+              for (int e = 0; e < 8; ++e) u[e] *= inv;
+              out[q] = Chunk<__nv_bfloat16>::round(u);
+            }
+            epilogue_barrier();                          // red_s is reused by the block's next row
+          } else if (ew == 0) {
+            // rows that are not a whole number of 32-chunk groups: one warp does the row
+            double ss = 0.0;
+            for (int c = lane; c < cpr; c += 32) {
+              double u[8];
+              Chunk<__nv_bfloat16>::sum(hp[c], er[c], u);
+#pragma unroll
+              for (int e = 0; e < 8; ++e) ss = fma(u[e], u[e], ss);
+            }
+            ss = warp_sum_f64(ss);
+            const double inv = 1.0 / sqrt(ss / (double)p.Hd + (double)p.eps);
+            for (int c = lane; c < cpr; c += 32) {
+              double u[8];
+              Chunk<__nv_bfloat16>::sum(hp[c], er[c], u);
+#pragma unroll
+              for (int e = 0; e < 8; ++e) u[e] *= inv;
+              out[c] = Chunk<__nv_bfloat16>::round(u);
+            }
+          }
+        }
+      }
+      if (!ok) break;
+      // ---- hand-over 2: this block's share of the next pass's state and hidden rows is written
+      epilogue_barrier();
+      if (et == 0) grid_arrive(cnt_hidden);
+    }
+    if (!ok && et == 0) *abort_flag = 1;
+  }
+
+  // ---- teardown: everyone meets, the MMAs are known to have ended (every accumulator that was
+  // committed has been read, or the block gave up after bounded waits), tensor memory is freed;
+  // the last block out resets the hand-over counters for the next draft
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (warp == 1) {
+    __syncwarp();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)fa.tmem_cols)
+                 : "memory");
+  }
+  if (threadIdx.x == 0) {
+    if (*abort_flag) atomicExch(abort_word, 1);
+    __threadfence();
+    if (atomicAdd(exit_ticket, 1) == G - 1) {
+      atomicExch(cnt_partials, 0);
+      atomicExch(cnt_hidden, 0);
+      atomicExch(abort_word, 0);
+      atomicExch(exit_ticket, 0);
+      __threadfence();
+    }
+  }
+}
+
+// The rerank and the mask of every sequence, after the draft: one block per sequence.
+__global__ void __launch_bounds__(1024) rerank_kernel(const Params p, const DraftIO io, const int keys_in_smem) {
+  griddep_wait();
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int b = blockIdx.x;
+  const int D = p.stop_depth[b];
+  if (keys_in_smem) rerank_mask_block<1024, true>(p, io, b, D, b == 0, smem_raw);
+  else rerank_mask_block<1024, false>(p, io, b, D, b == 0, smem_raw);
+}
+
+size_t rerank_kernel_smem(const Params& p, bool* keys_in_smem) {
+  const size_t both = (size_t)p.Nn * (sizeof(uint32_t) + sizeof(short));
+  *keys_in_smem = both <= 160 * 1024;
+  return *keys_in_smem ? both : (size_t)p.Nn * sizeof(short);
+}
+
+}  // namespace
+
+int fused_extra_smem(int k) { return tree_smem(k).total + 8; }
+
+bool fused_supported(const Params& p) {
+  return p.dtype == DDD_DTYPE_BF16 && p.Hd % kBlockK == 0 && p.k <= kNarrowK && p.lm_ctas <= kFusedMaxCtas;
+}
+
+int fused_prepare(const Params& p, const TcPlan& plan) {
+  if (!fused_supported(p)) return DDD_ERR_UNSUPPORTED;
+  if (allow_max_dynamic_smem(draft_fused_kernel) != cudaSuccess) return DDD_ERR_CUDA;
+  if (allow_max_dynamic_smem(rerank_kernel) != cudaSuccess) return DDD_ERR_CUDA;
+  // every block must be resident at once: the blocks wait for one another
+  int per_sm = 0, dev = 0, sms = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, draft_fused_kernel, kTcThreads, plan.smem) != cudaSuccess ||
+      cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return DDD_ERR_CUDA;
+  if (per_sm < 1 || plan.ctas > per_sm * sms) return DDD_ERR_UNSUPPORTED;
+  bool keys;
+  cudaFuncAttributes fattr;
+  if (cudaFuncGetAttributes(&fattr, rerank_kernel) != cudaSuccess) return DDD_ERR_CUDA;
+  if (rerank_kernel_smem(p, &keys) + fattr.sharedSizeBytes > (size_t)kSmemLimit) return DDD_ERR_UNSUPPORTED;
+  return DDD_OK;
+}
+
+cudaError_t launch_draft_fused(const Params& p, const TcPlan& plan, const FusedArgs& fa_in, cudaStream_t st) {
+  FusedArgs fa = fa_in;
+  fa.w_packed = plan.w_packed;
+  fa.n_pad = plan.n_pad;
+  fa.stages = plan.stages;
+  fa.ksub = plan.ksub;
+  fa.cpg = plan.epi_chunks;
+  fa.tmem_cols = plan.tmem_cols;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)plan.ctas, 1, 1);
+  cfg.blockDim = dim3(kTcThreads, 1, 1);
+  cfg.dynamicSmemBytes = plan.smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeCooperative;       // all blocks resident at once, or the launch fails
+  attr[0].val.cooperative = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, draft_fused_kernel, p, fa, plan.map_h[0], plan.map_h[1]);
+  if (e != cudaSuccess) return e;
+  // rerank + mask: started early (programmatic dependent launch), waits on the device for the draft
+  bool keys;
+  cudaLaunchConfig_t rc = {};
+  rc.gridDim = dim3((unsigned)p.B, 1, 1);
+  rc.blockDim = dim3(1024, 1, 1);
+  rc.dynamicSmemBytes = rerank_kernel_smem(p, &keys);
+  rc.stream = st;
+  cudaLaunchAttribute rattr[1];
+  rattr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  rattr[0].val.programmaticStreamSerializationAllowed = 1;
+  rc.attrs = rattr;
+  rc.numAttrs = 1;
+  return cudaLaunchKernelEx(&rc, rerank_kernel, p, fa.io, keys ? 1 : 0);
+}
+
+}  // namespace ddd

@@ -1,0 +1,33 @@
+// Host interface of the one-kernel-per-draft path (draft_fused.cu).
+#pragma once
+
+#include "ddd_common.cuh"
+#include "lm_head_tc.cuh"
+
+namespace ddd {
+
+// What the persistent kernel needs beyond Params: the caller's root and output pointers of this
+// draft and the state that only this path keeps (all device pointers into the workspace).
+struct FusedArgs {
+  const unsigned char* w_packed;
+  const void* root_hidden;
+  const int* root_token;
+  const int* root_pos;
+  DraftIO io;
+  float* beam_cum;      // [2][R] summed log-probability of the beam, by pass parity
+  int* beam_node;       // [2][R] tree node of each beam entry
+  int* row_plant;       // [2][R] planted column of each beam row, -1 = none
+  int* sync;            // [4] hand-over counters (partials, hidden rows), abort word, exit ticket
+  int n_pad, stages, ksub, cpg, tmem_cols;
+};
+
+// Shared memory the tree work needs behind the LM-head pipeline's own.
+int fused_extra_smem(int k);
+// Can this configuration run as one kernel (bf16, tensor-core kernel, beam width up to 32)?
+bool fused_supported(const Params& p);
+// Checks that all blocks fit on the device at once and sets the kernels' attributes.  DDD_* code.
+int fused_prepare(const Params& p, const TcPlan& plan);
+// Enqueues the draft kernel and, behind it, the rerank kernel.
+cudaError_t launch_draft_fused(const Params& p, const TcPlan& plan, const FusedArgs& fa, cudaStream_t st);
+
+}  // namespace ddd

@@ -23,7 +23,8 @@ struct TcPlan {
 size_t tc_packed_bytes(int vocab, int hidden);
 // Packs W into `w_packed` (device, 1024-byte aligned, tc_packed_bytes), encodes the tensor maps of
 // the hidden buffers and sizes the pipeline.  Synchronises the device.  Returns a DDD_* code.
-int tc_plan_create(const Params& p, int sm_count, void* w_packed, TcPlan* plan);
+// extra_smem: bytes kept free behind the pipeline's own shared memory (for a kernel that does more than the pass).
+int tc_plan_create(const Params& p, int sm_count, void* w_packed, TcPlan* plan, int extra_smem = 0);
 // pdl: launch with programmatic stream serialisation (see griddep_wait in ddd_common.cuh).
 cudaError_t launch_lm_head_tc(const Params& p, const TcPlan& plan, int d, int force_all, bool pdl, cudaStream_t st);
 

@@ -237,8 +237,11 @@ def random_shapes():
 @pytest.mark.parametrize("index", range(40))
 def test_random_shapes_match_oracle(index):
     cfg = random_shapes()[index]
-    mode = P.DDD_LAUNCH_GRAPH if index % 2 else P.DDD_LAUNCH_STREAM
-    eng = engine_for(cfg, SIMT if index % 5 == 4 else TC, mode)
+    kernel = SIMT if index % 5 == 4 else TC
+    mode = (P.DDD_LAUNCH_STREAM, P.DDD_LAUNCH_GRAPH, P.DDD_LAUNCH_FUSED)[index % 3]
+    if mode == P.DDD_LAUNCH_FUSED and kernel == SIMT:
+        mode = P.DDD_LAUNCH_GRAPH
+    eng = engine_for(cfg, kernel, mode)
     with torch.cuda.stream(torch.cuda.Stream()):
         for i in range(2):
             roots = S.make_roots(cfg, i)
@@ -331,6 +334,61 @@ def test_captured_drafts_of_every_stop_depth_equal_stream_launches(schedule):
         assert seen <= {4, 6}, sorted(seen)
 
 
+# ----------------------------------------------------------------------------- one persistent kernel per draft
+@pytest.mark.parametrize("case", list(small_cases()))
+def test_fused_draft_equals_kernel_by_kernel_draft(case):
+    # same partials, same merge order, same fp64 draft step: the one-kernel draft must give the
+    # results of the kernel-by-kernel launches bit for bit, and both must match the oracle
+    cfg = small_cases()[case]
+    eng_s = engine_for(cfg, TC, P.DDD_LAUNCH_STREAM)
+    eng_f = engine_for(cfg, TC, P.DDD_LAUNCH_FUSED)
+    assert P.ddd_launches_per_draft(eng_f.handle, 1) == 2
+    depths = set()
+    for i in range(4):
+        roots = S.make_roots(cfg, i)
+        a = parity.run_gpu(eng_s, roots)
+        b = parity.run_gpu(eng_f, roots)
+        for name in a:
+            if name in ("beam_sel", "row_lse", "H_trace"):
+                for q in range(cfg.batch):
+                    D = int(a["stop_depth"][q])
+                    np.testing.assert_array_equal(a[name][q, :D], b[name][q, :D], err_msg=name)
+            else:
+                np.testing.assert_array_equal(a[name], b[name], err_msg=name)
+        parity.compare_with_oracle(cfg, weights_for(cfg), roots, b)
+        depths.update(b["stop_depth"].tolist())
+    # two drafts back to back without a synchronisation in between, then the host-buffer entry point
+    r0, r1 = (parity.to_device(S.make_roots(cfg, j), eng_f.device) for j in (0, 1))
+    eng_f.draft(r0["root_hidden"], r0["root_token"], r0["root_pos"])
+    eng_f.draft(r1["root_hidden"], r1["root_token"], r1["root_pos"])
+    last = {k2: v.numpy() for k2, v in eng_f.results().items()}
+    want = parity.run_gpu(eng_s, S.make_roots(cfg, 1))
+    np.testing.assert_array_equal(last["token"], want["token"])
+    np.testing.assert_array_equal(last["mask"], want["mask"])
+    host_out = eng_f.make_host_out()
+    hr = S.make_roots(cfg, 1)
+    eng_f.draft_host(hr["root_hidden"].pin_memory(), hr["root_token"].pin_memory(), hr["root_pos"].pin_memory(), host_out)
+    for name in host_out:
+        if name == "H_trace":       # entries of passes that did not run keep whatever an earlier draft left
+            for q in range(cfg.batch):
+                D = int(want["stop_depth"][q])
+                np.testing.assert_array_equal(host_out[name].numpy()[q, :D], want[name][q, :D])
+        else:
+            np.testing.assert_array_equal(host_out[name].numpy(), want[name], err_msg=name)
+    eng_s.close()
+    eng_f.close()
+    if case == "full_depth":
+        assert depths == {cfg.max_depth}
+
+
+def test_fused_mode_is_refused_where_it_cannot_run():
+    base = S.scaled_down(S.CONFIGS["llama2_7b"], 256, 3000, threshold=NEG, max_depth=2, total_tokens=20)
+    for cfg, kernel in ((base.replace(k=33), TC), (S.CONFIGS["tiny"], P.DDD_LM_HEAD_AUTO), (base, SIMT)):
+        with pytest.raises(P.DddError) as err:
+            P.DraftEngine(cfg, weights_for(cfg), lm_head_kernel=kernel, launch_mode=P.DDD_LAUNCH_FUSED)
+        assert err.value.code == -6
+
+
 def test_handles_of_different_sizes_coexist():
     # kernel attributes (dynamic shared memory limit) are per process: a smaller handle created
     # later must not take room away from a larger one created earlier
@@ -386,7 +444,7 @@ FULL_SIZE = [
                          ids=[f"{c[0]}_x{c[1]:g}" for c in FULL_SIZE])
 def test_full_size_configs_in_bench_launch_configuration(name, threshold, n_drafts, min_strict, record_property):
     cfg = S.CONFIGS[name].replace(threshold=threshold)
-    eng = engine_for(cfg, P.DDD_LM_HEAD_AUTO, P.DDD_LAUNCH_GRAPH)
+    eng = engine_for(cfg, P.DDD_LM_HEAD_AUTO, P.DDD_LAUNCH_FUSED)
     depths, strict = [], 0
     with torch.cuda.stream(torch.cuda.Stream()):
         for i in range(n_drafts):
