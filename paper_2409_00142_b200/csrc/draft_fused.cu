@@ -38,9 +38,10 @@ namespace {
 using namespace tc;
 
 constexpr int kListDepth = 8;     // keys of a partial list a lane keeps in registers during a merge
+constexpr int kTreeOverZt = kChunkCols * kTile * 4;     // smallest transpose buffer of the epilogue (8 KB)
 
 struct TreeSmem {
-  int cand, lse, sel_flat, sel_tok, sel_cum, red, misc, bar, total;
+  int cand, lse, sel_flat, sel_tok, sel_cum, red, misc, total;
 };
 __host__ __device__ inline TreeSmem tree_smem(int k) {
   TreeSmem t;
@@ -53,7 +54,6 @@ __host__ __device__ inline TreeSmem tree_smem(int k) {
   off = (off + 7) / 8 * 8;
   t.red = off; off += 64 * 8;                // partial sums of squares of one row
   t.misc = off; off += 16;                   // stop flag, H
-  t.bar = off; off += 8;                     // spare mbarrier (end of the MMAs on a give-up)
   t.total = off;
   return t;
 }
@@ -178,7 +178,9 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
   const int stages = fa.stages, ksub = fa.ksub, n_pad = fa.n_pad, cpg = fa.cpg;
   const SmemPlan sp = smem_plan(stages, ksub, n_pad, p.R, p.k, cpg);
   const TreeSmem ts = tree_smem(p.k);
-  unsigned char* tree_base = smem + ((sp.total + 7) / 8 * 8);
+  // The tree work's scratch lies over the epilogue's transpose buffer, which is idle between the
+  // last tile of a pass and the first of the next (behind everything else where it is too large).
+  unsigned char* tree_base = ts.total <= kTreeOverZt ? smem + sp.zt : smem + ((sp.total + 7) / 8 * 8);
   float* zt = reinterpret_cast<float*>(smem + sp.zt);
   unsigned long long* st_key = reinterpret_cast<unsigned long long*>(smem + sp.key);
   float2* st_ms = reinterpret_cast<float2*>(smem + sp.ms);
@@ -195,13 +197,14 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
   double* red_s = reinterpret_cast<double*>(tree_base + ts.red);
   volatile int* s_misc = reinterpret_cast<volatile int*>(tree_base + ts.misc);    // [0] stop, [1] H bits
   __shared__ int s_pass_state[2];      // what the producer learnt at hand-over 2: pass number to run, or 0 = leave
+  __shared__ __align__(8) unsigned long long s_bar_spare;   // end of the MMAs when the block gives up
 
   const uint32_t a_base = smem_u32(smem + sp.a), b_base = smem_u32(smem + sp.b);
   const uint32_t b_bytes = (uint32_t)n_pad * kBlockK * 2;
   const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8u * stages;
   const uint32_t bar_tfull = bar_empty + 8u * stages, bar_tempty = bar_tfull + 16u;
   const uint32_t bar_pass = bar_tempty + 16u;      // the plan's fifth word: "the producer knows how the draft goes on"
-  const uint32_t bar_spare = smem_u32(tree_base + ts.bar);
+  const uint32_t bar_spare = smem_u32(&s_bar_spare);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = (int)gridDim.x, bid = (int)blockIdx.x;
@@ -709,7 +712,10 @@ size_t rerank_kernel_smem(const Params& p, bool* keys_in_smem) {
 
 }  // namespace
 
-int fused_extra_smem(int k) { return tree_smem(k).total + 8; }
+int fused_extra_smem(int k) {
+  const int t = tree_smem(k).total;
+  return t <= kTreeOverZt ? 0 : t + 8;
+}
 
 bool fused_supported(const Params& p) {
   return p.dtype == DDD_DTYPE_BF16 && p.Hd % kBlockK == 0 && p.k <= kNarrowK && p.lm_ctas <= kFusedMaxCtas;
