@@ -28,7 +28,7 @@ size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 struct Layout {
   size_t hbuf[2], part_key, part_ms, tree_token, tree_parent, tree_cum, beam_node, beam_tok, beam_cum,
       row_plant, active, stop_depth, root_pos, n_active, dev_status, lm_ticket, shard_counter, fused_sync,
-      fused_beam_cum, fused_beam_node, fused_row_plant, w_packed;
+      fused_beam_cum, fused_beam_node, fused_row_plant, fused_key, fused_ms, w_packed;
   // staging for ddd_draft_host: inputs, then the packed output block
   size_t in_hidden, in_token, in_pos, out_block;
   size_t o_n_out, o_stop, o_token, o_parent, o_depth, o_position, o_cum, o_mask, o_H, o_status, out_bytes;
@@ -90,6 +90,9 @@ Layout make_layout(const ddd_config* c) {
   L.fused_beam_cum = take(2 * R * 4);
   L.fused_beam_node = take(2 * R * 4);
   L.fused_row_plant = take(2 * R * 4);
+  const bool may_fuse = c->launch_mode == DDD_LAUNCH_FUSED && k <= 32;
+  L.fused_key = take(may_fuse ? R * k * 160 * 8 : 0);
+  L.fused_ms = take(may_fuse ? R * 160 * 8 : 0);
   // packed copy of W for the tensor-core kernel (kept 1024-byte aligned relative to the base)
   off = (off + 1023) / 1024 * 1024;
   const bool tc_possible = c->dtype == DDD_DTYPE_BF16 && c->hidden % 64 == 0 && c->lm_head_kernel != DDD_LM_HEAD_SIMT;
@@ -446,6 +449,8 @@ int ddd_draft(ddd_handle* h, const void* root_hidden, const int32_t* root_token,
     fa.beam_node = reinterpret_cast<int*>(h->ws + h->L.fused_beam_node);
     fa.row_plant = reinterpret_cast<int*>(h->ws + h->L.fused_row_plant);
     fa.sync = reinterpret_cast<int*>(h->ws + h->L.fused_sync);
+    fa.fkey = reinterpret_cast<unsigned long long*>(h->ws + h->L.fused_key);
+    fa.fms = reinterpret_cast<float2*>(h->ws + h->L.fused_ms);
     if (launch_draft_fused(h->p, h->tc, fa, st) != cudaSuccess) {
       note_cuda_error(__LINE__);
       return DDD_ERR_CUDA;

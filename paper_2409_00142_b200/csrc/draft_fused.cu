@@ -37,7 +37,6 @@ namespace {
 
 using namespace tc;
 
-constexpr int kListDepth = 8;     // keys of a partial list a lane keeps in registers during a merge
 constexpr int kTreeOverZt = kChunkCols * kTile * 4;     // smallest transpose buffer of the epilogue (8 KB)
 
 struct TreeSmem {
@@ -95,28 +94,42 @@ __device__ __forceinline__ void grid_arrive(int* counter) {
   atomicAdd(counter, 1);
 }
 
-// Merge of one beam row's partial lists (part_key [nc][R][k], sorted descending) by one warp,
-// straight from global memory: the k lists with the best heads are the only ones that can
-// contribute; lane j walks the j-th of them with its next kListDepth keys in registers.  Lane j
-// returns the j-th best key, and (M, S) = the row's merged max and sum-exp (all lanes).
-constexpr int kFusedMaxCtas = 160;     // partial lists per row the merge keeps heads of (five per lane)
+// Merge of one beam row's partial lists by one warp.  The warp is alone on the critical path, so
+// what counts is the number of dependent instructions and of loads of lines that another SM has
+// just written (those cost about three times an ordinary L2 hit).  Hence the layout: this path
+// keeps its partials position-major, fkey [R][k][kFusedMaxCtas] and fms [R][kFusedMaxCtas], so that
+// the heads of all blocks' lists are one contiguous run, the second entries the next, and a lane
+// fetches the first two entries of the lists of blocks lane, lane + 32, ... with coalesced loads
+// in a single round trip.  A round of the k-way merge is then a lane-local maximum, one 32-bit
+// warp maximum and a ballot, with no load in it; only a list that gives more than two entries
+// to the result is read again (two more entries per round trip).  Scores are compared as
+// order-preserving 32-bit integers; equal scores resolve to the lower block, which holds the
+// lower tokens, and inside a list equal scores already stand in ascending token order.
+// Lane j returns the j-th best key; (M, S) = the row's merged max and sum-exp, in all lanes.
+constexpr int kFusedMaxCtas = 160;     // partial lists per row: five per lane
+constexpr uint32_t kNotLoaded = 0xFFFFFFFFu;
 
-__device__ __forceinline__ unsigned long long merge_row_global(const Params& p, int r, float& M, float& S) {
+__device__ __forceinline__ unsigned long long merge_row_soa(const unsigned long long* __restrict__ keys,
+                                                            const float2* __restrict__ msrow, int nc, int k,
+                                                            float& M, float& S) {
   const int lane = threadIdx.x & 31;
-  const int k = p.k, nc = p.lm_ctas, R = p.R;
   constexpr int NL = kFusedMaxCtas / 32;
-  // heads and (max, sum-exp) of every block: one round trip
-  unsigned long long best_left[NL];
+  uint32_t s0[NL], s1[NL], t0[NL], t1[NL];
+  int used[NL];
   float2 ms[NL];
 #pragma unroll
   for (int q = 0; q < NL; ++q) {
     const int c = lane + 32 * q;
-    best_left[q] = 0ull;
+    unsigned long long k0 = 0ull, k1 = 0ull;
     ms[q] = make_float2(neg_inf(), 0.f);
     if (c < nc) {
-      best_left[q] = p.part_key[((size_t)c * R + r) * k];
-      ms[q] = p.part_ms[(size_t)c * R + r];
+      k0 = __ldcg(keys + c);
+      if (k > 1) k1 = __ldcg(keys + kFusedMaxCtas + c);
+      ms[q] = __ldcg(msrow + c);
     }
+    s0[q] = (uint32_t)(k0 >> 32); t0[q] = key_index(k0);
+    s1[q] = (uint32_t)(k1 >> 32); t1[q] = key_index(k1);
+    used[q] = 0;
   }
   M = neg_inf();
 #pragma unroll
@@ -127,42 +140,52 @@ __device__ __forceinline__ unsigned long long merge_row_global(const Params& p, 
   for (int q = 0; q < NL; ++q)
     if (ms[q].y > 0.f) S += ms[q].y * expf(ms[q].x - M);
   S = warp_sum(S);
-  // the k best heads: lane j takes the block that owns the j-th best
-  int my_c = -1;
-  for (int j = 0; j < k; ++j) {
-    unsigned long long best = 0ull;
-    int best_q = 0;
-#pragma unroll
-    for (int q = 0; q < NL; ++q)
-      if (best_left[q] > best) { best = best_left[q]; best_q = q; }
-    const unsigned long long wk = warp_max_key(best);
-    if (wk == 0ull) break;
-    const bool mine = best == wk;              // keys are unique: one lane
-    const int src = __ffs(__ballot_sync(kFullMask, mine)) - 1;
-    const int win_c = __shfl_sync(kFullMask, lane + 32 * best_q, src);
-    if (mine) {
-#pragma unroll
-      for (int q = 0; q < NL; ++q)
-        if (q == best_q) best_left[q] = 0ull;
-    }
-    if (lane == j) my_c = win_c;
-  }
-  // lane j's list: the first kListDepth keys in registers, refilled from global memory as it is consumed
-  const unsigned long long* list = my_c >= 0 ? p.part_key + ((size_t)my_c * R + r) * k : nullptr;
-  unsigned long long lk[kListDepth];
-#pragma unroll
-  for (int i = 0; i < kListDepth; ++i) lk[i] = (list && i < k) ? list[i] : 0ull;
-  int next = kListDepth;
+
   unsigned long long res = 0ull;
   for (int j = 0; j < k; ++j) {
-    const unsigned long long wk = warp_max_key(lk[0]);
-    if (wk == 0ull) break;
-    if (lane == j) res = wk;
-    if (lk[0] == wk) {
+    // a list whose two fetched entries are used up and which has more: fetch the next two
+    bool need = false;
 #pragma unroll
-      for (int i = 0; i + 1 < kListDepth; ++i) lk[i] = lk[i + 1];
-      lk[kListDepth - 1] = (list && next < k) ? list[next] : 0ull;
-      ++next;
+    for (int q = 0; q < NL; ++q) need |= s0[q] == kNotLoaded;
+    if (__any_sync(kFullMask, need)) {
+#pragma unroll
+      for (int q = 0; q < NL; ++q) {
+        if (s0[q] == kNotLoaded) {
+          const int c = lane + 32 * q;
+          const unsigned long long k0 = __ldcg(keys + (size_t)used[q] * kFusedMaxCtas + c);
+          const unsigned long long k1 = used[q] + 1 < k ? __ldcg(keys + (size_t)(used[q] + 1) * kFusedMaxCtas + c) : 0ull;
+          s0[q] = (uint32_t)(k0 >> 32); t0[q] = key_index(k0);
+          s1[q] = (uint32_t)(k1 >> 32); t1[q] = key_index(k1);
+        }
+      }
+    }
+    uint32_t best = s0[0];
+    int bq = 0;
+#pragma unroll
+    for (int q = 1; q < NL; ++q)
+      if (s0[q] > best) { best = s0[q]; bq = q; }      // strictly greater: the lower block wins a tie
+    const uint32_t top = __reduce_max_sync(kFullMask, best);
+    if (top == 0u) break;                              // nothing left anywhere (uniform)
+    const unsigned owners = __ballot_sync(kFullMask, best == top);
+    int src = __ffs(owners) - 1;
+    if (owners & (owners - 1u))                        // equal scores in several lanes: the lowest block
+      src = (int)__reduce_min_sync(kFullMask, best == top ? (unsigned)(lane + 32 * bq) : 0x7FFFFFFFu) & 31;
+    uint32_t tok = t0[0];
+#pragma unroll
+    for (int q = 1; q < NL; ++q)
+      if (q == bq) tok = t0[q];
+    tok = __shfl_sync(kFullMask, tok, src);
+    if (lane == j) res = ((unsigned long long)top << 32) | (unsigned long long)(0xFFFFFFFFu - tok);
+    if (lane == src) {
+#pragma unroll
+      for (int q = 0; q < NL; ++q) {
+        if (q == bq) {
+          ++used[q];
+          s0[q] = s1[q];
+          t0[q] = t1[q];
+          s1[q] = used[q] + 1 < k ? kNotLoaded : 0u;
+        }
+      }
     }
   }
   return res;
@@ -470,9 +493,8 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
       // ---- publish this block's partials: hand-over 1
       for (int r = ew; r < R; r += kEpiWarps) {
         if (!s_live[r]) continue;
-        const size_t slot = (size_t)bid * R + r;
-        if (lane < k) p.part_key[slot * k + lane] = st_key[r * k + lane];
-        if (lane == 0) p.part_ms[slot] = st_ms[r];
+        if (lane < k) fa.fkey[((size_t)r * k + lane) * kFusedMaxCtas + bid] = st_key[r * k + lane];
+        if (lane == 0) fa.fms[(size_t)r * kFusedMaxCtas + bid] = st_ms[r];
       }
       epilogue_barrier();
       if (et == 0) grid_arrive(cnt_partials);
@@ -480,6 +502,36 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
       // ---- tree work: the new beam rows this block owns
       const int P = (d == 1) ? 1 : k;
       const int base = (d == 1) ? 1 : 1 + k + (d - 2) * k * k;
+      // The books of sequence b after this pass: all P * k candidates become tree nodes, the new
+      // beam state is written for the next pass (the other parity), a stop is recorded.  Called by
+      // all epilogue threads of the block that owns the sequence's row 0; none of it is waited for
+      // until the hand-over at the end of the pass.
+      auto keep_books = [&](const int b) {
+        // this block keeps the sequence's books
+        for (int flat = et; flat < P * k; flat += kEpiThreads) {
+          const unsigned long long rec = cand_s[flat];
+          const size_t node = (size_t)b * p.Nn + base + flat;
+          p.tree_token[node] = (int)(uint32_t)rec;
+          p.tree_parent[node] = fa.beam_node[par_in * R + b * k + flat / k];
+          p.tree_cum[node] = __uint_as_float((uint32_t)(rec >> 32));
+        }
+        if (et < k) {
+          const int tok = sel_tok[et];
+          fa.beam_node[par_out * R + b * k + et] = base + sel_flat[et];
+          fa.beam_cum[par_out * R + b * k + et] = sel_cum[et];
+          fa.row_plant[par_out * R + b * k + et] = (p.plant_next && tok >= 0 && tok < p.V) ? p.plant_next[tok] : -1;
+          if (fa.io.trace.beam_sel) fa.io.trace.beam_sel[((size_t)b * p.n + (d - 1)) * k + et] = sel_flat[et];
+        }
+        if (et < P && fa.io.trace.row_lse) fa.io.trace.row_lse[((size_t)b * p.n + (d - 1)) * k + et] = lse_s[et];
+        if (et == 0) {
+          fa.io.out.H_trace[(size_t)b * p.n + (d - 1)] = __int_as_float(s_misc[1]);
+          if (s_misc[0]) {
+            p.stop_depth[b] = d;
+            p.active[b] = 0;
+            atomicSub(p.n_active, 1);
+          }
+        }
+      };
       bool waited = false;
       int cur_b = -1;
       for (int r_new = bid; r_new < R && ok; r_new += G) {
@@ -499,7 +551,8 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
           for (int pr = ew; pr < P; pr += kEpiWarps) {
             const int r = b * k + pr;
             float M, S;
-            unsigned long long res = merge_row_global(p, r, M, S);
+            unsigned long long res = merge_row_soa(fa.fkey + (size_t)r * k * kFusedMaxCtas,
+                                                   fa.fms + (size_t)r * kFusedMaxCtas, G, k, M, S);
             const int pc = s_plant[r];
             if (pc >= 0) {      // planted column: (max of the others) + delta; it was left out of the partials
               const float zc = M + p.plant_delta;
@@ -524,42 +577,28 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
           epilogue_barrier();
           // the new beam, Eq. 1 and the gate
           if (ew == 0) {
-            auto cand_key_of = [&](int idx) -> unsigned long long {
-              const unsigned long long rec = cand_s[idx];
-              return (int)(uint32_t)rec >= 0 ? make_key(__uint_as_float((uint32_t)(rec >> 32)), (uint32_t)idx) : 0ull;
-            };
-            const int n_cand = P * k;
-            unsigned long long mine = 0ull;
-            if (n_cand <= 128) {
-              unsigned long long ck[4];
-#pragma unroll
-              for (int q = 0; q < 4; ++q) ck[q] = lane + 32 * q < n_cand ? cand_key_of(lane + 32 * q) : 0ull;
-              for (int j = 0; j < k; ++j) {
-                unsigned long long best = ck[0];
-#pragma unroll
-                for (int q = 1; q < 4; ++q) best = ck[q] > best ? ck[q] : best;
-                const unsigned long long wk = warp_max_key(best);
-                if (lane == j) mine = wk;
-                if (wk == 0ull) break;
-#pragma unroll
-                for (int q = 0; q < 4; ++q)
-                  if (ck[q] == wk) ck[q] = 0ull;
+            // The k candidates of a beam row are already in descending order (same parent score,
+            // log-probabilities descending, ties by lower index), so lane p walks row p and the beam
+            // is a k-way merge of the P <= 32 rows: one 32-bit warp maximum and a ballot per entry.
+            // Equal scores go to the lower row, then the lower position: the lower candidate index.
+            int pos = 0;
+            int mine_flat = -1;
+            for (int j = 0; j < k; ++j) {
+              uint32_t hs = 0u;
+              if (lane < P && pos < k) {
+                const unsigned long long rec = cand_s[lane * k + pos];
+                if ((int)(uint32_t)rec >= 0) hs = float_to_ordered(__uint_as_float((uint32_t)(rec >> 32)));
               }
-            } else {
-              int pos = 0;
-              unsigned long long head = lane < P ? cand_key_of(lane * k) : 0ull;
-              for (int j = 0; j < k; ++j) {
-                const unsigned long long wk = warp_max_key(head);
-                if (lane == j) mine = wk;
-                if (wk == 0ull) break;
-                if (head == wk) {
-                  ++pos;
-                  head = pos < k ? cand_key_of(lane * k + pos) : 0ull;
-                }
-              }
+              const uint32_t top = __reduce_max_sync(kFullMask, hs);
+              if (top == 0u) break;
+              const int src = __ffs(__ballot_sync(kFullMask, hs == top)) - 1;
+              const int flat_j = src * k + __shfl_sync(kFullMask, pos, src);
+              if (lane == j) mine_flat = flat_j;
+              if (lane == src) ++pos;
             }
+            const unsigned long long mine = mine_flat >= 0 ? 1ull : 0ull;
             const bool have = lane < k && mine != 0ull;
-            const int flat = have ? (int)key_index(mine) : 0;
+            const int flat = have ? mine_flat : 0;
             const float cum = have ? __uint_as_float((uint32_t)(cand_s[flat] >> 32)) : neg_inf();
             const float M = __shfl_sync(kFullMask, cum, 0);
             const float sum = warp_sum(have ? expf(cum - M) : 0.f);
@@ -577,34 +616,11 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
             }
           }
           epilogue_barrier();
-          if (i == 0) {
-            // this block keeps the sequence's books
-            for (int flat = et; flat < P * k; flat += kEpiThreads) {
-              const unsigned long long rec = cand_s[flat];
-              const size_t node = (size_t)b * p.Nn + base + flat;
-              p.tree_token[node] = (int)(uint32_t)rec;
-              p.tree_parent[node] = fa.beam_node[par_in * R + b * k + flat / k];
-              p.tree_cum[node] = __uint_as_float((uint32_t)(rec >> 32));
-            }
-            if (et < k) {
-              const int tok = sel_tok[et];
-              fa.beam_node[par_out * R + b * k + et] = base + sel_flat[et];
-              fa.beam_cum[par_out * R + b * k + et] = sel_cum[et];
-              fa.row_plant[par_out * R + b * k + et] = (p.plant_next && tok >= 0 && tok < p.V) ? p.plant_next[tok] : -1;
-              if (fa.io.trace.beam_sel) fa.io.trace.beam_sel[((size_t)b * p.n + (d - 1)) * k + et] = sel_flat[et];
-            }
-            if (et < P && fa.io.trace.row_lse) fa.io.trace.row_lse[((size_t)b * p.n + (d - 1)) * k + et] = lse_s[et];
-            if (et == 0) {
-              fa.io.out.H_trace[(size_t)b * p.n + (d - 1)] = __int_as_float(s_misc[1]);
-              if (s_misc[0]) {
-                p.stop_depth[b] = d;
-                p.active[b] = 0;
-                atomicSub(p.n_active, 1);
-              }
-            }
-          }
         }
-        if (s_misc[0]) continue;                       // the sequence stops here: no draft step
+        if (s_misc[0]) {                               // the sequence stops here: no draft step
+          if (i == 0) keep_books(b);
+          continue;
+        }
         // ---- draft step of new beam row i: h = round(u / sqrt(mean(u^2) + eps)), u = h_parent + E[token]
         {
           const int tok = sel_tok[i];
@@ -615,9 +631,11 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
             // chunk q belongs to thread q mod 512; a warp's 32 chunks form one partial sum (slot q / 32)
             const int slots = cpr / 32;
             uint4 hv0 = make_uint4(0, 0, 0, 0), ev0 = hv0;
+            if (et - lane < cpr) { hv0 = hp[et]; ev0 = er[et]; }     // in flight while the books are kept
+            if (i == 0) keep_books(b);
             for (int q = et; q - lane < cpr; q += kEpiThreads) {
-              const uint4 hv = hp[q], ev = er[q];
-              if (q == et) { hv0 = hv; ev0 = ev; }
+              uint4 hv = hv0, ev = ev0;
+              if (q != et) { hv = hp[q]; ev = er[q]; }
               double u[8];
               Chunk<__nv_bfloat16>::sum(hv, ev, u);
               double ss = 0.0;
@@ -640,7 +658,9 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
               out[q] = Chunk<__nv_bfloat16>::round(u);
             }
             epilogue_barrier();                          // red_s is reused by the block's next row
-          } else if (ew == 0) {
+          } else {
+            if (i == 0) keep_books(b);
+            if (ew == 0) {
             // rows that are not a whole number of 32-chunk groups: one warp does the row
             double ss = 0.0;
             for (int c = lane; c < cpr; c += 32) {
@@ -657,6 +677,7 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
 #pragma unroll
               for (int e = 0; e < 8; ++e) u[e] *= inv;
               out[c] = Chunk<__nv_bfloat16>::round(u);
+            }
             }
           }
         }

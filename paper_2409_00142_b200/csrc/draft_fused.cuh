@@ -18,6 +18,8 @@ struct FusedArgs {
   int* beam_node;       // [2][R] tree node of each beam entry
   int* row_plant;       // [2][R] planted column of each beam row, -1 = none
   int* sync;            // [4] hand-over counters (partials, hidden rows), abort word, exit ticket
+  unsigned long long* fkey;   // [R][k][160] per-block top-k keys, position-major (entry j of all blocks together)
+  float2* fms;                // [R][160]    per-block (max, sum exp(z - max))
   int n_pad, stages, ksub, cpg, tmem_cols;
 };
 
