@@ -33,10 +33,9 @@ METRIC = "drafts_per_sec"
 UNIT = "drafts/s"
 NEG = -1e30
 FALLBACK_HBM_GBS = 6650.0
-# DRAM bytes (read + write) of one LM-head launch from the ncu capture summarised under
-# profiles/, valid only while the kernel source is the one that was profiled.
-NCU_TRAFFIC = {"llama2_7b": {"bytes": 267.5e6, "source_sha256_16": "0b876d8fed98b331",
-                             "profile": "profiles/lm_head_tc_llama2_7b.md"}}
+# DRAM bytes (read + write) of one launch of the persistent draft kernel (a full-depth draft) from the
+# ncu capture summarised under profiles/, valid only while the kernel source is the one that was profiled.
+NCU_TRAFFIC = {}
 BEAM_WIDTHS = (5, 10, 20, 50, 75, 100)      # fixed-depth-6 sweep: the widths of the paper's appendix table
 OTHER_WORKLOADS = ("vicuna_13b", "llama2_70b_b16", "llama3_8b_128k")
 CLOCK_QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
@@ -64,8 +63,9 @@ def parse_args():
                     help="skip the short runs of the other bf16 workloads (13B-, 70B-shaped, 128k vocabulary)")
     ap.add_argument("--dist-backend", default="nccl", choices=["nccl", "gloo"],
                     help="process-group backend of a multi-rank run (gloo: host-side tests of the rank logic)")
-    ap.add_argument("--launch-mode", default="graph", choices=["graph", "stream", "plain"],
-                    help="plain: ordinary stream-ordered launches, the mode profilers can follow")
+    ap.add_argument("--launch-mode", default="fused", choices=["fused", "graph", "stream", "plain"],
+                    help="fused: one persistent kernel per draft; plain: ordinary stream-ordered launches of the "
+                         "kernel-by-kernel path, which a profiler's launch list can follow")
     return ap.parse_args()
 
 
@@ -76,7 +76,7 @@ def ncu_traffic(workload: str):
         return None
     digest = hashlib.sha256()
     try:
-        for name in ("lm_head_tc.cu", "ddd_common.cuh"):      # the kernel and the row update it inlines
+        for name in ("draft_fused.cu", "tc_ptx.cuh", "ddd_common.cuh"):      # the kernel and what it inlines
             with open(os.path.join(ROOT, "paper_2409_00142_b200", "csrc", name), "rb") as f:
                 digest.update(f.read())
     except OSError:
@@ -333,7 +333,8 @@ def main():
     my_indices = S.shard_draft_indices(n_per_rank * world, rank, world)
     roots_host = stack_roots(cfg, my_indices)
     stream = torch.cuda.Stream(device)
-    mode = {"graph": P.DDD_LAUNCH_GRAPH, "stream": P.DDD_LAUNCH_STREAM, "plain": P.DDD_LAUNCH_PLAIN}[args.launch_mode]
+    mode = {"fused": P.DDD_LAUNCH_FUSED, "graph": P.DDD_LAUNCH_GRAPH, "stream": P.DDD_LAUNCH_STREAM,
+            "plain": P.DDD_LAUNCH_PLAIN}[args.launch_mode]
     peak, peak_kind = measured_peak()
     elt = 4 if cfg.dtype == "fp32" else 2
     w_bytes = cfg.vocab * cfg.hidden * elt
@@ -362,7 +363,10 @@ def main():
         lm_us, lm_iso_us = time_lm_head(eng, args.lm_head_reps, stream, device, flush)
         achieved = w_bytes / (lm_us * 1e-6) / 1e9
 
-        def variant(c, launch=P.DDD_LAUNCH_GRAPH, w=None):
+        def variant(c, launch=None, w=None):
+            launch = mode if launch is None else launch
+            if launch == P.DDD_LAUNCH_FUSED and c.k > 32:
+                launch = P.DDD_LAUNCH_GRAPH          # beams wider than 32 run kernel by kernel
             return P.DraftEngine(c, w or dev_weights, device=local, launch_mode=launch, with_trace=False)
 
         # ---- fixed full depth (x = -inf): per-expansion-step time independent of where drafts stop
@@ -496,20 +500,40 @@ def main():
         dist_teardown(world)
         return
 
-    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "traffic": ncu_traffic(cfg.name), "peak_kind": f"of {peak_kind}",
-                "kernel": "lm_head", "us_per_launch": lm_us,
-                "us_per_launch_kind": "period of back-to-back launches (set-up and first loads overlap the predecessor)",
-                "us_per_launch_isolated": lm_iso_us, "frac_isolated": w_bytes / (lm_iso_us * 1e-6) / 1e9 / peak,
-                "algorithmic_bytes_per_launch": w_bytes,
-                "frac_of_8TBs_nominal": achieved / 8000.0, "blocks": blocks,
-                # the whole draft against the same peak: W bytes of the passes a draft needs / time per draft
-                "draft_frac": passes_mean * w_bytes / (us_per_draft * 1e-6) / 1e9 / peak}
-    if step_us is not None:
-        # the expansion step (LM head + select / gate / draft step) at full depth: the figure the
-        # 70-%-of-HBM-bandwidth target is stated on
-        roofline["step_frac"] = w_bytes / (step_us * 1e-6) / 1e9 / peak
-        roofline["step_frac_of_8TBs_nominal"] = w_bytes / (step_us * 1e-6) / 1e9 / 8000.0
+    lm_head_alone = {"kernel": "lm_head_tc_kernel (one pass per launch)", "achieved": achieved, "frac": achieved / peak,
+                     "us_per_launch": lm_us,
+                     "us_per_launch_kind": "period of back-to-back launches (set-up and first loads overlap the predecessor)",
+                     "us_per_launch_isolated": lm_iso_us, "frac_isolated": w_bytes / (lm_iso_us * 1e-6) / 1e9 / peak,
+                     "algorithmic_bytes_per_launch": w_bytes, "frac_of_8TBs_nominal": achieved / 8000.0}
+    # the whole draft against the same peak: W bytes of the passes a draft needs / time per draft
+    draft_frac = passes_mean * w_bytes / (us_per_draft * 1e-6) / 1e9 / peak
+    if args.launch_mode == "fused" and step_us is not None:
+        # One launch of the persistent kernel is a whole draft, so the dominant kernel is timed on
+        # full-depth drafts (x = -inf): n passes, each streaming W once.  The events bracket whole
+        # drafts, i.e. they include the small rerank kernel behind every launch.
+        fused_bytes = cfg.max_depth * w_bytes
+        fused_us = step_us * cfg.max_depth
+        fused_gbs = fused_bytes / (fused_us * 1e-6) / 1e9
+        roofline = {"bound": "hbm", "achieved": fused_gbs, "peak": peak, "unit": "GB/s", "frac": fused_gbs / peak,
+                    "traffic": ncu_traffic(cfg.name), "peak_kind": f"of {peak_kind}",
+                    "kernel": "draft_fused_kernel (%d expansion steps per launch, full-depth drafts)" % cfg.max_depth,
+                    "us_per_launch": fused_us, "algorithmic_bytes_per_launch": fused_bytes,
+                    "frac_of_8TBs_nominal": fused_gbs / 8000.0, "blocks": blocks,
+                    "step_frac": fused_gbs / peak, "step_frac_of_8TBs_nominal": fused_gbs / 8000.0,
+                    "draft_frac": draft_frac, "lm_head_alone": lm_head_alone}
+    else:
+        roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                    "frac": achieved / peak, "traffic": None, "peak_kind": f"of {peak_kind}",
+                    "kernel": "lm_head", "us_per_launch": lm_us,
+                    "us_per_launch_kind": lm_head_alone["us_per_launch_kind"],
+                    "us_per_launch_isolated": lm_iso_us, "frac_isolated": lm_head_alone["frac_isolated"],
+                    "algorithmic_bytes_per_launch": w_bytes,
+                    "frac_of_8TBs_nominal": achieved / 8000.0, "blocks": blocks, "draft_frac": draft_frac}
+        if step_us is not None:
+            # the expansion step (LM head + select / gate / draft step) at full depth: the figure the
+            # 70-%-of-HBM-bandwidth target is stated on
+            roofline["step_frac"] = w_bytes / (step_us * 1e-6) / 1e9 / peak
+            roofline["step_frac_of_8TBs_nominal"] = w_bytes / (step_us * 1e-6) / 1e9 / 8000.0
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
