@@ -403,7 +403,8 @@ int ddd_create(const ddd_config* cfg, const void* W, const void* E, const float*
     if (prop.major != 10) rc = DDD_ERR_UNSUPPORTED;
     const bool fused = cfg->launch_mode == DDD_LAUNCH_FUSED;
     if (rc == DDD_OK && fused && cfg->k > 32) rc = DDD_ERR_UNSUPPORTED;
-    if (rc == DDD_OK) rc = tc_plan_create(p, h->sm_count, ws + L.w_packed, &h->tc, fused ? fused_extra_smem(cfg->k) : 0);
+    const int atiles = fused && cfg->k <= 32 && fused_pair_mode(p, h->sm_count) ? 2 : 1;
+    if (rc == DDD_OK) rc = tc_plan_create(p, h->sm_count, ws + L.w_packed, &h->tc, fused ? fused_extra_smem(cfg->k) : 0, atiles);
     if (rc == DDD_OK) p.lm_ctas = h->tc.ctas;
     if (rc == DDD_OK && fused) rc = fused_prepare(p, h->tc);
   } else if (rc == DDD_OK && cfg->launch_mode == DDD_LAUNCH_FUSED) {

@@ -200,7 +200,10 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
   unsigned char* smem = reinterpret_cast<unsigned char*>(
       (reinterpret_cast<uintptr_t>(smem_dyn) + 1023u) & ~static_cast<uintptr_t>(1023u));
   const int stages = fa.stages, ksub = fa.ksub, n_pad = fa.n_pad, cpg = fa.cpg;
-  const SmemPlan sp = smem_plan(stages, ksub, n_pad, p.R, p.k, cpg);
+  // pair mode: a block's two tiles share every stage, so the hidden rows cross from L2 once per pass
+  // instead of once per tile (what bounds a pass with many beam rows is L2 -> SM traffic)
+  const int pair = fa.pair;
+  const SmemPlan sp = smem_plan(stages, ksub, n_pad, p.R, p.k, cpg, pair ? 2 : 1);
   const TreeSmem ts = tree_smem(p.k);
   // The tree work's scratch lies over the epilogue's transpose buffer, which is idle between the
   // last tile of a pass and the first of the next (behind everything else where it is too large).
@@ -245,8 +248,9 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
   const int unit0 = bid * base_units + (bid < rem_units ? bid : rem_units);
   const int n_tiles = (my_units + 3) / 4;
   const int num_kb = p.Hd / (kBlockK * ksub);
-  const uint32_t a_stage = (uint32_t)ksub * kABytes, b_stage = (uint32_t)ksub * b_bytes;
-  const int total_iters = n_tiles * num_kb;                        // pipeline steps per pass
+  const uint32_t a_kblock = pair ? 2u * kABytes : (uint32_t)kABytes;     // bytes of W per K-block of a stage
+  const uint32_t a_stage = (uint32_t)ksub * a_kblock, b_stage = (uint32_t)ksub * b_bytes;
+  const int total_iters = pair ? num_kb : n_tiles * num_kb;         // pipeline steps per pass
   const int prefill = total_iters < stages ? total_iters : stages;
 
   if (threadIdx.x == 0) {
@@ -306,15 +310,16 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
     uint32_t itg = 0;                // pipeline steps issued since the start of the draft
     bool ok = true;
     auto issue_w = [&](int i, int stage) {
-      const int t = i / num_kb, kb = i - t * num_kb;
-      const int nu = min(4, my_units - 4 * t);
+      // step i of a pass: tile t, K-group kb - or, in pair mode, K-group i of all the block's units
+      const int t = pair ? 0 : i / num_kb, kb = pair ? i : i - t * num_kb;
+      const int nu = pair ? my_units : min(4, my_units - 4 * t);
       const uint32_t full = bar_full + 8u * stage;
       if (lane == 0) mbar_expect_tx(full, (uint32_t)ksub * ((uint32_t)nu * kUnitBytes + b_bytes));
       __syncwarp();
       const unsigned char* src = fa.w_packed + ((size_t)(kb * ksub) * n_units + (size_t)(unit0 + 4 * t)) * kUnitBytes;
       const uint32_t dst = a_base + (uint32_t)stage * a_stage;
       if (lane < ksub)
-        bulk_load_hint(dst + (uint32_t)lane * kABytes, src + (size_t)lane * n_units * kUnitBytes,
+        bulk_load_hint(dst + (uint32_t)lane * a_kblock, src + (size_t)lane * n_units * kUnitBytes,
                        (uint32_t)nu * kUnitBytes, full, evict_first);
     };
     auto issue_h = [&](const CUtensorMap* map, int i, int stage) {
@@ -343,7 +348,7 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
       // block, 38 MB in all) take 0.9 us off a pass, 24 already lose again (the burst delays the
       // loads of the tree work), and pass 1 has no tree work to hide behind.
       if (ok && d > 1) {
-        const int nu0 = min(4, my_units);
+        const int nu0 = pair ? my_units : min(4, my_units);
         const int kb_first = prefill * ksub;
         const int kb_last = min(p.Hd / kBlockK, kb_first + kL2AheadKBlocks);
         for (int kb64 = kb_first + lane; kb64 < kb_last; kb64 += 32)
@@ -403,6 +408,41 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
     for (int d = 1; d <= p.n && ok; ++d) {
       ok = __all_sync(kFullMask, mbar_wait(bar_pass, (uint32_t)(d - 1) & 1u, abort_flag, p.dev_status));
       if (!ok || s_pass_state[(d - 1) & 1] == 0) break;
+      if (pair) {
+        // both tiles at once: accumulator 0 takes units 0-3, accumulator 1 units 4-7, every stage feeds both
+        for (int a2 = 0; a2 < 2 && ok; ++a2)
+          ok = __all_sync(kFullMask, mbar_wait(bar_tempty + 8u * a2, (((tg + a2) >> 1) & 1u) ^ 1u, abort_flag, p.dev_status));
+        if (!ok) break;
+        tc_fence_after();
+        for (int kb = 0; kb < num_kb; ++kb, ++itg) {
+          const int stage = (int)(itg % stages);
+          ok = __all_sync(kFullMask, mbar_wait(bar_full + 8u * stage, (itg / stages) & 1u, abort_flag, p.dev_status));
+          if (!ok) break;
+          tc_fence_after();
+          if (lane == 0) {
+            for (int kk = 0; kk < ksub; ++kk) {
+              const uint32_t a_addr = a_base + (uint32_t)stage * a_stage + (uint32_t)kk * a_kblock;
+              const uint32_t b_addr = b_base + (uint32_t)stage * b_stage + (uint32_t)kk * b_bytes;
+#pragma unroll
+              for (int k4 = 0; k4 < kBlockK / kUmmaK; ++k4) {
+                const unsigned long long bd = make_smem_desc(b_addr + k4 * kUmmaK * 2);
+                const uint32_t accum = (kb | kk | k4) != 0 ? 1u : 0u;
+                tc_mma_bf16(tmem_base, make_smem_desc(a_addr + k4 * kUmmaK * 2), bd, idesc, accum);
+                tc_mma_bf16(tmem_base + (uint32_t)n_pad, make_smem_desc(a_addr + kABytes + k4 * kUmmaK * 2), bd, idesc, accum);
+              }
+            }
+            tc_commit(bar_empty + 8u * stage);
+          }
+          __syncwarp();
+        }
+        if (ok && lane == 0) {
+          tc_commit(bar_tfull);
+          tc_commit(bar_tfull + 8u);
+        }
+        __syncwarp();
+        tg += 2;
+        continue;
+      }
       for (int t = 0; t < n_tiles && ok; ++t, ++tg) {
         const int acc = (int)(tg & 1u);
         ok = __all_sync(kFullMask, mbar_wait(bar_tempty + 8u * acc, ((tg >> 1) & 1u) ^ 1u, abort_flag, p.dev_status));
@@ -754,6 +794,13 @@ bool fused_supported(const Params& p) {
   return p.dtype == DDD_DTYPE_BF16 && p.Hd % kBlockK == 0 && p.k <= kNarrowK && p.lm_ctas <= kFusedMaxCtas;
 }
 
+bool fused_pair_mode(const Params& p, int sm_count) {
+  const int n_units = (p.Vl + kUnitRows - 1) / kUnitRows;
+  const int ctas = sm_count < n_units ? sm_count : n_units;
+  const int lo = n_units / ctas, hi = lo + (n_units % ctas ? 1 : 0);
+  return p.R >= 48 && lo >= 5 && hi <= 8 && 2 * ((p.R + 15) / 16 * 16) <= 512;
+}
+
 int fused_prepare(const Params& p, const TcPlan& plan) {
   if (!fused_supported(p)) return DDD_ERR_UNSUPPORTED;
   if (allow_max_dynamic_smem(draft_fused_kernel) != cudaSuccess) return DDD_ERR_CUDA;
@@ -779,6 +826,7 @@ cudaError_t launch_draft_fused(const Params& p, const TcPlan& plan, const FusedA
   fa.stages = plan.stages;
   fa.ksub = plan.ksub;
   fa.cpg = plan.epi_chunks;
+  fa.pair = plan.atiles == 2 ? 1 : 0;
   fa.tmem_cols = plan.tmem_cols;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)plan.ctas, 1, 1);

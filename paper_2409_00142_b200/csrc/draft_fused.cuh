@@ -21,10 +21,14 @@ struct FusedArgs {
   unsigned long long* fkey;   // [R][k][160] per-block top-k keys, position-major (entry j of all blocks together)
   float2* fms;                // [R][160]    per-block (max, sum exp(z - max))
   int n_pad, stages, ksub, cpg, tmem_cols;
+  int pair;             // both tiles of a block share each stage (one fetch of the hidden rows per pass)
 };
 
 // Shared memory the tree work needs behind the LM-head pipeline's own.
 int fused_extra_smem(int k);
+// Should a block feed both of its tiles from one fetch of the hidden rows?  Needs every block to own
+// exactly two tiles (5 to 8 units of 32 vocabulary rows) and pays off once the hidden rows weigh: from 48 beam rows.
+bool fused_pair_mode(const Params& p, int sm_count);
 // Can this configuration run as one kernel (bf16, tensor-core kernel, beam width up to 32)?
 bool fused_supported(const Params& p);
 // Checks that all blocks fit on the device at once and sets the kernels' attributes.  DDD_* code.

@@ -171,10 +171,11 @@ struct SmemPlan {
 // rounded up to whole lanes of four (the wide-list layout).
 __host__ __device__ inline int key_stride(int k) { return k <= kNarrowK ? k : (k + 3) & ~3; }
 
-__host__ __device__ inline SmemPlan smem_plan(int stages, int ksub, int n_pad, int R, int k, int cpg) {
+// atiles: 128-row tiles of W a stage holds per K-block (2 when a block feeds both of its tiles from one fetch of h)
+__host__ __device__ inline SmemPlan smem_plan(int stages, int ksub, int n_pad, int R, int k, int cpg, int atiles = 1) {
   SmemPlan s;
   int off = 0;
-  s.a = off; off += stages * ksub * kABytes;
+  s.a = off; off += stages * ksub * atiles * kABytes;
   s.b = off; off += stages * ksub * n_pad * kBlockK * 2;
   s.zt = off; off += cpg * kChunkCols * kTile * 4;
   s.key = off; off += R * key_stride(k) * 8;

@@ -381,6 +381,26 @@ def test_fused_draft_equals_kernel_by_kernel_draft(case):
         assert depths == {cfg.max_depth}
 
 
+@pytest.mark.parametrize("vocab", [24000 + 8, 37000 - 3])
+def test_fused_draft_with_both_tiles_of_a_block_sharing_a_stage(vocab):
+    # from 48 beam rows on, and where every block owns five to eight 32-row units (two tiles), the
+    # persistent kernel feeds both tiles from one fetch of the hidden rows: 751 units = 5-6 per block
+    # of a 148-SM device, 1157 units = 7-8
+    cfg = S.scaled_down(S.CONFIGS["llama2_70b_b16"], 256, vocab, batch=5, threshold=-3.0, max_depth=4)
+    eng_s = engine_for(cfg, TC, P.DDD_LAUNCH_STREAM)
+    eng_f = engine_for(cfg, TC, P.DDD_LAUNCH_FUSED)
+    for i in range(3):
+        roots = S.make_roots(cfg, i)
+        a = parity.run_gpu(eng_s, roots)
+        b = parity.run_gpu(eng_f, roots)
+        for name in ("stop_depth", "n_out", "token", "parent", "depth", "position", "cum", "mask", "node_id",
+                     "tree_token", "tree_parent", "tree_cum"):
+            np.testing.assert_array_equal(a[name], b[name], err_msg=name)
+        parity.compare_with_oracle(cfg, weights_for(cfg), roots, b)
+    eng_s.close()
+    eng_f.close()
+
+
 def test_fused_mode_is_refused_where_it_cannot_run():
     base = S.scaled_down(S.CONFIGS["llama2_7b"], 256, 3000, threshold=NEG, max_depth=2, total_tokens=20)
     for cfg, kernel in ((base.replace(k=33), TC), (S.CONFIGS["tiny"], P.DDD_LM_HEAD_AUTO), (base, SIMT)):
