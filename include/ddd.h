@@ -23,8 +23,10 @@
  * Conventions
  *   - Every pointer argument says whether it is a HOST or a DEVICE pointer.  The library
  *     never allocates device memory: weights, workspace, inputs and outputs are allocated by
- *     the caller and only borrowed.  W, E, bias, plant_next and the workspace must stay valid
- *     and unchanged until ddd_destroy.
+ *     the caller and only borrowed.  E, bias, plant_next and the workspace must stay valid
+ *     and unchanged until ddd_destroy.  So must W for the CUDA-core kernel (DDD_LM_HEAD_SIMT,
+ *     every fp32 handle); a handle on the tensor-core kernel reads W only inside ddd_create,
+ *     which packs it into the workspace, and the caller may free or reuse W afterwards.
  *   - All functions return DDD_OK (0) or a negative DDD_ERR_* code; nothing throws, traps or
  *     aborts.  ddd_strerror maps a code to a static string.
  *   - ddd_draft only enqueues work on the given stream.  Outputs are valid once that stream

@@ -249,6 +249,9 @@ class DraftEngine:
     """Owns the torch buffers one handle needs: device copies of the weights, the workspace
     and one set of output / trace tensors.  All computation happens inside the library."""
 
+    GUARD_BYTES = 4096
+    GUARD_PATTERN = 0xA5
+
     def __init__(self, cfg, weights: Dict, device: int = 0, lm_head_kernel: int = DDD_LM_HEAD_AUTO,
                  launch_mode: int = DDD_LAUNCH_STREAM, with_trace: bool = True, vocab_slice=None):
         """vocab_slice = (begin, count): this engine owns only those rows of the LM head (one rank
@@ -280,8 +283,13 @@ class DraftEngine:
         nbytes = ddd_workspace_bytes(self.c)
         if nbytes == 0:
             raise DddError(-1, "ddd_workspace_bytes")
-        self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=dev)
-        ws_ptr = (self.workspace.data_ptr() + 255) // 256 * 256
+        # the workspace sits between two guard bands filled with a pattern: a kernel that wrote outside
+        # what ddd_workspace_bytes promised shows up in guards_intact()
+        guard = self.GUARD_BYTES
+        self.workspace = torch.full((nbytes + 256 + 2 * guard,), self.GUARD_PATTERN, dtype=torch.uint8, device=dev)
+        ws_ptr = (self.workspace.data_ptr() + guard + 255) // 256 * 256
+        self._ws_offset = ws_ptr - self.workspace.data_ptr()
+        self._ws_bytes = nbytes
         self.handle = ddd_create(self.c, self.W.data_ptr(), self.E.data_ptr(),
                                  None if self.bias is None else self.bias.data_ptr(),
                                  None if self.plant_next is None else self.plant_next.data_ptr(),
@@ -376,6 +384,12 @@ class DraftEngine:
     def shard_select(self, d: int, records, slots: int, flags=None) -> None:
         ddd_shard_select(self.handle, d, records.data_ptr(), slots,
                          None if flags is None else flags.data_ptr(), self.stream_ptr())
+
+    def guards_intact(self) -> bool:
+        """True while the bytes just before and just after the workspace still hold their pattern."""
+        before = self.workspace[:self._ws_offset]
+        after = self.workspace[self._ws_offset + self._ws_bytes:]
+        return bool((before == self.GUARD_PATTERN).all().item()) and bool((after == self.GUARD_PATTERN).all().item())
 
     def lm_head_pass(self) -> None:
         ddd_lm_head_pass(self.handle, self.stream_ptr())

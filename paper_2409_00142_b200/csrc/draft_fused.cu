@@ -58,35 +58,6 @@ __host__ __device__ inline TreeSmem tree_smem(int k) {
   return t;
 }
 
-__device__ __forceinline__ int ld_acquire(const int* p) {
-  int v;
-  asm volatile("ld.acquire.gpu.global.b32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-  return v;
-}
-__device__ __forceinline__ int ld_relaxed(const int* p) {
-  int v;
-  asm volatile("ld.relaxed.gpu.global.b32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-  return v;
-}
-
-// Waits until *counter >= target (every block adds one per hand-over; the counters only grow
-// during a draft).  False if the wait ran out or another block gave up.
-__device__ __forceinline__ bool grid_wait(const int* counter, int target, int* abort_word, int* status) {
-  unsigned long long t0 = 0;
-  for (uint32_t it = 0;; ++it) {
-    if (ld_acquire(counter) >= target) return true;
-    if ((it & 15u) == 15u) {
-      if (ld_relaxed(abort_word) != 0) return false;
-      const unsigned long long now = global_timer();
-      if (t0 == 0) t0 = now;
-      else if (now - t0 > kWaitLimitNs) {
-        atomicCAS(status, DDD_OK, DDD_ERR_TIMEOUT);
-        atomicExch(abort_word, 1);
-        return false;
-      }
-    }
-  }
-}
 // One arrival of this block at a hand-over: the caller has synchronised the threads whose writes
 // the other blocks are to see.
 __device__ __forceinline__ void grid_arrive(int* counter) {

@@ -56,9 +56,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait.  Returns false if the wait ran out of time or another role already gave up.
+// Bounded wait.  Returns false if the wait ran out of time (limit_ns by %globaltimer) or another
+// role already gave up; a wait that runs out records DDD_ERR_TIMEOUT and raises the block's flag.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
-                                          bool heed_abort = true) {
+                                          bool heed_abort = true, unsigned long long limit_ns = kWaitLimitNs) {
   unsigned long long t0 = 0;
   for (uint32_t it = 0;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
@@ -66,9 +67,39 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       if (heed_abort && *abort_flag) return false;
       const unsigned long long now = global_timer();
       if (t0 == 0) t0 = now;
-      else if (now - t0 > kWaitLimitNs) {
+      else if (now - t0 > limit_ns) {
         atomicCAS(status, DDD_OK, DDD_ERR_TIMEOUT);
         *abort_flag = 1;
+        return false;
+      }
+    }
+  }
+}
+__device__ __forceinline__ int ld_acquire_gpu(const int* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.b32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ int ld_relaxed_gpu(const int* p) {
+  int v;
+  asm volatile("ld.relaxed.gpu.global.b32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+// Grid-wide hand-over: waits until *counter >= target (every block adds one per hand-over; the
+// counters only grow during a launch).  False if the wait ran out - DDD_ERR_TIMEOUT is recorded
+// and the grid-wide abort word raised - or another block gave up.
+__device__ __forceinline__ bool grid_wait(const int* counter, int target, int* abort_word, int* status,
+                                          unsigned long long limit_ns = kWaitLimitNs) {
+  unsigned long long t0 = 0;
+  for (uint32_t it = 0;; ++it) {
+    if (ld_acquire_gpu(counter) >= target) return true;
+    if ((it & 15u) == 15u) {
+      if (ld_relaxed_gpu(abort_word) != 0) return false;
+      const unsigned long long now = global_timer();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > limit_ns) {
+        atomicCAS(status, DDD_OK, DDD_ERR_TIMEOUT);
+        atomicExch(abort_word, 1);
         return false;
       }
     }

@@ -25,6 +25,7 @@ def run_gpu(engine, roots):
     engine.draft(dev["root_hidden"], dev["root_token"], dev["root_pos"])
     res = engine.results()
     assert int(res["status"][0]) == 0, f"device status {int(res['status'][0])}"
+    assert engine.guards_intact(), "a kernel wrote outside the workspace"
     return {k: v.numpy() for k, v in res.items()}
 
 

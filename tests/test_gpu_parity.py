@@ -401,6 +401,19 @@ def test_fused_draft_with_both_tiles_of_a_block_sharing_a_stage(vocab):
     eng_f.close()
 
 
+@pytest.mark.parametrize("mode", [P.DDD_LAUNCH_STREAM, P.DDD_LAUNCH_FUSED], ids=["stream", "fused"])
+def test_w_may_be_released_after_create_on_the_tensor_core_path(mode):
+    # ddd_create packs W into the workspace; nothing on the tensor-core path reads the original again
+    cfg = small_cases()["7b"]
+    eng = engine_for(cfg, TC, mode)
+    eng.W.fill_(float("nan"))
+    torch.cuda.synchronize()
+    roots = S.make_roots(cfg, 2)
+    g = parity.run_gpu(eng, roots)
+    parity.compare_with_oracle(cfg, weights_for(cfg), roots, g)
+    eng.close()
+
+
 def test_fused_mode_is_refused_where_it_cannot_run():
     base = S.scaled_down(S.CONFIGS["llama2_7b"], 256, 3000, threshold=NEG, max_depth=2, total_tokens=20)
     for cfg, kernel in ((base.replace(k=33), TC), (S.CONFIGS["tiny"], P.DDD_LM_HEAD_AUTO), (base, SIMT)):
