@@ -73,7 +73,8 @@ enum { DDD_LM_HEAD_AUTO = 0, DDD_LM_HEAD_SIMT = 1, DDD_LM_HEAD_TCGEN05 = 2 };
  * kernel by kernel in ordinary stream order, one after the other: the slowest, and the one
  * profilers can follow.  FUSED runs the whole draft as ONE persistent kernel of one thread block
  * per SM (a cooperative launch) that loops over the passes itself and hands over between them
- * through counters in global memory, followed by one small kernel for the rerank and the mask:
+ * through counters in global memory; the rerank and the mask run inside it too where the tree
+ * fits the kernel's spare shared memory, else in one small kernel behind it:
  * the fastest, for bf16 handles on the tensor-core kernel with a beam of at most 32
  * (ddd_create returns DDD_ERR_UNSUPPORTED otherwise); nothing else should run on the device
  * meanwhile, since its blocks occupy every SM until the draft ends. */

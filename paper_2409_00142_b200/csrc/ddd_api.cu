@@ -677,7 +677,8 @@ int ddd_launches_per_draft(const ddd_handle* h, int32_t passes_needed) {
   if (!h) return DDD_ERR_INVALID_ARG;
   const int n = h->p.n;
   int passes = n;
-  if (h->cfg.launch_mode == DDD_LAUNCH_FUSED) return 2;     // the draft kernel and the rerank kernel
+  if (h->cfg.launch_mode == DDD_LAUNCH_FUSED)      // the draft kernel and, where the rerank does not fit in it, the rerank kernel
+    return fused_rerank_mode(h->p, h->tc) ? 1 : 2;
   if (h->cfg.launch_mode == DDD_LAUNCH_GRAPH) {
     const int nb = h->have_graph ? h->graph_bounds : h->n_bounds;
     for (int j = nb - 1; j >= 0; --j)

@@ -38,6 +38,7 @@ namespace {
 using namespace tc;
 
 constexpr int kTreeOverZt = kChunkCols * kTile * 4;     // smallest transpose buffer of the epilogue (8 KB)
+constexpr int kMaxStoppedPerBlock = 8;                  // sequences one block may keep the books of
 constexpr int kL2AheadKBlocks = 16;                     // K-blocks of W requested into L2 ahead of a pass
 
 struct TreeSmem {
@@ -163,6 +164,17 @@ __device__ __forceinline__ unsigned long long merge_row_soa(const unsigned long 
   return res;
 }
 
+struct EpiSync {      // the 16 epilogue warps on their named barrier
+  __device__ static __forceinline__ void sync() { epilogue_barrier(); }
+};
+
+__device__ __forceinline__ void rerank_in_epilogue(const Params& p, const DraftIO& io, int b, int D, int et,
+                                                bool keys_in_smem, unsigned char* rr, int cap, int* scratch,
+                                                short* out_parent) {
+  if (keys_in_smem) rerank_mask_impl<kEpiThreads, true, EpiSync>(p, io, b, D, false, et, rr, cap, scratch, out_parent);
+  else rerank_mask_impl<kEpiThreads, false, EpiSync>(p, io, b, D, false, et, rr, cap, scratch, out_parent);
+}
+
 // ---------------------------------------------------------------------------- kernel
 __global__ void __launch_bounds__(kTcThreads, 1)
 draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ CUtensorMap map_h0,
@@ -196,6 +208,8 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
   volatile int* s_misc = reinterpret_cast<volatile int*>(tree_base + ts.misc);    // [0] stop, [1] H bits
   __shared__ int s_pass_state[2];      // what the producer learnt at hand-over 2: pass number to run, or 0 = leave
   __shared__ __align__(8) unsigned long long s_bar_spare;   // end of the MMAs when the block gives up
+  __shared__ int s_stopped[kMaxStoppedPerBlock];            // sequences of this block's books that stopped in this pass
+  __shared__ int s_nstopped;
 
   const uint32_t a_base = smem_u32(smem + sp.a), b_base = smem_u32(smem + sp.b);
   const uint32_t b_bytes = (uint32_t)n_pad * kBlockK * 2;
@@ -237,6 +251,7 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
     mbar_init(bar_spare, 1);
     *abort_flag = 0;
     s_pass_state[0] = s_pass_state[1] = 0;
+    s_nstopped = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -552,6 +567,7 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
             p.stop_depth[b] = d;
             p.active[b] = 0;
             atomicSub(p.n_active, 1);
+            if (s_nstopped < kMaxStoppedPerBlock) s_stopped[s_nstopped++] = b;
           }
         }
       };
@@ -598,6 +614,17 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
             if (lane == 0) lse_s[pr] = lse;
           }
           epilogue_barrier();
+          // While one warp picks the beam, idle warps ask L2 for the embedding rows of this block's
+          // share of the candidates (the k blocks of a sequence cover all k * k between them), so that
+          // the draft step's gather finds them there: -1.2 us per pass on the 7B shape.
+          if (ew >= 12 && d < p.n) {
+            const int n_cand = P * k;
+            for (int flat = i + k * ((ew - 12) * 32 + lane); flat < n_cand; flat += k * 128) {
+              const int tokc = (int)(uint32_t)cand_s[flat];
+              if (tokc >= 0 && tokc < p.V)
+                l2_prefetch(static_cast<const unsigned char*>(p.E) + (size_t)tokc * p.Hd * 2, (uint32_t)p.Hd * 2);
+            }
+          }
           // the new beam, Eq. 1 and the gate
           if (ew == 0) {
             // The k candidates of a beam row are already in descending order (same parent score,
@@ -710,6 +737,23 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
       epilogue_barrier();
       if (et == 0) grid_arrive(cnt_hidden);
     }
+    // ---- the sequences whose books this block kept are finished here, after the last pass, where
+    // nobody waits for it: rerank to m nodes, rows, parents, positions, mask.  The transpose buffer
+    // is free now and holds keys, rows and scratch.
+    if (ok && fa.rerank_inside) {
+      epilogue_barrier();
+      const int cap = p.Nn;
+      unsigned char* rr = smem + sp.zt;
+      const size_t node_bytes = (size_t)cap * (fa.rerank_inside == 1 ? 6 : 2);
+      int* scratch = reinterpret_cast<int*>(rr + ((node_bytes + 7) / 8) * 8);
+      short* out_parent = reinterpret_cast<short*>(scratch + kRerankScratchInts);
+      const int n_stopped = s_nstopped;
+      for (int q = 0; q < n_stopped; ++q) {
+        const int b = s_stopped[q];
+        rerank_in_epilogue(p, fa.io, b, p.stop_depth[b], et, fa.rerank_inside == 1, rr, cap, scratch, out_parent);
+        epilogue_barrier();
+      }
+    }
     if (!ok && et == 0) *abort_flag = 1;
   }
 
@@ -729,6 +773,7 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
     if (*abort_flag) atomicExch(abort_word, 1);
     __threadfence();
     if (atomicAdd(exit_ticket, 1) == G - 1) {
+      if (fa.rerank_inside) *fa.io.out.status = *reinterpret_cast<volatile int*>(p.dev_status);
       atomicExch(cnt_partials, 0);
       atomicExch(cnt_hidden, 0);
       atomicExch(abort_word, 0);
@@ -772,6 +817,17 @@ bool fused_pair_mode(const Params& p, int sm_count) {
   return p.R >= 48 && lo >= 5 && hi <= 8 && 2 * ((p.R + 15) / 16 * 16) <= 512;
 }
 
+// Can the rerank run inside the draft kernel, in the epilogue's transpose buffer?  1: with the
+// tree's keys in shared memory, 2: keys read from global memory, 0: no (rerank_kernel follows).
+int fused_rerank_mode(const Params& p, const TcPlan& plan) {
+  const size_t room = (size_t)plan.epi_chunks * kChunkCols * kTile * 4;
+  const size_t fixed = 8 + kRerankScratchInts * sizeof(int) + (size_t)p.T * sizeof(short);
+  if ((size_t)p.R > (size_t)kMaxStoppedPerBlock * plan.ctas) return 0;
+  if ((size_t)p.Nn * 6 + fixed <= room) return 1;
+  if ((size_t)p.Nn * 2 + fixed <= room) return 2;
+  return 0;
+}
+
 int fused_prepare(const Params& p, const TcPlan& plan) {
   if (!fused_supported(p)) return DDD_ERR_UNSUPPORTED;
   if (allow_max_dynamic_smem(draft_fused_kernel) != cudaSuccess) return DDD_ERR_CUDA;
@@ -798,6 +854,7 @@ cudaError_t launch_draft_fused(const Params& p, const TcPlan& plan, const FusedA
   fa.ksub = plan.ksub;
   fa.cpg = plan.epi_chunks;
   fa.pair = plan.atiles == 2 ? 1 : 0;
+  fa.rerank_inside = fused_rerank_mode(p, plan);
   fa.tmem_cols = plan.tmem_cols;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)plan.ctas, 1, 1);
@@ -810,7 +867,7 @@ cudaError_t launch_draft_fused(const Params& p, const TcPlan& plan, const FusedA
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   cudaError_t e = cudaLaunchKernelEx(&cfg, draft_fused_kernel, p, fa, plan.map_h[0], plan.map_h[1]);
-  if (e != cudaSuccess) return e;
+  if (e != cudaSuccess || fa.rerank_inside) return e;
   // rerank + mask: started early (programmatic dependent launch), waits on the device for the draft
   bool keys;
   cudaLaunchConfig_t rc = {};

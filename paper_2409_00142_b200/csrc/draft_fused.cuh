@@ -21,6 +21,7 @@ struct FusedArgs {
   unsigned long long* fkey;   // [R][k][160] per-block top-k keys, position-major (entry j of all blocks together)
   float2* fms;                // [R][160]    per-block (max, sum exp(z - max))
   int n_pad, stages, ksub, cpg, tmem_cols;
+  int rerank_inside;    // the rerank runs inside the draft kernel (1: keys in shared memory, 2: from global memory)
   int pair;             // both tiles of a block share each stage (one fetch of the hidden rows per pass)
 };
 
@@ -33,7 +34,8 @@ bool fused_pair_mode(const Params& p, int sm_count);
 bool fused_supported(const Params& p);
 // Checks that all blocks fit on the device at once and sets the kernels' attributes.  DDD_* code.
 int fused_prepare(const Params& p, const TcPlan& plan);
-// Enqueues the draft kernel and, behind it, the rerank kernel.
+int fused_rerank_mode(const Params& p, const TcPlan& plan);
+// Enqueues the draft kernel and, where the rerank does not fit inside it, the rerank kernel behind it.
 cudaError_t launch_draft_fused(const Params& p, const TcPlan& plan, const FusedArgs& fa, cudaStream_t st);
 
 }  // namespace ddd

@@ -134,18 +134,23 @@ __device__ __forceinline__ int node_depth(int id, int k) {
 }
 
 // Block-wide exclusive prefix sum of one int per thread (THREADS threads).
-template <int THREADS>
-__device__ int block_exclusive_scan(int v, int* warp_tot /* [32] shared */, int* total) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+// Sync::sync() is the barrier of the THREADS threads that call this together (a whole block, or
+// a group of warps on a named barrier); tid is the caller's index in that group.
+struct BlockSync {
+  __device__ static __forceinline__ void sync() { __syncthreads(); }
+};
+template <int THREADS, typename Sync>
+__device__ int block_exclusive_scan(int v, int* warp_tot /* [32] shared */, int* total, const int tid) {
+  const int lane = tid & 31, warp = tid >> 5;
   int inc = v;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
     const int t = __shfl_up_sync(kFullMask, inc, o);
     if (lane >= o) inc += t;
   }
-  __syncthreads();                 // protect warp_tot from its previous use
+  Sync::sync();                 // protect warp_tot from its previous use
   if (lane == 31) warp_tot[warp] = inc;
-  __syncthreads();
+  Sync::sync();
   int offset = 0, tot = 0;
   for (int w = 0; w < THREADS / 32; ++w) {
     const int t = warp_tot[w];
@@ -162,20 +167,22 @@ __device__ int block_exclusive_scan(int v, int* warp_tot /* [32] shared */, int*
 // was the last sequence of the batch still drafting: that block also reports the device status.
 // KEYS_IN_SMEM false: the tree is too large to keep its keys in shared memory; they are formed from
 // the scores in global memory each time (smem_raw then holds only the 16-bit rows).
-template <int THREADS, bool KEYS_IN_SMEM>
-__device__ void rerank_mask_block(const Params& p, const DraftIO& io, const int b, const int D, const bool last,
-                                  unsigned char* smem_raw) {
-  const int tid = threadIdx.x;
+// The group's scratch: hist [256], warp_tot [32], two words (prefix, remaining), all 32-bit, and
+// out_parent [T] 16-bit; `cap` = node slots smem_raw has room for (at least N + 1).
+constexpr int kRerankScratchInts = 256 + 32 + 2;
+template <int THREADS, bool KEYS_IN_SMEM, typename Sync>
+__device__ void rerank_mask_impl(const Params& p, const DraftIO& io, const int b, const int D, const bool last,
+                                 const int tid, unsigned char* smem_raw, const int cap, int* scratch,
+                                 short* out_parent) {
   const int k = p.k, T = p.T;
   const int N = (D >= 1) ? k + (D - 1) * k * k : 0;     // generated non-root nodes
   uint32_t* key_s = reinterpret_cast<uint32_t*>(smem_raw);         // key of node id i+1 at [i]
-  short* slot_of = reinterpret_cast<short*>(KEYS_IN_SMEM ? smem_raw + (size_t)p.Nn * sizeof(uint32_t) : smem_raw);
+  short* slot_of = reinterpret_cast<short*>(KEYS_IN_SMEM ? smem_raw + (size_t)cap * sizeof(uint32_t) : smem_raw);
                                                                     // output row of node id (< 1024), -1 = dropped
-  __shared__ int hist[256];
-  __shared__ int warp_tot[32];
-  __shared__ uint32_t s_prefix;
-  __shared__ int s_remaining;
-  __shared__ int out_parent[DDD_MAX_TOTAL + 1];
+  int* hist = scratch;
+  int* warp_tot = scratch + 256;
+  uint32_t& s_prefix = *reinterpret_cast<uint32_t*>(scratch + 288);
+  int& s_remaining = scratch[289];
 
   const float* cum = p.tree_cum + (size_t)b * p.Nn;
   const int* tparent = p.tree_parent + (size_t)b * p.Nn;
@@ -185,76 +192,103 @@ __device__ void rerank_mask_block(const Params& p, const DraftIO& io, const int 
     for (int i = tid; i < N; i += THREADS) key_s[i] = float_to_ordered(cum[i + 1]);
   const int m_eff = min(p.m, N);
   if (tid == 0) { s_prefix = 0u; s_remaining = m_eff; }
-  __syncthreads();
+  Sync::sync();
 
-  // ---- radix select: value of the m_eff-th largest key and how many of its ties to keep
-  uint32_t known_mask = 0u;
-  for (int pass = 3; pass >= 0 && m_eff > 0; --pass) {
-    const int shift = 8 * pass;
-    for (int i = tid; i < 256; i += THREADS) hist[i] = 0;
-    __syncthreads();
-    const uint32_t prefix = s_prefix;
-    for (int i = tid; i < N; i += THREADS) {
-      const uint32_t q = key(i);
-      if ((q & known_mask) == prefix) atomicAdd(&hist[(q >> shift) & 0xFF], 1);
-    }
-    __syncthreads();
-    if (tid < 32) {
-      // warp 0 finds the bin holding the `remaining`-th largest key: lane l owns bins 8l .. 8l+7
-      const int remaining = s_remaining;
-      int local[8], mine = 0;
-#pragma unroll
-      for (int i = 0; i < 8; ++i) { local[i] = hist[8 * tid + i]; mine += local[i]; }
-      int above = mine;                                   // suffix sum over lanes >= tid ...
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int t = __shfl_down_sync(kFullMask, above, o);
-        if (tid + o < 32) above += t;
-      }
-      above -= mine;                                      // ... made exclusive: keys in higher lanes' bins
-      if (above < remaining && remaining <= above + mine) {   // exactly one lane
-        int rem = remaining - above, bin = 7;
-        for (; bin > 0; --bin) {
-          if (local[bin] >= rem) break;
-          rem -= local[bin];
-        }
-        s_prefix = prefix | ((uint32_t)(8 * tid + bin) << shift);
-        s_remaining = rem;
-      }
-    }
-    known_mask |= 0xFFu << shift;
-    __syncthreads();
-  }
-  const uint32_t thr = s_prefix;
-  const int keep_ties = s_remaining;      // among keys equal to thr, the lowest node ids win
-
-  // ---- selection flags in node-id order; each thread owns a contiguous chunk of ids
-  const int chunk = (N + THREADS - 1) / THREADS;
-  const int lo = min(N, tid * chunk), hi = min(N, lo + chunk);
-  int n_eq = 0;
-  for (int i = lo; i < hi; ++i) n_eq += (key(i) == thr);
-  int tot_unused;
-  int eq_before = block_exclusive_scan<THREADS>(n_eq, warp_tot, &tot_unused);
-  int n_sel = 0;
-  for (int i = lo; i < hi; ++i) {
-    const uint32_t q = key(i);
-    bool sel = false;
-    if (m_eff > 0) {
-      if (q > thr) sel = true;
-      else if (q == thr) sel = (eq_before++ < keep_ties);
-    }
-    slot_of[i + 1] = sel ? 1 : 0;
-    n_sel += sel;
-  }
   int n_selected;
-  int sel_before = block_exclusive_scan<THREADS>(n_sel, warp_tot, &n_selected);
-  for (int i = lo; i < hi; ++i) {
-    const bool sel = slot_of[i + 1] != 0;
-    slot_of[i + 1] = sel ? (short)(1 + sel_before) : (short)-1;
-    sel_before += sel;
+  if (KEYS_IN_SMEM && N <= THREADS) {
+    // ---- few nodes (a draft that stopped early: the common case): one node per thread, ranked by
+    // counting the nodes that come before it in (score descending, node id ascending) order;
+    // five barriers instead of the thirty-odd of the radix path
+    const uint32_t mine = tid < N ? key_s[tid] : 0u;
+    int rank = 0;
+    for (int j = 0; j < N; ++j) {
+      const uint32_t q = key_s[j];
+      rank += (q > mine || (q == mine && j < tid)) ? 1 : 0;
+    }
+    const bool sel = tid < N && rank < m_eff;
+    if (tid < N) slot_of[tid + 1] = sel ? 1 : 0;
+    Sync::sync();
+    int before = 0, total = 0;
+    for (int j = 0; j < N; ++j) {
+      const int f = slot_of[j + 1];
+      total += f;
+      before += j < tid ? f : 0;
+    }
+    n_selected = total;
+    Sync::sync();
+    if (tid < N) slot_of[tid + 1] = sel ? (short)(1 + before) : (short)-1;
+    if (tid == 0) slot_of[0] = 0;
+    Sync::sync();
+  } else {
+    // ---- radix select: value of the m_eff-th largest key and how many of its ties to keep
+    uint32_t known_mask = 0u;
+    for (int pass = 3; pass >= 0 && m_eff > 0; --pass) {
+      const int shift = 8 * pass;
+      for (int i = tid; i < 256; i += THREADS) hist[i] = 0;
+      Sync::sync();
+      const uint32_t prefix = s_prefix;
+      for (int i = tid; i < N; i += THREADS) {
+        const uint32_t q = key(i);
+        if ((q & known_mask) == prefix) atomicAdd(&hist[(q >> shift) & 0xFF], 1);
+      }
+      Sync::sync();
+      if (tid < 32) {
+        // warp 0 finds the bin holding the `remaining`-th largest key: lane l owns bins 8l .. 8l+7
+        const int remaining = s_remaining;
+        int local[8], mine = 0;
+  #pragma unroll
+        for (int i = 0; i < 8; ++i) { local[i] = hist[8 * tid + i]; mine += local[i]; }
+        int above = mine;                                   // suffix sum over lanes >= tid ...
+  #pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int t = __shfl_down_sync(kFullMask, above, o);
+          if (tid + o < 32) above += t;
+        }
+        above -= mine;                                      // ... made exclusive: keys in higher lanes' bins
+        if (above < remaining && remaining <= above + mine) {   // exactly one lane
+          int rem = remaining - above, bin = 7;
+          for (; bin > 0; --bin) {
+            if (local[bin] >= rem) break;
+            rem -= local[bin];
+          }
+          s_prefix = prefix | ((uint32_t)(8 * tid + bin) << shift);
+          s_remaining = rem;
+        }
+      }
+      known_mask |= 0xFFu << shift;
+      Sync::sync();
+    }
+    const uint32_t thr = s_prefix;
+    const int keep_ties = s_remaining;      // among keys equal to thr, the lowest node ids win
+
+    // ---- selection flags in node-id order; each thread owns a contiguous chunk of ids
+    const int chunk = (N + THREADS - 1) / THREADS;
+    const int lo = min(N, tid * chunk), hi = min(N, lo + chunk);
+    int n_eq = 0;
+    for (int i = lo; i < hi; ++i) n_eq += (key(i) == thr);
+    int tot_unused;
+    int eq_before = block_exclusive_scan<THREADS, Sync>(n_eq, warp_tot, &tot_unused, tid);
+    int n_sel = 0;
+    for (int i = lo; i < hi; ++i) {
+      const uint32_t q = key(i);
+      bool sel = false;
+      if (m_eff > 0) {
+        if (q > thr) sel = true;
+        else if (q == thr) sel = (eq_before++ < keep_ties);
+      }
+      slot_of[i + 1] = sel ? 1 : 0;
+      n_sel += sel;
+    }
+    int sel_before = block_exclusive_scan<THREADS, Sync>(n_sel, warp_tot, &n_selected, tid);
+    for (int i = lo; i < hi; ++i) {
+      const bool sel = slot_of[i + 1] != 0;
+      slot_of[i + 1] = sel ? (short)(1 + sel_before) : (short)-1;
+      sel_before += sel;
+    }
+    if (tid == 0) slot_of[0] = 0;
+    Sync::sync();
+
   }
-  if (tid == 0) slot_of[0] = 0;
-  __syncthreads();
 
   // ---- emit rows: the root, then the kept nodes in ascending node id
   const int n_out = 1 + n_selected;
@@ -285,7 +319,7 @@ __device__ void rerank_mask_block(const Params& p, const DraftIO& io, const int 
     io.out.stop_depth[b] = D;
     if (last) *io.out.status = *reinterpret_cast<volatile int*>(p.dev_status);
   }
-  __syncthreads();
+  Sync::sync();
 
   // ---- ancestor mask: row i has bit j set iff j is i or an ancestor of i
   for (int slot = tid; slot < T; slot += THREADS) {
@@ -312,6 +346,17 @@ __device__ void rerank_mask_block(const Params& p, const DraftIO& io, const int 
       if (io.trace.tree_cum) io.trace.tree_cum[o] = gen ? cum[id] : 0.f;
     }
   }
+}
+
+// The same for a whole thread block with its own static scratch (the kernels that end a sequence's
+// last pass, and rerank_kernel).
+template <int THREADS, bool KEYS_IN_SMEM>
+__device__ void rerank_mask_block(const Params& p, const DraftIO& io, const int b, const int D, const bool last,
+                                  unsigned char* smem_raw) {
+  __shared__ int scratch[kRerankScratchInts];
+  __shared__ short out_parent[DDD_MAX_TOTAL + 1];
+  rerank_mask_impl<THREADS, KEYS_IN_SMEM, BlockSync>(p, io, b, D, last, (int)threadIdx.x, smem_raw, p.Nn, scratch,
+                                                     out_parent);
 }
 
 

@@ -342,7 +342,7 @@ def test_fused_draft_equals_kernel_by_kernel_draft(case):
     cfg = small_cases()[case]
     eng_s = engine_for(cfg, TC, P.DDD_LAUNCH_STREAM)
     eng_f = engine_for(cfg, TC, P.DDD_LAUNCH_FUSED)
-    assert P.ddd_launches_per_draft(eng_f.handle, 1) == 2
+    assert P.ddd_launches_per_draft(eng_f.handle, 1) in (1, 2)      # the rerank kernel only where it does not fit inside
     depths = set()
     for i in range(4):
         roots = S.make_roots(cfg, i)
