@@ -401,6 +401,25 @@ def test_fused_draft_with_both_tiles_of_a_block_sharing_a_stage(vocab):
     eng_f.close()
 
 
+@pytest.mark.parametrize("k,n,launches", [(10, 12, 1), (10, 16, 1), (16, 16, 2)], ids=["keys_in_smem", "keys_from_global", "kernel"])
+def test_fused_draft_rerank_inside_or_behind_the_kernel(k, n, launches):
+    # The persistent kernel reranks in its 8 KB transpose buffer where the tree fits: 1111 nodes with
+    # their keys, 1511 nodes with keys read from global memory; 3857 nodes go to the rerank kernel.
+    cfg = S.scaled_down(S.CONFIGS["llama2_7b"], 256, 3000 + 8, threshold=NEG, k=k, max_depth=n, total_tokens=90)
+    eng_s = engine_for(cfg, TC, P.DDD_LAUNCH_STREAM)
+    eng_f = engine_for(cfg, TC, P.DDD_LAUNCH_FUSED)
+    assert P.ddd_launches_per_draft(eng_f.handle, n) == launches
+    for i in range(2):
+        roots = S.make_roots(cfg, i)
+        a = parity.run_gpu(eng_s, roots)
+        b = parity.run_gpu(eng_f, roots)
+        for name in a:
+            np.testing.assert_array_equal(a[name], b[name], err_msg=name)
+        parity.compare_with_oracle(cfg, weights_for(cfg), roots, b)
+    eng_s.close()
+    eng_f.close()
+
+
 @pytest.mark.parametrize("mode", [P.DDD_LAUNCH_STREAM, P.DDD_LAUNCH_FUSED], ids=["stream", "fused"])
 def test_w_may_be_released_after_create_on_the_tensor_core_path(mode):
     # ddd_create packs W into the workspace; nothing on the tensor-core path reads the original again
