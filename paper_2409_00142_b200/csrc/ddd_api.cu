@@ -28,7 +28,7 @@ size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 struct Layout {
   size_t hbuf[2], part_key, part_ms, tree_token, tree_parent, tree_cum, beam_node, beam_tok, beam_cum,
       row_plant, active, stop_depth, root_pos, n_active, dev_status, lm_ticket, shard_counter, fused_sync,
-      fused_beam_cum, fused_beam_node, fused_row_plant, fused_key, fused_ms, w_packed;
+      fused_beam_cum, fused_beam_node, fused_row_plant, fused_key, fused_ms, wide_records, w_packed;
   // staging for ddd_draft_host: inputs, then the packed output block
   size_t in_hidden, in_token, in_pos, out_block;
   size_t o_n_out, o_stop, o_token, o_parent, o_depth, o_position, o_cum, o_mask, o_H, o_status, out_bytes;
@@ -93,6 +93,7 @@ Layout make_layout(const ddd_config* c) {
   const bool may_fuse = c->launch_mode == DDD_LAUNCH_FUSED && k <= 32;
   L.fused_key = take(may_fuse ? R * k * 160 * 8 : 0);
   L.fused_ms = take(may_fuse ? R * 160 * 8 : 0);
+  L.wide_records = take(k > 32 ? R * (k + 1) * 8 : 0);      // beams wider than 32: one folded partial per row
   // packed copy of W for the tensor-core kernel (kept 1024-byte aligned relative to the base)
   off = (off + 1023) / 1024 * 1024;
   const bool tc_possible = c->dtype == DDD_DTYPE_BF16 && c->hidden % 64 == 0 && c->lm_head_kernel != DDD_LM_HEAD_SIMT;
@@ -185,9 +186,21 @@ cudaError_t enqueue_passes(const ddd_handle* h, const DraftIO& io, bool pdl, int
                            cudaGraphConditionalHandle cond, int cond_pass, cudaStream_t st,
                            bool after_kernel = false) {
   cudaError_t e = cudaSuccess;
+  // Beams wider than 32: a kernel of one block per beam row folds the per-block partials into one
+  // list per row first (the select kernel's eight blocks per sequence would otherwise merge
+  // k x 148 lists one row after the other), and the select kernel reads that one partial.
+  const bool wide = h->p.k > 32;
+  Params q = h->p;
+  void* rec = h->ws + h->L.wide_records;
+  if (wide) {
+    q.part_key = reinterpret_cast<unsigned long long*>(rec);
+    q.part_ms = reinterpret_cast<float2*>(h->ws + h->L.wide_records + (size_t)q.R * q.k * sizeof(unsigned long long));
+    q.lm_ctas = 1;
+  }
   for (int d = first; d <= last && e == cudaSuccess; ++d) {
     e = launch_lm_head(h, d, 0, pdl && (d > first || after_kernel), st);
-    if (e == cudaSuccess) e = launch_select(h->p, io, d, pdl, cond, d == cond_pass, st);
+    if (e == cudaSuccess && wide) e = launch_shard_reduce(h->p, d, 0, 1, &rec, nullptr, 1, 0, h->shard_counter, st);
+    if (e == cudaSuccess) e = launch_select(wide ? q : h->p, io, d, pdl, cond, d == cond_pass, st);
   }
   return e;
 }
@@ -684,7 +697,9 @@ int ddd_launches_per_draft(const ddd_handle* h, int32_t passes_needed) {
     for (int j = nb - 1; j >= 0; --j)
       if (passes_needed <= h->bounds[j]) passes = h->bounds[j];   // the group that holds the last needed pass
   }
-  return 1 + 2 * passes;   // init, then (LM head + select) per launched pass
+  // init, then per launched pass LM head + select, and between them for beams wider than 32 the kernel
+  // that folds the per-block partials
+  return 1 + (h->p.k > 32 ? 3 : 2) * passes;
 }
 
 int ddd_lm_head_blocks(const ddd_handle* h) {

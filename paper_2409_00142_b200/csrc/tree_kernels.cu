@@ -526,62 +526,82 @@ __global__ void __launch_bounds__(kWideThreads) select_gate_step_wide_kernel(con
   __shared__ bool s_last;
   (void)part_slots;
 
-  // ---- phase 1: merge the partial lists of this block's beam rows, one row at a time
-  bool waited = false;
-  for (int pr = crank; pr < P; pr += kSelCluster) {
+  // ---- phase 1: merge the partial lists of this block's beam rows
+  // What a warp does with a row's merged list acc and the row's (max, sum-exp) over all partials:
+  // planted column, log-sum-exp, the k candidates to every block of the cluster, the tree nodes.
+  auto finish_row = [&](const int pr, unsigned long long (&acc)[4], float M, float S) {
     const int r = b * k + pr;
-    unsigned long long acc[4] = {0ull, 0ull, 0ull, 0ull};
-    for (int c = warp; c < nc; c += kWideWarps) {
-      unsigned long long t[4];
-      wide_load(t, p.part_key + ((size_t)c * R + r) * k, k);
-      wide_merge(acc, t);
+    const int pc = p.row_plant[r];
+    if (pc >= 0) {          // planted column: (max of the others) + delta; it was left out of the partials
+      const float zc = M + p.plant_delta;
+      const float M2 = fmaxf(M, zc);
+      S = S * expf(M - M2) + expf(zc - M2);
+      M = M2;
+      unsigned long long one[4] = {lane == 0 ? make_key(zc, (uint32_t)pc) : 0ull, 0ull, 0ull, 0ull};
+      wide_merge(acc, one);
     }
-    block_merge_lists(acc, buf);
-    if (!waited) {
-      asm volatile("barrier.cluster.wait.aligned;" ::: "memory");
-      waited = true;
-    }
-    if (warp == 0) {
-      float M = neg_inf();
-      for (int c = lane; c < nc; c += 32) M = fmaxf(M, p.part_ms[(size_t)c * R + r].x);
-      M = ordered_to_float(__reduce_max_sync(kFullMask, float_to_ordered(M)));
-      float S = 0.f;
-      for (int c = lane; c < nc; c += 32) {
-        const float2 ms = p.part_ms[(size_t)c * R + r];
-        if (ms.y > 0.f) S += ms.y * expf(ms.x - M);
-      }
-      S = warp_sum(S);
-      const int pc = p.row_plant[r];
-      if (pc >= 0) {          // planted column: (max of the others) + delta; it was left out of the partials
-        const float zc = M + p.plant_delta;
-        const float M2 = fmaxf(M, zc);
-        S = S * expf(M - M2) + expf(zc - M2);
-        M = M2;
-        unsigned long long one[4] = {lane == 0 ? make_key(zc, (uint32_t)pc) : 0ull, 0ull, 0ull, 0ull};
-        wide_merge(acc, one);
-      }
-      const float lse = M + logf(S);
-      const float cum0 = p.beam_cum[r];
-      const int parent_node = p.beam_node[r];
+    const float lse = M + logf(S);
+    const float cum0 = p.beam_cum[r];
+    const int parent_node = p.beam_node[r];
 #pragma unroll
-      for (int s4 = 0; s4 < 4; ++s4) {
-        const int e = 4 * lane + s4;
-        if (e >= k) continue;
-        const unsigned long long key = acc[s4];
-        const float lp = key != 0ull ? fminf(key_value(key) - lse, 0.f) : neg_inf();
-        const int tok = key != 0ull ? (int)key_index(key) : -1;
-        const float cand = cum0 + lp;
-        const int flat = pr * k + e;
-        const unsigned long long rec = ((unsigned long long)__float_as_uint(cand) << 32) | (uint32_t)tok;
-        for (int rk = 0; rk < kSelCluster; ++rk) cluster.map_shared_rank(cand_rec, rk)[flat] = rec;
-        const size_t node = (size_t)b * p.Nn + base + flat;
-        p.tree_token[node] = tok;
-        p.tree_parent[node] = parent_node;
-        p.tree_cum[node] = cand;
-      }
-      if (lane == 0 && io.trace.row_lse) io.trace.row_lse[((size_t)b * p.n + (d - 1)) * k + pr] = lse;
+    for (int s4 = 0; s4 < 4; ++s4) {
+      const int e = 4 * lane + s4;
+      if (e >= k) continue;
+      const unsigned long long key = acc[s4];
+      const float lp = key != 0ull ? fminf(key_value(key) - lse, 0.f) : neg_inf();
+      const int tok = key != 0ull ? (int)key_index(key) : -1;
+      const float cand = cum0 + lp;
+      const int flat = pr * k + e;
+      const unsigned long long rec = ((unsigned long long)__float_as_uint(cand) << 32) | (uint32_t)tok;
+      for (int rk = 0; rk < kSelCluster; ++rk) cluster.map_shared_rank(cand_rec, rk)[flat] = rec;
+      const size_t node = (size_t)b * p.Nn + base + flat;
+      p.tree_token[node] = tok;
+      p.tree_parent[node] = parent_node;
+      p.tree_cum[node] = cand;
     }
-    __syncthreads();
+    if (lane == 0 && io.trace.row_lse) io.trace.row_lse[((size_t)b * p.n + (d - 1)) * k + pr] = lse;
+  };
+  bool waited = false;
+  if (nc == 1) {
+    // one partial per row (the per-block partials were folded by a kernel of their own, or there is
+    // one record set slot): nothing to merge, a warp per row, all rows of the block at once
+    asm volatile("barrier.cluster.wait.aligned;" ::: "memory");
+    waited = true;
+    for (int pr = crank + kSelCluster * warp; pr < P; pr += kSelCluster * kWideWarps) {
+      const int r = b * k + pr;
+      unsigned long long acc[4];
+      wide_load(acc, p.part_key + (size_t)r * k, k);
+      const float2 ms = p.part_ms[r];
+      finish_row(pr, acc, ms.x, ms.y);
+    }
+  } else {
+    for (int pr = crank; pr < P; pr += kSelCluster) {
+      const int r = b * k + pr;
+      unsigned long long acc[4] = {0ull, 0ull, 0ull, 0ull};
+      for (int c = warp; c < nc; c += kWideWarps) {
+        unsigned long long t[4];
+        wide_load(t, p.part_key + ((size_t)c * R + r) * k, k);
+        wide_merge(acc, t);
+      }
+      block_merge_lists(acc, buf);
+      if (!waited) {
+        asm volatile("barrier.cluster.wait.aligned;" ::: "memory");
+        waited = true;
+      }
+      if (warp == 0) {
+        float M = neg_inf();
+        for (int c = lane; c < nc; c += 32) M = fmaxf(M, p.part_ms[(size_t)c * R + r].x);
+        M = ordered_to_float(__reduce_max_sync(kFullMask, float_to_ordered(M)));
+        float S = 0.f;
+        for (int c = lane; c < nc; c += 32) {
+          const float2 ms = p.part_ms[(size_t)c * R + r];
+          if (ms.y > 0.f) S += ms.y * expf(ms.x - M);
+        }
+        S = warp_sum(S);
+        finish_row(pr, acc, M, S);
+      }
+      __syncthreads();
+    }
   }
   if (!waited) asm volatile("barrier.cluster.wait.aligned;" ::: "memory");
   cluster.sync();
