@@ -547,7 +547,10 @@ def main():
                    "launch": args.launch_mode},
         "clocks": clocks,
         "e2e": {"value": n_per_rank * world * cfg.batch / (e2e_ms / 1e3), "unit": UNIT,
-                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "transfer": ("ddd_draft_host: the kernel reads the roots from and writes the rows to pinned host memory"
+                             if args.launch_mode == "fused" else
+                             "ddd_draft_host: one copy command in each direction through a pinned bounce buffer")},
         "gpu_launches": launches,
         "gpu_launches_kind": "computed: ddd_launches_per_draft(stop depth) summed over the timed drafts",
         "us_per_draft": us_per_draft,

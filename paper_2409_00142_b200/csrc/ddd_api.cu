@@ -538,7 +538,9 @@ int ddd_draft_host(ddd_handle* h, const void* root_hidden, const int32_t* root_t
   const Layout& L = h->L;
   const Params& p = h->p;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  const size_t need = (L.in_bytes > L.out_bytes ? L.in_bytes : L.out_bytes);
+  // inputs first, results behind them (the fused mode reads and writes this buffer from the device)
+  const size_t out_off = align_up(L.in_bytes);
+  const size_t need = out_off + L.out_bytes;
   if (!h->bounce) {
     if (cudaMallocHost(reinterpret_cast<void**>(&h->bounce), need) != cudaSuccess) {
       note_cuda_error(__LINE__);
@@ -564,7 +566,33 @@ int ddd_draft_host(ddd_handle* h, const void* root_hidden, const int32_t* root_t
   dev.mask = reinterpret_cast<uint32_t*>(ob + L.o_mask);
   dev.H_trace = reinterpret_cast<float*>(ob + L.o_H);
   dev.status = reinterpret_cast<int32_t*>(ob + L.o_status);
-  if (h->cfg.launch_mode == DDD_LAUNCH_GRAPH && st != nullptr) {
+  const unsigned char* hb = h->bounce;      // where the packed results end up
+  if (h->cfg.launch_mode == DDD_LAUNCH_FUSED) {
+    // Pinned host memory is addressable from the device: the persistent kernel reads the roots from
+    // the bounce buffer itself (8 KB, under its first W copies) and writes the rows straight into it,
+    // so the call is one kernel launch and one synchronisation, with no copy commands.
+    unsigned char* hob = h->bounce + out_off;
+    ddd_output direct;
+    direct.n_out = reinterpret_cast<int32_t*>(hob + L.o_n_out);
+    direct.stop_depth = reinterpret_cast<int32_t*>(hob + L.o_stop);
+    direct.token = reinterpret_cast<int32_t*>(hob + L.o_token);
+    direct.parent = reinterpret_cast<int32_t*>(hob + L.o_parent);
+    direct.depth = reinterpret_cast<int32_t*>(hob + L.o_depth);
+    direct.position = reinterpret_cast<int32_t*>(hob + L.o_position);
+    direct.cum = reinterpret_cast<float*>(hob + L.o_cum);
+    direct.mask = reinterpret_cast<uint32_t*>(hob + L.o_mask);
+    direct.H_trace = reinterpret_cast<float*>(hob + L.o_H);
+    direct.status = reinterpret_cast<int32_t*>(hob + L.o_status);
+    const int rc = ddd_draft(h, h->bounce, reinterpret_cast<const int32_t*>(h->bounce + (L.in_token - L.in_hidden)),
+                             reinterpret_cast<const int32_t*>(h->bounce + (L.in_pos - L.in_hidden)), &direct, nullptr,
+                             cuda_stream);
+    if (rc != DDD_OK) return rc;
+    if (cudaStreamSynchronize(st) != cudaSuccess) {
+      note_cuda_error(__LINE__);
+      return DDD_ERR_CUDA;
+    }
+    hb = hob;
+  } else if (h->cfg.launch_mode == DDD_LAUNCH_GRAPH && st != nullptr) {
     // the whole call is one graph launch: input copy, init kernel, the passes, output copy
     if (!h->exec_host || h->host_stream != st) {
       if (h->exec_host) { cudaGraphExecDestroy(h->exec_host); h->exec_host = nullptr; }
@@ -594,7 +622,6 @@ int ddd_draft_host(ddd_handle* h, const void* root_hidden, const int32_t* root_t
     }
   }
   // scatter the packed results to the caller's arrays
-  const unsigned char* hb = h->bounce;
   std::memcpy(out->n_out, hb + L.o_n_out, B * 4);
   std::memcpy(out->stop_depth, hb + L.o_stop, B * 4);
   std::memcpy(out->token, hb + L.o_token, B * T * 4);
