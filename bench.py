@@ -35,7 +35,7 @@ NEG = -1e30
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes (read + write) of one launch of the persistent draft kernel (a full-depth draft) from the
 # ncu capture summarised under profiles/, valid only while the kernel source is the one that was profiled.
-NCU_TRAFFIC = {"llama2_7b": {"bytes": 2941.0e6, "source_sha256_16": "7c09441afd0fff5c",
+NCU_TRAFFIC = {"llama2_7b": {"bytes": 2941.0e6, "source_sha256_16": "3aa5f989121ea0e8",
                              "profile": "profiles/draft_fused_llama2_7b.md"}}
 BEAM_WIDTHS = (5, 10, 20, 50, 75, 100)      # fixed-depth-6 sweep: the widths of the paper's appendix table
 OTHER_WORKLOADS = ("vicuna_13b", "llama2_70b_b16", "llama3_8b_128k")

@@ -22,7 +22,8 @@
 // (tree nodes, beam state, trace, stop).  Blocks without a row go straight to hand-over 2, after
 // which the producers fetch the new hidden rows and the next pass runs.  The beam state is kept
 // twice, by pass parity: a block may still read the old beam while the book-keeper writes the new.
-// The rerank and the mask run in a small kernel of their own afterwards.
+// After the last pass the blocks that kept a sequence's books rerank its tree and write the rows
+// and the mask (in the epilogue's transpose buffer; a tree too large for it goes to rerank_kernel).
 //
 // Every wait is bounded.  A wait that runs out records DDD_ERR_TIMEOUT, raises a grid-wide abort
 // word that ends every other wait, and each block drains its copies, frees its tensor memory and
