@@ -208,6 +208,32 @@ def test_edge_shapes_match_oracle(case, kernel):
     eng.close()
 
 
+def fused_edge_cases():
+    cases = dict(edge_cases())
+    base = S.scaled_down(S.CONFIGS["llama2_7b"], 128, 1000, threshold=-6.0)
+    cases.update({
+        "more_sequences_than_blocks": base.replace(batch=200, k=1, max_depth=5, total_tokens=4),   # 200 rows, 32 blocks
+        "two_blocks_for_eight_rows": base.replace(vocab=40, k=8, max_depth=4, total_tokens=30),    # a block owns 4 rows of one sequence
+        "batch_stops_apart": base.replace(batch=6, k=5, max_depth=8, total_tokens=40, threshold=-2.5),
+    })
+    return cases
+
+
+@pytest.mark.parametrize("case", list(fused_edge_cases()))
+def test_edge_shapes_in_one_persistent_kernel(case):
+    cfg = fused_edge_cases()[case]
+    eng = engine_for(cfg, TC, P.DDD_LAUNCH_FUSED)
+    stops = set()
+    for i in range(2):
+        roots = S.make_roots(cfg, i)
+        g = parity.run_gpu(eng, roots)
+        parity.compare_with_oracle(cfg, weights_for(cfg), roots, g)
+        stops.update(g["stop_depth"].tolist())
+    if case == "batch_stops_apart":
+        assert len(stops) > 1, stops
+    eng.close()
+
+
 # ----------------------------------------------------------------------------- seeded random shapes
 def random_shapes():
     """Forty seeded configurations spread over the legal ranges: beam rows 1..256 (so every
