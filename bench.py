@@ -444,6 +444,56 @@ def main():
                 we.close()
             extra["beam_width_sweep_depth6"] = sweep_w
 
+        # ---- vocabulary-parallel LM head, compute side only: the G ranks' kernels of a pass (LM head over a
+        # slice, fold to one record per row, select over the G records) run one after the other on this one
+        # GPU; the time of a pass divided by G is what one rank computes.  No exchange is timed: one GPU.
+        if not args.no_sweep and world == 1 and cfg.dtype == "bf16":
+            G = 8
+            vcfg = cfg.replace(threshold=NEG)
+            ranks = [P.DraftEngine(vcfg, dev_weights, device=local, with_trace=False,
+                                   vocab_slice=P.vocab_slice(vcfg.vocab, G, g)) for g in range(G)]
+            nbytes = P.ddd_shard_records_bytes(ranks[0].c, G)
+            recs = [[torch.zeros(nbytes, dtype=torch.uint8, device=device) for _ in range(2)] for _ in range(G)]
+            flags = [[torch.zeros(G, dtype=torch.int32, device=device) for _ in range(2)] for _ in range(G)]
+
+            def sharded_draft(r):
+                for e in ranks:
+                    e.shard_begin(r["root_hidden"], r["root_token"], r["root_pos"])
+                for d in range(1, vcfg.max_depth + 1):
+                    par = d & 1
+                    for g, e in enumerate(ranks):
+                        e.shard_lm_head(d, g, G, [recs[q][par] for q in range(G)], [flags[q][par] for q in range(G)])
+                    for g, e in enumerate(ranks):
+                        e.shard_select(d, recs[g][par], G, flags[g][par])
+
+            for r in roots_dev[:2]:
+                sharded_draft(r)
+            torch.cuda.synchronize(device)
+            # replayed from a captured graph: launched call by call from Python the 4 x G small kernels of a pass
+            # would measure the host, not the device
+            vp_graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(vp_graph, stream=stream):
+                sharded_draft(roots_dev[0])
+            vp_graph.replay()
+            torch.cuda.synchronize(device)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            n_vp = 8
+            e0.record(stream)
+            for _ in range(n_vp):
+                vp_graph.replay()
+            e1.record(stream)
+            torch.cuda.synchronize(device)
+            del vp_graph
+            assert all(int(e.out["status"].item()) == 0 for e in ranks)
+            per_pass = 1e3 * e0.elapsed_time(e1) / n_vp / vcfg.max_depth
+            extra["vocab_parallel"] = {
+                "ranks": G, "us_per_pass_per_rank_compute": per_pass / G, "us_per_pass_all_ranks_serialised": per_pass,
+                "record_bytes_per_rank_per_pass": nbytes // G,
+                "note": "the ranks' kernels run back to back on one GPU; no exchange is timed (unmeasured on hardware)"}
+            for e in ranks:
+                e.close()
+            del ranks, recs, flags
+
         # ---- end to end through the host-buffer entry point (pinned host memory, copies inside)
         host_out = eng.make_host_out(pinned=True)
         pinned = rows_of({k: v.pin_memory() for k, v in roots_host.items()})
