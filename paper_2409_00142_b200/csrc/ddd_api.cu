@@ -28,7 +28,7 @@ size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 struct Layout {
   size_t hbuf[2], part_key, part_ms, tree_token, tree_parent, tree_cum, beam_node, beam_tok, beam_cum,
       row_plant, active, stop_depth, root_pos, n_active, dev_status, lm_ticket, shard_counter, fused_sync,
-      fused_beam_cum, fused_beam_node, fused_row_plant, fused_key, fused_ms, wide_records, w_packed;
+      fused_beam_cum, fused_beam_node, fused_row_plant, fused_key, fused_ms, fused_gmax, wide_records, w_packed;
   // staging for ddd_draft_host: inputs, then the packed output block
   size_t in_hidden, in_token, in_pos, out_block;
   size_t o_n_out, o_stop, o_token, o_parent, o_depth, o_position, o_cum, o_mask, o_H, o_status, out_bytes;
@@ -86,13 +86,14 @@ Layout make_layout(const ddd_config* c) {
   L.dev_status = take(4);
   L.lm_ticket = take(8);
   L.shard_counter = take(8);
-  L.fused_sync = take(16);
+  L.fused_sync = take(32);
   L.fused_beam_cum = take(2 * R * 4);
   L.fused_beam_node = take(2 * R * 4);
   L.fused_row_plant = take(2 * R * 4);
   const bool may_fuse = c->launch_mode == DDD_LAUNCH_FUSED && k <= 32;
   L.fused_key = take(may_fuse ? R * k * 160 * 8 : 0);
   L.fused_ms = take(may_fuse ? R * 160 * 8 : 0);
+  L.fused_gmax = take(may_fuse ? R * 32 * 4 : 0);
   L.wide_records = take(k > 32 ? R * (k + 1) * 8 : 0);      // beams wider than 32: one folded partial per row
   // packed copy of W for the tensor-core kernel (kept 1024-byte aligned relative to the base)
   off = (off + 1023) / 1024 * 1024;
@@ -416,8 +417,8 @@ int ddd_create(const ddd_config* cfg, const void* W, const void* E, const float*
     if (prop.major != 10) rc = DDD_ERR_UNSUPPORTED;
     const bool fused = cfg->launch_mode == DDD_LAUNCH_FUSED;
     if (rc == DDD_OK && fused && cfg->k > 32) rc = DDD_ERR_UNSUPPORTED;
-    const int atiles = fused && cfg->k <= 32 && fused_pair_mode(p, h->sm_count) ? 2 : 1;
-    if (rc == DDD_OK) rc = tc_plan_create(p, h->sm_count, ws + L.w_packed, &h->tc, fused ? fused_extra_smem(cfg->k) : 0, atiles);
+    const int a_units = fused && cfg->k <= 32 ? fused_stage_units(p, h->sm_count) : 4;
+    if (rc == DDD_OK) rc = tc_plan_create(p, h->sm_count, ws + L.w_packed, &h->tc, fused ? fused_extra_smem(cfg->k) : 0, a_units);
     if (rc == DDD_OK) p.lm_ctas = h->tc.ctas;
     if (rc == DDD_OK && fused) rc = fused_prepare(p, h->tc);
   } else if (rc == DDD_OK && cfg->launch_mode == DDD_LAUNCH_FUSED) {
@@ -465,6 +466,7 @@ int ddd_draft(ddd_handle* h, const void* root_hidden, const int32_t* root_token,
     fa.sync = reinterpret_cast<int*>(h->ws + h->L.fused_sync);
     fa.fkey = reinterpret_cast<unsigned long long*>(h->ws + h->L.fused_key);
     fa.fms = reinterpret_cast<float2*>(h->ws + h->L.fused_ms);
+    fa.gmax = reinterpret_cast<unsigned int*>(h->ws + h->L.fused_gmax);
     if (launch_draft_fused(h->p, h->tc, fa, st) != cudaSuccess) {
       note_cuda_error(__LINE__);
       return DDD_ERR_CUDA;

@@ -82,6 +82,10 @@ __device__ __forceinline__ void grid_arrive(int* counter) {
 // Lane j returns the j-th best key; (M, S) = the row's merged max and sum-exp, in all lanes.
 constexpr int kFusedMaxCtas = 160;     // partial lists per row: five per lane
 constexpr uint32_t kNotLoaded = 0xFFFFFFFFu;
+constexpr int kFloorQueue = 512;       // entries a block can pick up above the rows' floors in one pass
+// scratch of the floor epilogue: [6][n_pad] floats, then the queue (8-byte keys, 2-byte rows)
+__host__ __device__ inline int floor_queue_offset(int n_pad) { return (6 * n_pad * 4 + 7) / 8 * 8; }
+__host__ __device__ inline int floor_scratch_bytes(int n_pad) { return floor_queue_offset(n_pad) + kFloorQueue * 10; }
 
 __device__ __forceinline__ unsigned long long merge_row_soa(const unsigned long long* __restrict__ keys,
                                                             const float2* __restrict__ msrow, int nc, int k,
@@ -187,7 +191,7 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
   // pair mode: a block's two tiles share every stage, so the hidden rows cross from L2 once per pass
   // instead of once per tile (what bounds a pass with many beam rows is L2 -> SM traffic)
   const int pair = fa.pair;
-  const SmemPlan sp = smem_plan(stages, ksub, n_pad, p.R, p.k, cpg, pair ? 2 : 1);
+  const SmemPlan sp = smem_plan(stages, ksub, n_pad, p.R, p.k, cpg, pair ? pair : 4);
   const TreeSmem ts = tree_smem(p.k);
   // The tree work's scratch lies over the epilogue's transpose buffer, which is idle between the
   // last tile of a pass and the first of the next (behind everything else where it is too large).
@@ -211,6 +215,7 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
   __shared__ __align__(8) unsigned long long s_bar_spare;   // end of the MMAs when the block gives up
   __shared__ int s_stopped[kMaxStoppedPerBlock];            // sequences of this block's books that stopped in this pass
   __shared__ int s_nstopped;
+  __shared__ int s_queue_n;                                 // entries in the queue of the floor epilogue
 
   const uint32_t a_base = smem_u32(smem + sp.a), b_base = smem_u32(smem + sp.b);
   const uint32_t b_bytes = (uint32_t)n_pad * kBlockK * 2;
@@ -226,6 +231,7 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
   int* const cnt_hidden = fa.sync + 1;       // hand-over 2: state and hidden rows of the next pass written
   int* const abort_word = fa.sync + 2;
   int* const exit_ticket = fa.sync + 3;
+  int* const cnt_floor = fa.sync + 4;        // floor hand-over: every block's row maxima are recorded
 
   // this block's contiguous range of 32-row units (fixed: block i always covers the same rows)
   const int n_units = (p.Vl + kUnitRows - 1) / kUnitRows;
@@ -234,7 +240,7 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
   const int unit0 = bid * base_units + (bid < rem_units ? bid : rem_units);
   const int n_tiles = (my_units + 3) / 4;
   const int num_kb = p.Hd / (kBlockK * ksub);
-  const uint32_t a_kblock = pair ? 2u * kABytes : (uint32_t)kABytes;     // bytes of W per K-block of a stage
+  const uint32_t a_kblock = (uint32_t)(pair ? pair : 4) * kUnitBytes;     // bytes of W per K-block of a stage
   const uint32_t a_stage = (uint32_t)ksub * a_kblock, b_stage = (uint32_t)ksub * b_bytes;
   const int total_iters = pair ? num_kb : n_tiles * num_kb;         // pipeline steps per pass
   const int prefill = total_iters < stages ? total_iters : stages;
@@ -284,6 +290,8 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
     *p.n_active = p.B;
     *p.dev_status = DDD_OK;
   }
+  if (fa.floor && threadIdx.x < kNarrowK)      // group maxima of the rows this block looks after: none yet
+    for (int r = bid; r < R; r += G) fa.gmax[r * kNarrowK + threadIdx.x] = 0u;
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -475,6 +483,217 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
     const bool row_by_block = (cpr % 32 == 0) && (cpr / 32 <= 64);
     uint32_t tg = 0;
     bool ok = true;
+    // The new beam rows this block looks after (merge, beam, gate, draft step), in ascending order,
+    // -1 behind the last.  Up to one row per block they are dealt out cyclically.  With more rows than
+    // blocks a block's rows should belong to one sequence, whose lists it then merges once: sequence
+    // b gets blocks b * bps .. b * bps + bps - 1, row i < bps goes to block i of them, the others
+    // are dealt out from the far end (row 0's block also keeps the sequence's books).
+    const int bps = (R > G && p.B <= G) ? G / p.B : 0;
+    auto owned_row = [&](const int j) -> int {
+      if (bps == 0) {
+        const int r = bid + j * G;
+        return r < R ? r : -1;
+      }
+      const int b = bid / bps, q = bid - b * bps;
+      if (b >= p.B) return -1;
+      const int i = j == 0 ? q : 2 * bps - 1 - q + (j - 1) * bps;
+      return i < k ? b * k + i : -1;
+    };
+    // The epilogue of a pass whose two accumulators (tile 0: units 0-3, tile 1: the rest) finish
+    // together.  A logit below the k-th best of its row over the whole vocabulary is of no use
+    // to anyone, and a floor under that k-th best is cheap: the blocks fall into k groups (block
+    // mod k), every group records the largest logit any of its blocks holds for the row (one atomic
+    // maximum per row and block), and the smallest of the k group maxima has k entries of k
+    // different blocks at or above it.  Steps, each over the 2 x n_chunks chunks of 16 beam rows
+    // dealt to the 16 warps (warp = one 32-lane quarter of tensor memory, every fourth chunk):
+    //   1. the largest logit per row: warp maxima, then the block's over its 8 quarter-tiles;
+    //      published with the atomic maximum, and the block arrives at the floor hand-over
+    //   2. sum exp(z - block maximum) per row, under the other blocks' way to the hand-over
+    //   3. wait for the hand-over (bounded), floor per row = minimum over the k groups
+    //   4. logits at or above the floor go to a queue in shared memory, the rest is dropped
+    //   5. the queue (tens of entries) is sorted into the rows' lists by counting
+    // Returns 1: lists and (max, sum) of this pass are in st_key / st_ms; 0: the queue ran over
+    // (a floor that says nothing, e.g. k groups of which one holds no valid entry): nothing is
+    // lost, the accumulators are still there and the tile loop does the pass; -1: a wait ran out.
+    unsigned char* const fl_base = smem + sp.zt;
+    float* const fl_part = reinterpret_cast<float*>(fl_base);                       // [4][n_pad] per quarter of the 128 lanes
+    float* const fl_max = fl_part + 4 * n_pad;                                      // [n_pad] block maximum
+    float* const fl_floor = fl_max + n_pad;                                         // [n_pad] floor of the row
+    unsigned long long* const fl_qkey = reinterpret_cast<unsigned long long*>(fl_base + floor_queue_offset(n_pad));
+    short* const fl_qrow = reinterpret_cast<short*>(fl_qkey + kFloorQueue);
+    auto floor_epilogue = [&](const int d) -> int {
+      for (int a2 = 0; a2 < 2; ++a2)
+        if (!epilogue_all(mbar_wait(bar_tfull + 8u * a2, (tg >> 1) & 1u, abort_flag, p.dev_status, false))) return -1;
+      tc_fence_after();
+      if (et == 0) s_queue_n = 0;
+      // This thread's vocabulary row in either tile.  The work is instruction-bound (80 logits per
+      // thread and step), so the common case - the warp's 32 rows all exist and no column is
+      // planted - is one multiply-add per logit; anything else takes the checked form.
+      const bool plants = p.plant_next != nullptr;
+      int tok_t[2];
+      float bias_t[2];
+      bool valid_t[2], plain_t[2], none_t[2];
+#pragma unroll
+      for (int t = 0; t < 2; ++t) {
+        const int rows = min(4, my_units - 4 * t) * kUnitRows;
+        const int vrow = quarter * 32 + lane;
+        const int v = (unit0 + 4 * t) * kUnitRows + vrow;
+        valid_t[t] = vrow < rows && v < p.Vl;
+        bias_t[t] = (valid_t[t] && p.bias) ? p.bias[v] : 0.f;
+        tok_t[t] = v + p.v0;
+        plain_t[t] = !plants && __all_sync(kFullMask, valid_t[t]);
+        none_t[t] = !__any_sync(kFullMask, valid_t[t]);
+      }
+      // logits of 8 beam rows (columns c0 .. c0 + 7) of tile t, -inf where there is none; padded
+      // columns hold whatever the zero rows behind the last beam row give and are never looked at
+      auto load8 = [&](const int t, const int c0, float (&zv)[8]) {
+        if (none_t[t]) {
+#pragma unroll
+          for (int c = 0; c < 8; ++c) zv[c] = neg_inf();
+          return;
+        }
+        float accv[8];
+        tc_load_8cols(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(t * n_pad + c0), accv);
+        if (plain_t[t]) {
+#pragma unroll
+          for (int c = 0; c < 8; ++c) zv[c] = fmaf(accv[c], p.s, bias_t[t]);
+        } else {
+#pragma unroll
+          for (int c = 0; c < 8; ++c)
+            zv[c] = (valid_t[t] && s_plant[min(c0 + c, R - 1)] != tok_t[t]) ? fmaf(accv[c], p.s, bias_t[t]) : neg_inf();
+        }
+      };
+      // One value per column over the warp's 32 lanes, 8 columns at once: the first three steps
+      // halve the columns a lane still holds; lane l ends with column l / 4.
+      auto fold8 = [&](float (&e)[8], auto op) -> float {
+        float v4[4], v2[2];
+        const bool b16 = lane & 16, b8 = lane & 8, b4 = lane & 4;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) v4[j] = op(b16 ? e[j + 4] : e[j], __shfl_xor_sync(kFullMask, b16 ? e[j] : e[j + 4], 16));
+#pragma unroll
+        for (int j = 0; j < 2; ++j) v2[j] = op(b8 ? v4[j + 2] : v4[j], __shfl_xor_sync(kFullMask, b8 ? v4[j] : v4[j + 2], 8));
+        float v1 = op(b4 ? v2[1] : v2[0], __shfl_xor_sync(kFullMask, b4 ? v2[0] : v2[1], 4));
+        v1 = op(v1, __shfl_xor_sync(kFullMask, v1, 2));
+        return op(v1, __shfl_xor_sync(kFullMask, v1, 1));
+      };
+      const int col = lane >> 2;
+      const int n_eights = n_pad / 8;
+      // ---- 1. maxima (both tiles hold the same beam rows: joined before the lanes are)
+      for (int hc = lw; hc < n_eights; hc += 4) {
+        const int c0 = hc * 8;
+        float z0[8], z1[8];
+        load8(0, c0, z0);
+        load8(1, c0, z1);
+#pragma unroll
+        for (int c = 0; c < 8; ++c) z0[c] = fmaxf(z0[c], z1[c]);
+        const float mx = fold8(z0, [](float x, float y) { return fmaxf(x, y); });
+        if (!(lane & 3)) fl_part[quarter * n_pad + c0 + col] = mx;
+      }
+      epilogue_barrier();
+      if (et < n_pad) {
+        const float M = fmaxf(fmaxf(fl_part[et], fl_part[n_pad + et]), fmaxf(fl_part[2 * n_pad + et], fl_part[3 * n_pad + et]));
+        const bool live = et < R && s_live[et];
+        if (live && M != neg_inf()) atomicMax(fa.gmax + et * kNarrowK + bid % k, float_to_ordered(M));
+        fl_max[et] = M == neg_inf() ? 0.f : M;         // reference of the exponentials; the row's maximum if it has one
+        if (et < R) st_ms[et].x = M;
+      }
+      epilogue_barrier();
+      if (et == 0) grid_arrive(cnt_floor);
+      // ---- 2. sums, while the other blocks find their way to the hand-over
+      for (int hc = lw; hc < n_eights; hc += 4) {
+        const int c0 = hc * 8;
+        float z0[8], z1[8];
+        load8(0, c0, z0);
+        load8(1, c0, z1);
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          const float M = fl_max[c0 + c];
+          z0[c] = __expf(z0[c] - M) + __expf(z1[c] - M);
+        }
+        const float sum = fold8(z0, [](float x, float y) { return x + y; });
+        if (!(lane & 3)) fl_part[quarter * n_pad + c0 + col] = sum;
+      }
+      // ---- 3. the floor: the smallest of the k group maxima, one warp per row
+      bool w_ok = true;
+      if (et == 0) w_ok = grid_wait(cnt_floor, d * G, abort_word, p.dev_status);
+      if (!epilogue_all(w_ok)) return -1;
+      {
+        uint32_t g[16];                                // n_pad <= 256: at most 16 rows per warp, all loads in flight at once
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const int r = ew + j * kEpiWarps;
+          g[j] = 0xFFFFFFFFu;
+          if (r < R && lane < k && s_live[r]) g[j] = __ldcg(fa.gmax + r * kNarrowK + lane);
+        }
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const int r = ew + j * kEpiWarps;
+          if (r >= n_pad) break;
+          const uint32_t fl = __reduce_min_sync(kFullMask, g[j]);
+          // rows that are not drafting, and padded columns, keep nothing; a group without any entry says nothing
+          if (lane == 0)
+            fl_floor[r] = fl == 0xFFFFFFFFu ? __int_as_float(0x7F800000) : (fl == 0u ? -3.4028234664e38f : ordered_to_float(fl));
+        }
+      }
+      if (et < R) {
+        const float S = (fl_part[et] + fl_part[n_pad + et]) + (fl_part[2 * n_pad + et] + fl_part[3 * n_pad + et]);
+        st_ms[et].y = st_ms[et].x == neg_inf() ? 0.f : S;
+      }
+      epilogue_barrier();
+      // ---- 4. what lies at or above the floor
+      for (int hc = lw; hc < n_eights; hc += 4) {
+        const int c0 = hc * 8;
+        float z0[8], z1[8], fl[8];
+        load8(0, c0, z0);
+        load8(1, c0, z1);
+        bool any = false;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          fl[c] = fl_floor[c0 + c];
+          any |= z0[c] >= fl[c];
+          any |= z1[c] >= fl[c];
+        }
+        if (any) {
+#pragma unroll
+          for (int c = 0; c < 8; ++c) {
+#pragma unroll
+            for (int t = 0; t < 2; ++t) {
+              const float z = t ? z1[c] : z0[c];
+              if (z >= fl[c]) {
+                const int at = atomicAdd(&s_queue_n, 1);
+                if (at < kFloorQueue) {
+                  fl_qkey[at] = make_key(z, (uint32_t)tok_t[t]);
+                  fl_qrow[at] = (short)(c0 + c);
+                }
+              }
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      epilogue_barrier();
+      const int n_q = s_queue_n;
+      if (n_q > kFloorQueue) {
+        // start over with the tile loop: its running state as at the start of the pass
+        for (int r = et; r < R; r += kEpiThreads) st_ms[r] = make_float2(neg_inf(), 0.f);
+        epilogue_barrier();
+        return 0;
+      }
+      if (ew < 4 && lane == 0) {                      // both accumulators may be overwritten
+        mbar_arrive(bar_tempty);
+        mbar_arrive(bar_tempty + 8u);
+      }
+      // ---- 5. the lists: entry e goes to place (number of better entries of its row)
+      for (int e = et; e < n_q; e += kEpiThreads) {
+        const unsigned long long key = fl_qkey[e];
+        const int r = fl_qrow[e];
+        int place = 0;
+        for (int o = 0; o < n_q; ++o) place += (fl_qrow[o] == r && fl_qkey[o] > key) ? 1 : 0;
+        if (place < k) st_key[r * k + place] = key;
+      }
+      epilogue_barrier();
+      return 1;
+    };
     for (int d = 1; d <= p.n; ++d) {
       ok = epilogue_all(mbar_wait(bar_pass, (uint32_t)(d - 1) & 1u, abort_flag, p.dev_status, false));
       if (!ok || s_pass_state[(d - 1) & 1] == 0) break;
@@ -487,8 +706,19 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
       }
       for (int i = et; i < R * k; i += kEpiThreads) st_key[i] = 0ull;
       epilogue_barrier();
+      // ---- many beam rows, both tiles fed together: nothing runs beside this epilogue, and a top-k
+      // per row and tile would cost it 40 us.  So the blocks first agree on a floor per row below which
+      // no logit can reach the row's k best anywhere (see floor_epilogue), then only pick up what
+      // lies above it: a fraction of an entry per row and block.
+      bool lists_done = false;
+      if (fa.floor) {
+        int state = floor_epilogue(d);
+        if (state < 0) { ok = false; break; }
+        lists_done = state == 1;
+        if (lists_done) tg += 2;
+      }
       // ---- the tiles of this block's vocabulary range
-      for (int t = 0; t < n_tiles && ok; ++t, ++tg) {
+      for (int t = 0; t < n_tiles && ok && !lists_done; ++t, ++tg) {
         const int acc = (int)(tg & 1u);
         const int rows = min(4, my_units - 4 * t) * kUnitRows;
         const int row0 = (unit0 + 4 * t) * kUnitRows;
@@ -532,7 +762,9 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
       // ---- publish this block's partials: hand-over 1
       for (int r = ew; r < R; r += kEpiWarps) {
         if (!s_live[r]) continue;
-        if (lane < k) fa.fkey[((size_t)r * k + lane) * kFusedMaxCtas + bid] = st_key[r * k + lane];
+        // a list is read up to its first empty entry: nothing behind that one needs to be written
+        if (lane < k && (lane == 0 || st_key[r * k + lane - 1] != 0ull))
+          fa.fkey[((size_t)r * k + lane) * kFusedMaxCtas + bid] = st_key[r * k + lane];
         if (lane == 0) fa.fms[(size_t)r * kFusedMaxCtas + bid] = st_ms[r];
       }
       epilogue_barrier();
@@ -574,7 +806,9 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
       };
       bool waited = false;
       int cur_b = -1;
-      for (int r_new = bid; r_new < R && ok; r_new += G) {
+      for (int own = 0; ok; ++own) {
+        const int r_new = owned_row(own);
+        if (r_new < 0) break;
         const int b = r_new / k, i = r_new - b * k;
         if (!s_live[b * k]) continue;                 // sequence not drafting in this pass
         if (d == p.n && i != 0) continue;             // after the last pass there is no draft step
@@ -584,6 +818,10 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
           ok = epilogue_all(w_ok);
           waited = true;
           if (!ok) break;
+          // every block has published, so none reads this pass's group maxima any more: clear those
+          // of this block's rows for the next pass (ordered before it by hand-over 2)
+          if (fa.floor && et < kNarrowK)
+            for (int j = 0, r; (r = owned_row(j)) >= 0; ++j) fa.gmax[r * kNarrowK + et] = 0u;
         }
         if (b != cur_b) {
           cur_b = b;
@@ -777,6 +1015,7 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
       if (fa.rerank_inside) *fa.io.out.status = *reinterpret_cast<volatile int*>(p.dev_status);
       atomicExch(cnt_partials, 0);
       atomicExch(cnt_hidden, 0);
+      atomicExch(cnt_floor, 0);
       atomicExch(abort_word, 0);
       atomicExch(exit_ticket, 0);
       __threadfence();
@@ -811,11 +1050,12 @@ bool fused_supported(const Params& p) {
   return p.dtype == DDD_DTYPE_BF16 && p.Hd % kBlockK == 0 && p.k <= kNarrowK && p.lm_ctas <= kFusedMaxCtas;
 }
 
-bool fused_pair_mode(const Params& p, int sm_count) {
+int fused_stage_units(const Params& p, int sm_count) {
   const int n_units = (p.Vl + kUnitRows - 1) / kUnitRows;
   const int ctas = sm_count < n_units ? sm_count : n_units;
   const int lo = n_units / ctas, hi = lo + (n_units % ctas ? 1 : 0);
-  return p.R >= 48 && lo >= 5 && hi <= 8 && 2 * ((p.R + 15) / 16 * 16) <= 512;
+  const bool pair = p.R >= 48 && lo >= 5 && hi <= 8 && 2 * ((p.R + 15) / 16 * 16) <= 512;
+  return pair ? hi : 4;
 }
 
 // Can the rerank run inside the draft kernel, in the epilogue's transpose buffer?  1: with the
@@ -854,7 +1094,10 @@ cudaError_t launch_draft_fused(const Params& p, const TcPlan& plan, const FusedA
   fa.stages = plan.stages;
   fa.ksub = plan.ksub;
   fa.cpg = plan.epi_chunks;
-  fa.pair = plan.atiles == 2 ? 1 : 0;
+  fa.pair = plan.a_units > 4 ? plan.a_units : 0;
+  // the floor epilogue: its scratch lies in the transpose buffer, and k groups of blocks need k blocks
+  fa.floor = (fa.pair && plan.ctas >= p.k &&
+              floor_scratch_bytes(plan.n_pad) <= plan.epi_chunks * kChunkCols * kTile * 4) ? 1 : 0;
   fa.rerank_inside = fused_rerank_mode(p, plan);
   fa.tmem_cols = plan.tmem_cols;
   cudaLaunchConfig_t cfg = {};

@@ -394,7 +394,7 @@ size_t tc_packed_bytes(int vocab, int hidden) {
   return units * kUnitRows * (size_t)hidden * 2;
 }
 
-int tc_plan_create(const Params& p, int sm_count, void* w_packed, TcPlan* plan, int extra_smem, int atiles) {
+int tc_plan_create(const Params& p, int sm_count, void* w_packed, TcPlan* plan, int extra_smem, int a_units) {
   if (p.dtype != DDD_DTYPE_BF16 || p.Hd % kBlockK != 0) return DDD_ERR_UNSUPPORTED;
   const int n_pad = (p.R + 15) / 16 * 16;
   if (n_pad > 256) return DDD_ERR_UNSUPPORTED;
@@ -412,7 +412,7 @@ int tc_plan_create(const Params& p, int sm_count, void* w_packed, TcPlan* plan, 
   // barriers, 8 KB of shared memory each; it gives way to the stage size when both do not fit.
   int ksub = 4, cpg = epi_group(p.R);
   auto fits = [&](int st, int ks, int cg) {
-    return smem_plan(st, ks, n_pad, p.R, p.k, cg, atiles).total + extra_smem + 1024 <= kSmemLimit;
+    return smem_plan(st, ks, n_pad, p.R, p.k, cg, a_units).total + extra_smem + 1024 <= kSmemLimit;
   };
   for (;;) {
     if (p.Hd % (kBlockK * ksub) == 0 && fits(2, ksub, cpg)) break;
@@ -425,6 +425,18 @@ int tc_plan_create(const Params& p, int sm_count, void* w_packed, TcPlan* plan, 
   for (int s = 8; s >= 2; --s) {
     if (fits(s, ksub, cpg)) { stages = s; break; }
   }
+  if (a_units > 4) {
+    // Both tiles of a block fed per stage (many beam rows): what bounds the pass there is the bytes
+    // a block has in flight, all stages but the one being multiplied.  So stages of one K-block,
+    // as many as fit beside the smallest epilogue buffer, then the largest buffer that still fits.
+    ksub = 1;
+    cpg = 1;
+    stages = 0;
+    for (int s = 8; s >= 2; --s) {
+      if (fits(s, 1, 1)) { stages = s; break; }
+    }
+    while (stages && cpg * 2 <= epi_group(p.R) && fits(stages, 1, cpg * 2)) cpg *= 2;
+  }
   if (stages == 0) return DDD_ERR_UNSUPPORTED;
   plan->ksub = ksub;
   plan->ctas = ctas;
@@ -432,8 +444,8 @@ int tc_plan_create(const Params& p, int sm_count, void* w_packed, TcPlan* plan, 
   plan->stages = stages;
   plan->tmem_cols = cols;
   plan->epi_chunks = cpg;
-  plan->smem = (size_t)smem_plan(stages, ksub, n_pad, p.R, p.k, cpg, atiles).total + extra_smem + 1024;
-  plan->atiles = atiles;
+  plan->smem = (size_t)smem_plan(stages, ksub, n_pad, p.R, p.k, cpg, a_units).total + extra_smem + 1024;
+  plan->a_units = a_units;
   plan->w_packed = static_cast<unsigned char*>(w_packed);
   {
     const size_t chunks = tc_packed_bytes(p.Vl, p.Hd) / kUnitBytes;

@@ -16,7 +16,7 @@ struct TcPlan {
   int ksub;               // 64-element K-blocks per stage
   int epi_chunks;         // 16-row accumulator chunks the epilogue unloads per barrier pair (1..4)
   int tmem_cols;          // allocated tensor-memory columns (power of two)
-  int atiles;             // W tiles per K-block of a stage the shared memory was sized for (1, or 2: see draft_fused.cu)
+  int a_units;            // 32-row units of W per K-block of a stage (4 = one tile; 5-8: both tiles of a block, see draft_fused.cu)
   size_t smem;            // dynamic shared memory per block
 };
 
@@ -25,7 +25,7 @@ size_t tc_packed_bytes(int vocab, int hidden);
 // Packs W into `w_packed` (device, 1024-byte aligned, tc_packed_bytes), encodes the tensor maps of
 // the hidden buffers and sizes the pipeline.  Synchronises the device.  Returns a DDD_* code.
 // extra_smem: bytes kept free behind the pipeline's own shared memory (for a kernel that does more than the pass).
-int tc_plan_create(const Params& p, int sm_count, void* w_packed, TcPlan* plan, int extra_smem = 0, int atiles = 1);
+int tc_plan_create(const Params& p, int sm_count, void* w_packed, TcPlan* plan, int extra_smem = 0, int a_units = 4);
 // pdl: launch with programmatic stream serialisation (see griddep_wait in ddd_common.cuh).
 cudaError_t launch_lm_head_tc(const Params& p, const TcPlan& plan, int d, int force_all, bool pdl, cudaStream_t st);
 

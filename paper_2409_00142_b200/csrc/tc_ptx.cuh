@@ -152,6 +152,18 @@ __device__ __forceinline__ void tc_load_16cols(uint32_t taddr, float (&v)[16]) {
 #pragma unroll
   for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
+__device__ __forceinline__ void tc_load_8cols(uint32_t taddr, float (&v)[8]) {
+  uint32_t r[8];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x8.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
+}
 __device__ __forceinline__ void epilogue_barrier() {
   asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
 }
@@ -202,11 +214,12 @@ struct SmemPlan {
 // rounded up to whole lanes of four (the wide-list layout).
 __host__ __device__ inline int key_stride(int k) { return k <= kNarrowK ? k : (k + 3) & ~3; }
 
-// atiles: 128-row tiles of W a stage holds per K-block (2 when a block feeds both of its tiles from one fetch of h)
-__host__ __device__ inline SmemPlan smem_plan(int stages, int ksub, int n_pad, int R, int k, int cpg, int atiles = 1) {
+// a_units: 32-row units of W a stage holds per K-block (4 = one tile; 5-8 when a block feeds both of its tiles
+// from one fetch of h)
+__host__ __device__ inline SmemPlan smem_plan(int stages, int ksub, int n_pad, int R, int k, int cpg, int a_units = 4) {
   SmemPlan s;
   int off = 0;
-  s.a = off; off += stages * ksub * atiles * kABytes;
+  s.a = off; off += stages * ksub * a_units * kUnitBytes;
   s.b = off; off += stages * ksub * n_pad * kBlockK * 2;
   s.zt = off; off += cpg * kChunkCols * kTile * 4;
   s.key = off; off += R * key_stride(k) * 8;

@@ -419,9 +419,13 @@ def test_fused_draft_with_both_tiles_of_a_block_sharing_a_stage(vocab):
         roots = S.make_roots(cfg, i)
         a = parity.run_gpu(eng_s, roots)
         b = parity.run_gpu(eng_f, roots)
-        for name in ("stop_depth", "n_out", "token", "parent", "depth", "position", "cum", "mask", "node_id",
-                     "tree_token", "tree_parent", "tree_cum"):
+        for name in ("stop_depth", "n_out", "token", "parent", "depth", "position", "mask", "node_id",
+                     "tree_token", "tree_parent"):
             np.testing.assert_array_equal(a[name], b[name], err_msg=name)
+        # the persistent kernel adds up a row's exp(z - max) in another order there (per quarter of a
+        # tile against the block's maximum): scores agree to rounding, choices are the same
+        for name in ("cum", "tree_cum"):
+            np.testing.assert_allclose(a[name], b[name], rtol=0, atol=2e-5, err_msg=name)
         parity.compare_with_oracle(cfg, weights_for(cfg), roots, b)
     eng_s.close()
     eng_f.close()
