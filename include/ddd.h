@@ -241,10 +241,17 @@ int ddd_lm_head_pass(ddd_handle *h, void *cuda_stream);
  * launched (kernels of passes after the stop exit at once); in graph mode the passes up to the
  * end of the group that holds pass `passes_needed` are launched.
  * ddd_lm_head_blocks: thread blocks of the LM-head kernel.
+ * ddd_fused_pass_kind: how a DDD_LAUNCH_FUSED handle runs a pass on this device: 0 = a block walks
+ * its 128-row tiles one after the other, 1 = both tiles of a block are fed from one fetch of the
+ * hidden rows (48 beam rows or more, five to eight 32-row units of the vocabulary per block),
+ * 2 = as 1, and the blocks agree on a lower bound of every row's k-th best logit before they
+ * pick their k best; handles of other launch modes give 0.  Results do not depend on it
+ * (scores agree to rounding): it exists for tests and benchmarks that want to know which path ran.
  * Pure host queries; negative on a NULL handle.
  */
 int ddd_launches_per_draft(const ddd_handle *h, int32_t passes_needed);
 int ddd_lm_head_blocks(const ddd_handle *h);
+int ddd_fused_pass_kind(const ddd_handle *h);
 
 /*
  * One LM-head pass that allocates nothing.  (The paper has no counterpart: this exists for

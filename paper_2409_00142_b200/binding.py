@@ -81,6 +81,8 @@ def load_library():
     lib.ddd_launches_per_draft.argtypes = [vp, ctypes.c_int32]
     lib.ddd_lm_head_blocks.restype = ctypes.c_int
     lib.ddd_lm_head_blocks.argtypes = [vp]
+    lib.ddd_fused_pass_kind.restype = ctypes.c_int
+    lib.ddd_fused_pass_kind.argtypes = [vp]
     lib.ddd_lm_head_topk_noalloc.restype = ctypes.c_int
     lib.ddd_lm_head_topk_noalloc.argtypes = [vp, vp, vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
                                              ctypes.c_int32, ctypes.c_int32, ctypes.c_float, vp, vp, vp, vp]
@@ -108,7 +110,7 @@ def load_library():
 def exported_symbols():
     """Names this binding expects the library to export (all of include/ddd.h)."""
     return ["ddd_workspace_bytes", "ddd_create", "ddd_draft", "ddd_draft_host", "ddd_draft_host_gated", "ddd_lm_head_pass",
-            "ddd_launches_per_draft", "ddd_lm_head_blocks", "ddd_lm_head_topk_noalloc", "ddd_verify_greedy",
+            "ddd_launches_per_draft", "ddd_lm_head_blocks", "ddd_fused_pass_kind", "ddd_lm_head_topk_noalloc", "ddd_verify_greedy",
             "ddd_shard_records_bytes", "ddd_shard_begin", "ddd_shard_lm_head", "ddd_shard_select",
             "ddd_destroy", "ddd_strerror"]
 
@@ -173,6 +175,10 @@ def ddd_launches_per_draft(handle: int, passes_needed: int) -> int:
 
 def ddd_lm_head_blocks(handle: int) -> int:
     return int(load_library().ddd_lm_head_blocks(handle))
+
+
+def ddd_fused_pass_kind(handle: int) -> int:
+    return int(load_library().ddd_fused_pass_kind(handle))
 
 
 def ddd_lm_head_topk_noalloc(W: int, bias: Optional[int], hidden_rows: int, dtype: int, rows: int, hidden: int,

@@ -736,6 +736,12 @@ int ddd_lm_head_blocks(const ddd_handle* h) {
   return h->p.lm_ctas;
 }
 
+int ddd_fused_pass_kind(const ddd_handle* h) {
+  if (!h) return DDD_ERR_INVALID_ARG;
+  if (h->cfg.launch_mode != DDD_LAUNCH_FUSED) return 0;
+  return fused_pass_kind(h->p, h->tc);
+}
+
 int ddd_destroy(ddd_handle* h) {
   if (!h) return DDD_ERR_INVALID_ARG;
   if (h->exec) cudaGraphExecDestroy(h->exec);

@@ -181,6 +181,11 @@ __device__ __forceinline__ void rerank_in_epilogue(const Params& p, const DraftI
 }
 
 // ---------------------------------------------------------------------------- kernel
+// MANY: the instantiation for many beam rows (fa.pair != 0: both tiles of a block per stage, the
+// floor epilogue, a sequence's rows on its own blocks).  The other one is kept as it was measured
+// before that mode existed: the serial section of a pass is a chain of single-warp steps, and
+// the same source with one more branch in it has come out 1.5 us per pass slower on the 7B shape.
+template <bool MANY>
 __global__ void __launch_bounds__(kTcThreads, 1)
 draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ CUtensorMap map_h0,
                    const __grid_constant__ CUtensorMap map_h1) {
@@ -191,6 +196,7 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
   // pair mode: a block's two tiles share every stage, so the hidden rows cross from L2 once per pass
   // instead of once per tile (what bounds a pass with many beam rows is L2 -> SM traffic)
   const int pair = fa.pair;
+  const bool use_floor = MANY && fa.floor;
   const SmemPlan sp = smem_plan(stages, ksub, n_pad, p.R, p.k, cpg, pair ? pair : 4);
   const TreeSmem ts = tree_smem(p.k);
   // The tree work's scratch lies over the epilogue's transpose buffer, which is idle between the
@@ -290,7 +296,7 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
     *p.n_active = p.B;
     *p.dev_status = DDD_OK;
   }
-  if (fa.floor && threadIdx.x < kNarrowK)      // group maxima of the rows this block looks after: none yet
+  if (use_floor && threadIdx.x < kNarrowK)      // group maxima of the rows this block looks after: none yet
     for (int r = bid; r < R; r += G) fa.gmax[r * kNarrowK + threadIdx.x] = 0u;
   tc_fence_before();
   __syncthreads();
@@ -488,7 +494,7 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
     // blocks a block's rows should belong to one sequence, whose lists it then merges once: sequence
     // b gets blocks b * bps .. b * bps + bps - 1, row i < bps goes to block i of them, the others
     // are dealt out from the far end (row 0's block also keeps the sequence's books).
-    const int bps = (R > G && p.B <= G) ? G / p.B : 0;
+    const int bps = (MANY && R > G && p.B <= G) ? G / p.B : 0;
     auto owned_row = [&](const int j) -> int {
       if (bps == 0) {
         const int r = bid + j * G;
@@ -711,11 +717,13 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
       // no logit can reach the row's k best anywhere (see floor_epilogue), then only pick up what
       // lies above it: a fraction of an entry per row and block.
       bool lists_done = false;
-      if (fa.floor) {
-        int state = floor_epilogue(d);
-        if (state < 0) { ok = false; break; }
-        lists_done = state == 1;
-        if (lists_done) tg += 2;
+      if constexpr (MANY) {
+        if (use_floor) {
+          int state = floor_epilogue(d);
+          if (state < 0) { ok = false; break; }
+          lists_done = state == 1;
+          if (lists_done) tg += 2;
+        }
       }
       // ---- the tiles of this block's vocabulary range
       for (int t = 0; t < n_tiles && ok && !lists_done; ++t, ++tg) {
@@ -763,7 +771,7 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
       for (int r = ew; r < R; r += kEpiWarps) {
         if (!s_live[r]) continue;
         // a list is read up to its first empty entry: nothing behind that one needs to be written
-        if (lane < k && (lane == 0 || st_key[r * k + lane - 1] != 0ull))
+        if (lane < k && (!MANY || lane == 0 || st_key[r * k + lane - 1] != 0ull))
           fa.fkey[((size_t)r * k + lane) * kFusedMaxCtas + bid] = st_key[r * k + lane];
         if (lane == 0) fa.fms[(size_t)r * kFusedMaxCtas + bid] = st_ms[r];
       }
@@ -806,9 +814,7 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
       };
       bool waited = false;
       int cur_b = -1;
-      for (int own = 0; ok; ++own) {
-        const int r_new = owned_row(own);
-        if (r_new < 0) break;
+      for (int own = 0, r_new = bid; (MANY ? (r_new = owned_row(own)) >= 0 : r_new < R) && ok; ++own, r_new += MANY ? 0 : G) {
         const int b = r_new / k, i = r_new - b * k;
         if (!s_live[b * k]) continue;                 // sequence not drafting in this pass
         if (d == p.n && i != 0) continue;             // after the last pass there is no draft step
@@ -820,7 +826,7 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
           if (!ok) break;
           // every block has published, so none reads this pass's group maxima any more: clear those
           // of this block's rows for the next pass (ordered before it by hand-over 2)
-          if (fa.floor && et < kNarrowK)
+          if (use_floor && et < kNarrowK)
             for (int j = 0, r; (r = owned_row(j)) >= 0; ++j) fa.gmax[r * kNarrowK + et] = 0u;
         }
         if (b != cur_b) {
@@ -1015,7 +1021,7 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
       if (fa.rerank_inside) *fa.io.out.status = *reinterpret_cast<volatile int*>(p.dev_status);
       atomicExch(cnt_partials, 0);
       atomicExch(cnt_hidden, 0);
-      atomicExch(cnt_floor, 0);
+      if (MANY) atomicExch(cnt_floor, 0);
       atomicExch(abort_word, 0);
       atomicExch(exit_ticket, 0);
       __threadfence();
@@ -1069,13 +1075,22 @@ int fused_rerank_mode(const Params& p, const TcPlan& plan) {
   return 0;
 }
 
+int fused_pass_kind(const Params& p, const TcPlan& plan) {
+  if (plan.a_units <= 4) return 0;
+  // the floor epilogue: its scratch lies in the transpose buffer, and k groups of blocks need k blocks
+  const bool floor = plan.ctas >= p.k && floor_scratch_bytes(plan.n_pad) <= plan.epi_chunks * kChunkCols * kTile * 4;
+  return floor ? 2 : 1;
+}
+
 int fused_prepare(const Params& p, const TcPlan& plan) {
   if (!fused_supported(p)) return DDD_ERR_UNSUPPORTED;
-  if (allow_max_dynamic_smem(draft_fused_kernel) != cudaSuccess) return DDD_ERR_CUDA;
+  if (allow_max_dynamic_smem(draft_fused_kernel<false>) != cudaSuccess) return DDD_ERR_CUDA;
+  if (allow_max_dynamic_smem(draft_fused_kernel<true>) != cudaSuccess) return DDD_ERR_CUDA;
   if (allow_max_dynamic_smem(rerank_kernel) != cudaSuccess) return DDD_ERR_CUDA;
   // every block must be resident at once: the blocks wait for one another
   int per_sm = 0, dev = 0, sms = 0;
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, draft_fused_kernel, kTcThreads, plan.smem) != cudaSuccess ||
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, plan.a_units > 4 ? draft_fused_kernel<true> : draft_fused_kernel<false>,
+                                                    kTcThreads, plan.smem) != cudaSuccess ||
       cudaGetDevice(&dev) != cudaSuccess ||
       cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
     return DDD_ERR_CUDA;
@@ -1095,9 +1110,7 @@ cudaError_t launch_draft_fused(const Params& p, const TcPlan& plan, const FusedA
   fa.ksub = plan.ksub;
   fa.cpg = plan.epi_chunks;
   fa.pair = plan.a_units > 4 ? plan.a_units : 0;
-  // the floor epilogue: its scratch lies in the transpose buffer, and k groups of blocks need k blocks
-  fa.floor = (fa.pair && plan.ctas >= p.k &&
-              floor_scratch_bytes(plan.n_pad) <= plan.epi_chunks * kChunkCols * kTile * 4) ? 1 : 0;
+  fa.floor = fused_pass_kind(p, plan) == 2 ? 1 : 0;
   fa.rerank_inside = fused_rerank_mode(p, plan);
   fa.tmem_cols = plan.tmem_cols;
   cudaLaunchConfig_t cfg = {};
@@ -1110,7 +1123,8 @@ cudaError_t launch_draft_fused(const Params& p, const TcPlan& plan, const FusedA
   attr[0].val.cooperative = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  cudaError_t e = cudaLaunchKernelEx(&cfg, draft_fused_kernel, p, fa, plan.map_h[0], plan.map_h[1]);
+  cudaError_t e = fa.pair ? cudaLaunchKernelEx(&cfg, draft_fused_kernel<true>, p, fa, plan.map_h[0], plan.map_h[1])
+                          : cudaLaunchKernelEx(&cfg, draft_fused_kernel<false>, p, fa, plan.map_h[0], plan.map_h[1]);
   if (e != cudaSuccess || fa.rerank_inside) return e;
   // rerank + mask: started early (programmatic dependent launch), waits on the device for the draft
   bool keys;

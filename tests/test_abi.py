@@ -64,7 +64,7 @@ def test_create_rejects_bad_arguments_without_a_device():
     assert lib.ddd_draft_host_gated(None, fake, fake, fake, None, None, None, None) == -1
     assert lib.ddd_lm_head_pass(None, None) == -1
     assert lib.ddd_destroy(None) == -1
-    assert lib.ddd_launches_per_draft(None, 1) < 0 and lib.ddd_lm_head_blocks(None) < 0
+    assert lib.ddd_launches_per_draft(None, 1) < 0 and lib.ddd_lm_head_blocks(None) < 0 and lib.ddd_fused_pass_kind(None) < 0
 
 
 def test_verify_greedy_rejects_bad_arguments_without_a_device():

@@ -415,6 +415,8 @@ def test_fused_draft_with_both_tiles_of_a_block_sharing_a_stage(vocab):
     cfg = S.scaled_down(S.CONFIGS["llama2_70b_b16"], 256, vocab, batch=5, threshold=-3.0, max_depth=4)
     eng_s = engine_for(cfg, TC, P.DDD_LAUNCH_STREAM)
     eng_f = engine_for(cfg, TC, P.DDD_LAUNCH_FUSED)
+    if torch.cuda.get_device_properties(0).multi_processor_count == 148:
+        assert P.ddd_fused_pass_kind(eng_f.handle) >= 1
     for i in range(3):
         roots = S.make_roots(cfg, i)
         a = parity.run_gpu(eng_s, roots)
@@ -429,6 +431,68 @@ def test_fused_draft_with_both_tiles_of_a_block_sharing_a_stage(vocab):
         parity.compare_with_oracle(cfg, weights_for(cfg), roots, b)
     eng_s.close()
     eng_f.close()
+
+
+def floor_cases():
+    # Shapes where the persistent kernel's blocks agree on a floor per row before they pick
+    # their k best (48 beam rows or more, five to eight 32-row units per block on a 148-SM device).
+    base = S.CONFIGS["llama2_70b_b16"]
+    return {
+        # more rows than blocks: a sequence's ten rows on its own nine blocks
+        "160_rows": S.scaled_down(base, 256, 32000, batch=16, threshold=-2.5, max_depth=4),
+        # eight rows per sequence on seven blocks, ragged last unit
+        "k8_b20": S.scaled_down(base, 256, 31000 + 8, batch=20, k=8, total_tokens=40, threshold=-2.5, max_depth=4),
+        # planted columns take the checked form of the logit
+        "plant": S.scaled_down(base, 256, 30000 + 8, batch=6, threshold=-3.0, max_depth=4, plant_frac=0.3,
+                               plant_delta=8.0),
+        # a bias that puts every winner into the first blocks: their queues fill, the others' stay empty
+        "zipf_bias": S.scaled_down(base, 256, 26000, batch=5, threshold=-3.0, max_depth=3, bias_kind="zipf"),
+        "k16": S.scaled_down(base, 256, 28000, batch=4, k=16, total_tokens=64, threshold=-3.0, max_depth=3),
+        "k32": S.scaled_down(base, 256, 36000, batch=2, k=32, total_tokens=96, threshold=NEG, max_depth=3),
+    }
+
+
+@pytest.mark.parametrize("case", list(floor_cases()))
+def test_fused_draft_with_a_floor_per_row(case):
+    cfg = floor_cases()[case]
+    eng_s = engine_for(cfg, TC, P.DDD_LAUNCH_STREAM)
+    eng_f = engine_for(cfg, TC, P.DDD_LAUNCH_FUSED)
+    if torch.cuda.get_device_properties(0).multi_processor_count == 148:
+        assert P.ddd_fused_pass_kind(eng_f.handle) == 2
+    assert P.ddd_fused_pass_kind(eng_s.handle) == 0
+    for i in range(2):
+        roots = S.make_roots(cfg, i)
+        a = parity.run_gpu(eng_s, roots)
+        b = parity.run_gpu(eng_f, roots)
+        parity.compare_with_oracle(cfg, weights_for(cfg), roots, b)
+        for name in ("stop_depth", "n_out", "token", "parent", "depth", "position", "mask", "tree_token", "tree_parent"):
+            np.testing.assert_array_equal(a[name], b[name], err_msg=name)
+        np.testing.assert_allclose(a["cum"], b["cum"], rtol=0, atol=2e-5)
+    eng_s.close()
+    eng_f.close()
+
+
+def test_fused_draft_where_the_floor_says_nothing():
+    # W = 0: all logits of a row are equal, every one of them lies on the floor, the queue of
+    # each block runs over and the pass is done by the tile loop instead; the result is the
+    # closed form (ties to the lowest token and candidate index)
+    cfg = S.scaled_down(S.CONFIGS["llama2_70b_b16"], 256, 32000, batch=6, threshold=NEG, max_depth=3)
+    w = dict(weights_for(cfg))
+    w["W"] = torch.zeros_like(w["W"])
+    eng = P.DraftEngine(cfg, w, lm_head_kernel=TC, launch_mode=P.DDD_LAUNCH_FUSED)
+    if torch.cuda.get_device_properties(0).multi_processor_count == 148:
+        assert P.ddd_fused_pass_kind(eng.handle) == 2
+    roots = S.make_roots(cfg, 0)
+    g = parity.run_gpu(eng, roots)
+    k, V = cfg.k, cfg.vocab
+    for q in range(cfg.batch):
+        assert int(g["stop_depth"][q]) == cfg.max_depth
+        for d in range(1, cfg.max_depth + 1):
+            assert abs(g["H_trace"][q, d - 1] - (math.log(k) - d * math.log(V))) < 1e-3
+            assert g["beam_sel"][q, d - 1].tolist() == list(range(k))
+        assert g["tree_token"][q, 1:k + 1].tolist() == list(range(k))
+    parity.compare_with_oracle(cfg, w, roots, g, strict=True)
+    eng.close()
 
 
 @pytest.mark.parametrize("k,n,launches", [(10, 12, 1), (10, 16, 1), (16, 16, 2)], ids=["keys_in_smem", "keys_from_global", "kernel"])
