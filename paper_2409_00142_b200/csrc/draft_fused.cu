@@ -918,34 +918,49 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
         }
         // ---- draft step of new beam row i: h = round(u / sqrt(mean(u^2) + eps)), u = h_parent + E[token]
         {
-          const int tok = sel_tok[i];
-          const uint4* hp = reinterpret_cast<const uint4*>(p.hbuf[par_in]) + (size_t)(b * k + sel_flat[i] / k) * cpr;
+          // MANY: a block with a second row of the same sequence takes both at once, half of the
+          // threads each: the step is a chain of round trips that 256 threads get through as fast as 512
+          int i2 = -1;
+          if constexpr (MANY) {
+            const int r2 = owned_row(own + 1);
+            if (r2 >= 0 && r2 / k == b && row_by_block && 2 * (cpr / 32) <= 64) {
+              i2 = r2 - b * k;
+              ++own;
+            }
+          }
+          const int tpr = (MANY && i2 >= 0) ? kEpiThreads / 2 : kEpiThreads;       // threads per row
+          const int second = (MANY && et >= tpr) ? 1 : 0;
+          const int lt = MANY ? et - second * tpr : et;                            // this thread's index among its row's
+          const int my_i = second ? i2 : i;
+          const int tok = sel_tok[my_i];
+          const uint4* hp = reinterpret_cast<const uint4*>(p.hbuf[par_in]) + (size_t)(b * k + sel_flat[my_i] / k) * cpr;
           const uint4* er = reinterpret_cast<const uint4*>(p.E) + (size_t)(tok >= 0 && tok < p.V ? tok : 0) * cpr;
-          uint4* out = reinterpret_cast<uint4*>(p.hbuf[par_out]) + (size_t)(b * k + i) * cpr;
+          uint4* out = reinterpret_cast<uint4*>(p.hbuf[par_out]) + (size_t)(b * k + my_i) * cpr;
           if (row_by_block) {
-            // chunk q belongs to thread q mod 512; a warp's 32 chunks form one partial sum (slot q / 32)
+            // chunk q belongs to thread q mod 512 (256); a warp's 32 chunks form one partial sum (slot q / 32)
             const int slots = cpr / 32;
+            double* const red_row = MANY ? red_s + second * slots : red_s;
             uint4 hv0 = make_uint4(0, 0, 0, 0), ev0 = hv0;
-            if (et - lane < cpr) { hv0 = hp[et]; ev0 = er[et]; }     // in flight while the books are kept
+            if (lt - lane < cpr) { hv0 = hp[lt]; ev0 = er[lt]; }     // in flight while the books are kept
             if (i == 0) keep_books(b);
-            for (int q = et; q - lane < cpr; q += kEpiThreads) {
+            for (int q = lt; q - lane < cpr; q += tpr) {
               uint4 hv = hv0, ev = ev0;
-              if (q != et) { hv = hp[q]; ev = er[q]; }
+              if (q != lt) { hv = hp[q]; ev = er[q]; }
               double u[8];
               Chunk<__nv_bfloat16>::sum(hv, ev, u);
               double ss = 0.0;
 #pragma unroll
               for (int e = 0; e < 8; ++e) ss = fma(u[e], u[e], ss);
               ss = warp_sum_f64(ss);
-              if (lane == 0) red_s[q / 32] = ss;
+              if (lane == 0) red_row[q / 32] = ss;
             }
             epilogue_barrier();
             double ss = 0.0;
-            for (int j = 0; j < slots; ++j) ss += red_s[j];
+            for (int j = 0; j < slots; ++j) ss += red_row[j];
             const double inv = 1.0 / sqrt(ss / (double)p.Hd + (double)p.eps);
-            for (int q = et; q < cpr; q += kEpiThreads) {
+            for (int q = lt; q < cpr; q += tpr) {
               uint4 hv = hv0, ev = ev0;
-              if (q != et) { hv = hp[q]; ev = er[q]; }
+              if (q != lt) { hv = hp[q]; ev = er[q]; }
               double u[8];
               Chunk<__nv_bfloat16>::sum(hv, ev, u);
 #pragma unroll
