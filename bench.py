@@ -35,8 +35,10 @@ NEG = -1e30
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes (read + write) of one launch of the persistent draft kernel (a full-depth draft) from the
 # ncu capture summarised under profiles/, valid only while the kernel source is the one that was profiled.
-NCU_TRAFFIC = {"llama2_7b": {"bytes": 2941.0e6, "source_sha256_16": "3aa5f989121ea0e8",
-                             "profile": "profiles/draft_fused_llama2_7b.md"}}
+NCU_TRAFFIC = {"llama2_7b": {"bytes": 2943.0e6, "source_sha256_16": "4eaa333136df7e35",
+                             "profile": "profiles/draft_fused_llama2_7b.md"},
+               "llama2_70b_b16": {"bytes": 5129.7e6, "source_sha256_16": "4eaa333136df7e35",
+                                  "profile": "profiles/draft_fused_llama2_70b_b16.md"}}
 BEAM_WIDTHS = (5, 10, 20, 50, 75, 100)      # fixed-depth-6 sweep: the widths of the paper's appendix table
 OTHER_WORKLOADS = ("vicuna_13b", "llama2_70b_b16", "llama3_8b_128k")
 CLOCK_QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
@@ -77,7 +79,7 @@ def ncu_traffic(workload: str):
         return None
     digest = hashlib.sha256()
     try:
-        for name in ("draft_fused.cu", "tc_ptx.cuh", "ddd_common.cuh"):      # the kernel and what it inlines
+        for name in ("draft_fused.cu", "tc_ptx.cuh", "ddd_common.cuh", "tree_device.cuh"):      # the kernel and what it inlines
             with open(os.path.join(ROOT, "paper_2409_00142_b200", "csrc", name), "rb") as f:
                 digest.update(f.read())
     except OSError:
@@ -536,6 +538,7 @@ def main():
                 o_step = 1e3 * ofms / len(oroots[:8]) / oc.max_depth
                 others[name] = {
                     "threshold": oc.threshold, "beam_rows": oc.batch * oc.k, "mean_stop_depth": odepth,
+                    "fused_pass_kind": P.ddd_fused_pass_kind(of.handle),
                     "drafts_per_sec": n_o * oc.batch / (oms / 1e3),
                     "lm_head_us_back_to_back": o_period, "lm_head_us_isolated": o_iso,
                     "lm_head_gbs": o_bytes / (o_period * 1e-6) / 1e9, "lm_head_frac": o_bytes / (o_period * 1e-6) / 1e9 / peak,

@@ -33,9 +33,10 @@
  *     has been synchronised.  Problems found on the device (a bounded wait that ran out)
  *     are reported through ddd_output.status, never as a fault.
  *   - One draft in flight per handle; a handle is not thread-safe.
- *   - The library reads one environment variable, DDD_DEBUG: if it is set (to anything), a
- *     failed CUDA call is described on stderr before DDD_ERR_CUDA is returned.  Nothing else
- *     about its behaviour depends on the environment.
+ *   - The library reads two environment variables.  DDD_DEBUG: if it is set (to anything), a
+ *     failed CUDA call is described on stderr before DDD_ERR_CUDA is returned.
+ *     DDD_FUSED_COOPERATIVE: see DDD_LAUNCH_FUSED.  Nothing else about its behaviour depends
+ *     on the environment.
  */
 #ifndef DDD_H_
 #define DDD_H_
@@ -72,12 +73,19 @@ enum { DDD_LM_HEAD_AUTO = 0, DDD_LM_HEAD_SIMT = 1, DDD_LM_HEAD_TCGEN05 = 2 };
  * on, so that a draft that stops early launches little that has nothing to do.  PLAIN launches
  * kernel by kernel in ordinary stream order, one after the other: the slowest, and the one
  * profilers can follow.  FUSED runs the whole draft as ONE persistent kernel of one thread block
- * per SM (a cooperative launch) that loops over the passes itself and hands over between them
+ * per SM that loops over the passes itself and hands over between them
  * through counters in global memory; the rerank and the mask run inside it too where the tree
  * fits the kernel's spare shared memory, else in one small kernel behind it:
  * the fastest, for bf16 handles on the tensor-core kernel with a beam of at most 32
- * (ddd_create returns DDD_ERR_UNSUPPORTED otherwise); nothing else should run on the device
- * meanwhile, since its blocks occupy every SM until the draft ends. */
+ * (ddd_create returns DDD_ERR_UNSUPPORTED otherwise, also where the device cannot hold all
+ * blocks at once).  Its blocks wait for one another, a whole SM each, so nothing else should
+ * run on the device meanwhile: a block kept off its SM by other work for longer than the
+ * waits' limit (2 s) ends the draft with DDD_ERR_TIMEOUT in ddd_output.status, never in a hang.
+ * The kernel is launched as a programmatic dependent of the kernel before it in the stream:
+ * blocks of the next draft set themselves up on the SMs that those of the running draft have
+ * left, and wait for its end before they touch anything the two share.  With
+ * DDD_FUSED_COOPERATIVE set in the environment it is a cooperative launch instead (all blocks
+ * resident at once or the launch fails; no overlap between drafts). */
 enum { DDD_LAUNCH_STREAM = 0, DDD_LAUNCH_GRAPH = 1, DDD_LAUNCH_PLAIN = 2, DDD_LAUNCH_FUSED = 3 };
 
 #define DDD_MAX_K 128         /* beam width limit (the paper's appendix table goes to 100) */

@@ -467,7 +467,8 @@ int ddd_draft(ddd_handle* h, const void* root_hidden, const int32_t* root_token,
     fa.fkey = reinterpret_cast<unsigned long long*>(h->ws + h->L.fused_key);
     fa.fms = reinterpret_cast<float2*>(h->ws + h->L.fused_ms);
     fa.gmax = reinterpret_cast<unsigned int*>(h->ws + h->L.fused_gmax);
-    if (launch_draft_fused(h->p, h->tc, fa, st) != cudaSuccess) {
+    static const bool cooperative = std::getenv("DDD_FUSED_COOPERATIVE") != nullptr;
+    if (launch_draft_fused(h->p, h->tc, fa, cooperative, st) != cudaSuccess) {
       note_cuda_error(__LINE__);
       return DDD_ERR_CUDA;
     }

@@ -273,6 +273,11 @@ draft_fused_kernel(const Params p, const FusedArgs fa, const __grid_constant__ C
                  ::"r"(smem_u32(tmem_ptr)), "r"((uint32_t)fa.tmem_cols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
+  // Nothing above touches what the kernel before this one in the stream may still be using, so a
+  // draft launched as a programmatic dependent sets itself up on every SM the previous draft has
+  // left (all but the one that still picks the beam and reranks) and waits here for its end.
+  griddep_launch_dependents();
+  griddep_wait();
   // ---- start of a draft: per-sequence state and the root rows (version 0 of the beam state)
   for (int b = bid; b < p.B; b += G) {
     const uint4* src = reinterpret_cast<const uint4*>(static_cast<const unsigned char*>(fa.root_hidden) +
@@ -1117,7 +1122,8 @@ int fused_prepare(const Params& p, const TcPlan& plan) {
   return DDD_OK;
 }
 
-cudaError_t launch_draft_fused(const Params& p, const TcPlan& plan, const FusedArgs& fa_in, cudaStream_t st) {
+cudaError_t launch_draft_fused(const Params& p, const TcPlan& plan, const FusedArgs& fa_in, bool cooperative,
+                               cudaStream_t st) {
   FusedArgs fa = fa_in;
   fa.w_packed = plan.w_packed;
   fa.n_pad = plan.n_pad;
@@ -1133,9 +1139,21 @@ cudaError_t launch_draft_fused(const Params& p, const TcPlan& plan, const FusedA
   cfg.blockDim = dim3(kTcThreads, 1, 1);
   cfg.dynamicSmemBytes = plan.smem;
   cfg.stream = st;
+  // The blocks wait for one another, so all of them must be resident at once.  fused_prepare has
+  // checked that the device has room for them, and a draft kernel holds a whole SM per block, so on
+  // a device that runs nothing else they are: blocks of the next draft move in as those of this one
+  // leave (programmatic dependent launch: 3 us per draft at stop depth 2) and wait for its end.
+  // Under other long-running work a block may come late; the others' waits are bounded and end
+  // in DDD_ERR_TIMEOUT.  A cooperative launch (all blocks at once, or not at all) excludes that and
+  // the overlap with it.
   cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeCooperative;       // all blocks resident at once, or the launch fails
-  attr[0].val.cooperative = 1;
+  if (cooperative) {
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+  } else {
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+  }
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   cudaError_t e = fa.pair ? cudaLaunchKernelEx(&cfg, draft_fused_kernel<true>, p, fa, plan.map_h[0], plan.map_h[1])

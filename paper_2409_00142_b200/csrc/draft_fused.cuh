@@ -42,6 +42,7 @@ int fused_rerank_mode(const Params& p, const TcPlan& plan);
 // 0: tile after tile, 1: both tiles of a block per stage, 2: as 1 with a floor per row agreed between the blocks.
 int fused_pass_kind(const Params& p, const TcPlan& plan);
 // Enqueues the draft kernel and, where the rerank does not fit inside it, the rerank kernel behind it.
-cudaError_t launch_draft_fused(const Params& p, const TcPlan& plan, const FusedArgs& fa, cudaStream_t st);
+// cooperative: launch with the cooperative attribute instead of as a programmatic dependent of the kernel before it.
+cudaError_t launch_draft_fused(const Params& p, const TcPlan& plan, const FusedArgs& fa, bool cooperative, cudaStream_t st);
 
 }  // namespace ddd
