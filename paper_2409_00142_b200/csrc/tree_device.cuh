@@ -196,26 +196,35 @@ __device__ void rerank_mask_impl(const Params& p, const DraftIO& io, const int b
 
   int n_selected;
   if (KEYS_IN_SMEM && N <= THREADS) {
-    // ---- few nodes (a draft that stopped early: the common case): one node per thread, ranked by
-    // counting the nodes that come before it in (score descending, node id ascending) order;
-    // five barriers instead of the thirty-odd of the radix path
-    const uint32_t mine = tid < N ? key_s[tid] : 0u;
+    // ---- few nodes (a draft that stopped early: the common case): a node is ranked by counting the
+    // nodes that come before it in (score descending, node id ascending) order, the count shared
+    // between as many threads as the block has per node (a power of two inside one warp); the
+    // kept nodes' rows follow from a ballot per warp.  Four barriers against the thirty-odd of the
+    // radix path, and no loop over the nodes longer than N / (threads per node).
+    int tpn = 1;
+    while (tpn < 32 && 2 * tpn * N <= THREADS) tpn *= 2;
+    const int node = tid / tpn, part = tid - node * tpn;
+    const uint32_t mine = node < N ? key_s[node] : 0u;
     int rank = 0;
-    for (int j = 0; j < N; ++j) {
+    for (int j = part; j < N; j += tpn) {
       const uint32_t q = key_s[j];
-      rank += (q > mine || (q == mine && j < tid)) ? 1 : 0;
+      rank += (q > mine || (q == mine && j < node)) ? 1 : 0;
     }
-    const bool sel = tid < N && rank < m_eff;
-    if (tid < N) slot_of[tid + 1] = sel ? 1 : 0;
+    for (int o = tpn >> 1; o > 0; o >>= 1) rank += __shfl_xor_sync(kFullMask, rank, o);
+    if (node < N && part == 0) slot_of[node + 1] = rank < m_eff ? 1 : 0;
     Sync::sync();
-    int before = 0, total = 0;
-    for (int j = 0; j < N; ++j) {
-      const int f = slot_of[j + 1];
-      total += f;
-      before += j < tid ? f : 0;
+    // thread t now speaks for node t: rows are dealt out in node order
+    const bool sel = tid < N && slot_of[tid + 1] != 0;
+    const unsigned warp_sel = __ballot_sync(kFullMask, sel);
+    if ((tid & 31) == 0) warp_tot[tid >> 5] = __popc(warp_sel);
+    Sync::sync();
+    int before = __popc(warp_sel & ((1u << (tid & 31)) - 1u)), total = 0;
+    for (int w = 0; w * 32 < N; ++w) {
+      const int c = warp_tot[w];
+      total += c;
+      before += w < (tid >> 5) ? c : 0;
     }
     n_selected = total;
-    Sync::sync();
     if (tid < N) slot_of[tid + 1] = sel ? (short)(1 + before) : (short)-1;
     if (tid == 0) slot_of[0] = 0;
     Sync::sync();
