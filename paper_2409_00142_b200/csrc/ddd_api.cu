@@ -28,7 +28,7 @@ size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 struct Layout {
   size_t hbuf[2], part_key, part_ms, tree_token, tree_parent, tree_cum, beam_node, beam_tok, beam_cum,
       row_plant, active, stop_depth, root_pos, n_active, dev_status, lm_ticket, shard_counter, fused_sync,
-      fused_beam_cum, fused_beam_node, fused_row_plant, fused_key, fused_ms, fused_gmax, wide_records, w_packed;
+      fused_beam_cum, fused_beam_node, fused_row_plant, fused_key, fused_ms, fused_gmax, wide_records, wide_logits, wide_ldl, w_packed;
   // staging for ddd_draft_host: inputs, then the packed output block
   size_t in_hidden, in_token, in_pos, out_block;
   size_t o_n_out, o_stop, o_token, o_parent, o_depth, o_position, o_cum, o_mask, o_H, o_status, out_bytes;
@@ -95,6 +95,11 @@ Layout make_layout(const ddd_config* c) {
   L.fused_ms = take(may_fuse ? R * 160 * 8 : 0);
   L.fused_gmax = take(may_fuse ? R * 32 * 4 : 0);
   L.wide_records = take(k > 32 ? R * (k + 1) * 8 : 0);      // beams wider than 32: one folded partial per row
+  // ... and, on the tensor-core kernel with an unsliced vocabulary, the logits of a pass [R][ldl] fp32
+  const bool wide_dense = k > 32 && c->vocab_count == 0 && c->dtype == DDD_DTYPE_BF16 && c->hidden % 64 == 0 &&
+                          c->lm_head_kernel != DDD_LM_HEAD_SIMT;
+  L.wide_ldl = (size_t)(c->vocab + 31) / 32 * 32;
+  L.wide_logits = take(wide_dense ? R * L.wide_ldl * 4 : 0);
   // packed copy of W for the tensor-core kernel (kept 1024-byte aligned relative to the base)
   off = (off + 1023) / 1024 * 1024;
   const bool tc_possible = c->dtype == DDD_DTYPE_BF16 && c->hidden % 64 == 0 && c->lm_head_kernel != DDD_LM_HEAD_SIMT;
@@ -171,7 +176,9 @@ struct ddd_handle {
 namespace {
 
 cudaError_t launch_lm_head(const ddd_handle* h, int d, int force_all, bool pdl, cudaStream_t st) {
-  if (h->lm_kind == DDD_LM_HEAD_TCGEN05) return launch_lm_head_tc(h->p, h->tc, d, force_all, pdl, st);
+  if (h->lm_kind == DDD_LM_HEAD_TCGEN05)
+    return launch_lm_head_tc(h->p, h->tc, d, force_all, pdl, st,
+                             h->tc.dense ? reinterpret_cast<float*>(h->ws + h->L.wide_logits) : nullptr, h->L.wide_ldl);
   return launch_lm_head_simt(h->p, d, force_all, h->p.lm_ctas, st);
 }
 
@@ -200,7 +207,13 @@ cudaError_t enqueue_passes(const ddd_handle* h, const DraftIO& io, bool pdl, int
   }
   for (int d = first; d <= last && e == cudaSuccess; ++d) {
     e = launch_lm_head(h, d, 0, pdl && (d > first || after_kernel), st);
-    if (e == cudaSuccess && wide) e = launch_shard_reduce(h->p, d, 0, 1, &rec, nullptr, 1, 0, h->shard_counter, st);
+    if (e == cudaSuccess && wide) {
+      // the record of a row: from its logits where the LM-head kernel wrote them out, else folded from the blocks' lists
+      if (h->lm_kind == DDD_LM_HEAD_TCGEN05 && h->tc.dense)
+        e = launch_row_topk(h->p, d, reinterpret_cast<const float*>(h->ws + h->L.wide_logits), h->L.wide_ldl, rec, st);
+      else
+        e = launch_shard_reduce(h->p, d, 0, 1, &rec, nullptr, 1, 0, h->shard_counter, st);
+    }
     if (e == cudaSuccess) e = launch_select(wide ? q : h->p, io, d, pdl, cond, d == cond_pass, st);
   }
   return e;
@@ -418,7 +431,9 @@ int ddd_create(const ddd_config* cfg, const void* W, const void* E, const float*
     const bool fused = cfg->launch_mode == DDD_LAUNCH_FUSED;
     if (rc == DDD_OK && fused && cfg->k > 32) rc = DDD_ERR_UNSUPPORTED;
     const int a_units = fused && cfg->k <= 32 ? fused_stage_units(p, h->sm_count) : 4;
-    if (rc == DDD_OK) rc = tc_plan_create(p, h->sm_count, ws + L.w_packed, &h->tc, fused ? fused_extra_smem(cfg->k) : 0, a_units);
+    const bool dense = cfg->k > 32 && cfg->vocab_count == 0;      // wide beams: logits out, top-k per row behind (row_topk.cu)
+    if (rc == DDD_OK)
+      rc = tc_plan_create(p, h->sm_count, ws + L.w_packed, &h->tc, fused ? fused_extra_smem(cfg->k) : 0, a_units, dense);
     if (rc == DDD_OK) p.lm_ctas = h->tc.ctas;
     if (rc == DDD_OK && fused) rc = fused_prepare(p, h->tc);
   } else if (rc == DDD_OK && cfg->launch_mode == DDD_LAUNCH_FUSED) {
@@ -727,9 +742,9 @@ int ddd_launches_per_draft(const ddd_handle* h, int32_t passes_needed) {
     for (int j = nb - 1; j >= 0; --j)
       if (passes_needed <= h->bounds[j]) passes = h->bounds[j];   // the group that holds the last needed pass
   }
-  // init, then per launched pass LM head + select, and between them for beams wider than 32 the kernel
-  // that folds the per-block partials
-  return 1 + (h->p.k > 32 ? 3 : 2) * passes;
+  // init, then per launched pass LM head + select; for beams wider than 32 also the kernel between them
+  // that makes one record per row, and the draft step of the new rows as a kernel behind the select
+  return 1 + (h->p.k > 32 ? 4 : 2) * passes;
 }
 
 int ddd_lm_head_blocks(const ddd_handle* h) {

@@ -30,10 +30,18 @@ namespace {
 using namespace tc;
 
 // ---------------------------------------------------------------------------- kernel
+// DENSE: the instantiation for wide beams (33..128) on an unsliced vocabulary.  There the sorted
+// 128-key list per row and tile would cost the epilogue more than the stream (the pass took 77-117 us
+// at widths 50-100 against 42), and R * V logits are little beside V * Hd weights (5 % at 100 rows), so
+// this form writes the scaled logits to `logits` [R][ldl] (fp32, -inf for a planted column) and
+// leaves the top-k and the log-sum-exp of every row to row_topk_kernel (row_topk.cu); it keeps no
+// lists, so the ring gets the shared memory they took.
+template <bool DENSE>
 __global__ void __launch_bounds__(kTcThreads, 1)
 lm_head_tc_kernel(const Params p, const unsigned char* __restrict__ w_packed,
                   const __grid_constant__ CUtensorMap map_h, const int d, const int force_all,
-                  const int n_pad, const int stages, const int tmem_cols, const int ksub, const int cpg) {
+                  const int n_pad, const int stages, const int tmem_cols, const int ksub, const int cpg,
+                  float* __restrict__ logits, const size_t ldl) {
   // The kernel may have been launched while the select kernel of the previous pass is still
   // running (programmatic dependent launch).  Until griddep_wait() below it touches nothing
   // that kernel writes, except for one speculative look at the activity counter: if drafting
@@ -55,7 +63,7 @@ lm_head_tc_kernel(const Params p, const unsigned char* __restrict__ w_packed,
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(
       (reinterpret_cast<uintptr_t>(smem_dyn) + 1023u) & ~static_cast<uintptr_t>(1023u));
-  const SmemPlan sp = smem_plan(stages, ksub, n_pad, p.R, p.k, cpg);
+  const SmemPlan sp = smem_plan(stages, ksub, n_pad, p.R, DENSE ? 0 : p.k, cpg);
   float* zt = reinterpret_cast<float*>(smem + sp.zt);
   unsigned long long* st_key = reinterpret_cast<unsigned long long*>(smem + sp.key);
   float2* st_ms = reinterpret_cast<float2*>(smem + sp.ms);
@@ -176,7 +184,7 @@ lm_head_tc_kernel(const Params p, const unsigned char* __restrict__ w_packed,
     s_live[r] = row_live(p, r, d, force_all) ? 1 : 0;
     st_ms[r] = make_float2(neg_inf(), 0.f);
   }
-  const int kst = key_stride(p.k);
+  const int kst = DENSE ? 0 : key_stride(p.k);
   for (int i = threadIdx.x; i < p.R * kst; i += kTcThreads) st_key[i] = 0ull;
   tc_fence_before();
   __syncthreads();
@@ -272,6 +280,24 @@ lm_head_tc_kernel(const Params p, const unsigned char* __restrict__ w_packed,
       const int v = row0 + vrow;
       const bool v_ok = vrow < rows && v < p.Vl;
       const float bias = (v_ok && p.bias) ? p.bias[v] : 0.f;
+      if constexpr (DENSE) {
+        // chunk ch of 16 beam rows by warp (quarter, ch mod 4): a warp's store is 32 consecutive logits of one row
+        for (int ch = lw; ch < n_chunks; ch += kEpiWarps / 4) {
+          const int c0 = ch * kChunkCols;
+          float accv[16];
+          tc_load_16cols(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * n_pad + c0), accv);
+#pragma unroll
+          for (int c = 0; c < kChunkCols; ++c) {
+            const int r = c0 + c;
+            if (v_ok && r < p.R && s_live[r])
+              logits[(size_t)r * ldl + v] = s_plant[r] != v + p.v0 ? fmaf(accv[c], p.s, bias) : neg_inf();
+          }
+        }
+        tc_fence_before();
+        epilogue_barrier();
+        if (ew < 4 && lane == 0) mbar_arrive(bar_tempty + 8u * acc);
+        continue;
+      }
       for (int g0 = 0; g0 < n_chunks; g0 += cpg) {
         const int ch = g0 + lw;
         if (lw < cpg && ch < n_chunks) {
@@ -312,7 +338,7 @@ lm_head_tc_kernel(const Params p, const unsigned char* __restrict__ w_packed,
       }
     }
     // publish this block's partial results (each row by its owning warp)
-    if (ok) {
+    if (ok && !DENSE) {
       for (int r = ew; r < p.R; r += kEpiWarps) {
         if (!s_live[r]) continue;
         const size_t slot = (size_t)bid * p.R + r;
@@ -394,7 +420,7 @@ size_t tc_packed_bytes(int vocab, int hidden) {
   return units * kUnitRows * (size_t)hidden * 2;
 }
 
-int tc_plan_create(const Params& p, int sm_count, void* w_packed, TcPlan* plan, int extra_smem, int a_units) {
+int tc_plan_create(const Params& p, int sm_count, void* w_packed, TcPlan* plan, int extra_smem, int a_units, bool dense) {
   if (p.dtype != DDD_DTYPE_BF16 || p.Hd % kBlockK != 0) return DDD_ERR_UNSUPPORTED;
   const int n_pad = (p.R + 15) / 16 * 16;
   if (n_pad > 256) return DDD_ERR_UNSUPPORTED;
@@ -412,7 +438,7 @@ int tc_plan_create(const Params& p, int sm_count, void* w_packed, TcPlan* plan, 
   // barriers, 8 KB of shared memory each; it gives way to the stage size when both do not fit.
   int ksub = 4, cpg = epi_group(p.R);
   auto fits = [&](int st, int ks, int cg) {
-    return smem_plan(st, ks, n_pad, p.R, p.k, cg, a_units).total + extra_smem + 1024 <= kSmemLimit;
+    return smem_plan(st, ks, n_pad, p.R, dense ? 0 : p.k, cg, a_units).total + extra_smem + 1024 <= kSmemLimit;
   };
   for (;;) {
     if (p.Hd % (kBlockK * ksub) == 0 && fits(2, ksub, cpg)) break;
@@ -444,8 +470,9 @@ int tc_plan_create(const Params& p, int sm_count, void* w_packed, TcPlan* plan, 
   plan->stages = stages;
   plan->tmem_cols = cols;
   plan->epi_chunks = cpg;
-  plan->smem = (size_t)smem_plan(stages, ksub, n_pad, p.R, p.k, cpg, a_units).total + extra_smem + 1024;
+  plan->smem = (size_t)smem_plan(stages, ksub, n_pad, p.R, dense ? 0 : p.k, cpg, a_units).total + extra_smem + 1024;
   plan->a_units = a_units;
+  plan->dense = dense;
   plan->w_packed = static_cast<unsigned char*>(w_packed);
   {
     const size_t chunks = tc_packed_bytes(p.Vl, p.Hd) / kUnitBytes;
@@ -456,11 +483,13 @@ int tc_plan_create(const Params& p, int sm_count, void* w_packed, TcPlan* plan, 
   for (int i = 0; i < 2; ++i)
     if (!encode_hidden_3d(&plan->map_h[i], p.hbuf[i], (uint64_t)p.R, (uint64_t)p.Hd, (uint32_t)n_pad, (uint32_t)ksub))
       return DDD_ERR_CUDA;
-  if (allow_max_dynamic_smem(lm_head_tc_kernel) != cudaSuccess) return DDD_ERR_CUDA;
+  if (allow_max_dynamic_smem(lm_head_tc_kernel<false>) != cudaSuccess) return DDD_ERR_CUDA;
+  if (allow_max_dynamic_smem(lm_head_tc_kernel<true>) != cudaSuccess) return DDD_ERR_CUDA;
   return DDD_OK;
 }
 
-cudaError_t launch_lm_head_tc(const Params& p, const TcPlan& plan, int d, int force_all, bool pdl, cudaStream_t st) {
+cudaError_t launch_lm_head_tc(const Params& p, const TcPlan& plan, int d, int force_all, bool pdl, cudaStream_t st,
+                              float* logits, size_t ldl) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)plan.ctas, 1, 1);
   cfg.blockDim = dim3(kTcThreads, 1, 1);
@@ -471,8 +500,14 @@ cudaError_t launch_lm_head_tc(const Params& p, const TcPlan& plan, int d, int fo
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = pdl ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, lm_head_tc_kernel, p, (const unsigned char*)plan.w_packed, plan.map_h[(d - 1) & 1], d,
-                            force_all, plan.n_pad, plan.stages, plan.tmem_cols, plan.ksub, plan.epi_chunks);
+  if (plan.dense) {
+    if (!logits) return cudaErrorInvalidValue;
+    return cudaLaunchKernelEx(&cfg, lm_head_tc_kernel<true>, p, (const unsigned char*)plan.w_packed, plan.map_h[(d - 1) & 1],
+                              d, force_all, plan.n_pad, plan.stages, plan.tmem_cols, plan.ksub, plan.epi_chunks, logits, ldl);
+  }
+  return cudaLaunchKernelEx(&cfg, lm_head_tc_kernel<false>, p, (const unsigned char*)plan.w_packed, plan.map_h[(d - 1) & 1],
+                            d, force_all, plan.n_pad, plan.stages, plan.tmem_cols, plan.ksub, plan.epi_chunks,
+                            static_cast<float*>(nullptr), (size_t)0);
 }
 
 }  // namespace ddd

@@ -18,6 +18,7 @@ struct TcPlan {
   int tmem_cols;          // allocated tensor-memory columns (power of two)
   int a_units;            // 32-row units of W per K-block of a stage (4 = one tile; 5-8: both tiles of a block, see draft_fused.cu)
   size_t smem;            // dynamic shared memory per block
+  bool dense;             // sized for the form that writes the logits out (no per-row lists in shared memory)
 };
 
 // Bytes of the packed copy of W (vocab rounded up to whole 128-row tiles).
@@ -25,8 +26,15 @@ size_t tc_packed_bytes(int vocab, int hidden);
 // Packs W into `w_packed` (device, 1024-byte aligned, tc_packed_bytes), encodes the tensor maps of
 // the hidden buffers and sizes the pipeline.  Synchronises the device.  Returns a DDD_* code.
 // extra_smem: bytes kept free behind the pipeline's own shared memory (for a kernel that does more than the pass).
-int tc_plan_create(const Params& p, int sm_count, void* w_packed, TcPlan* plan, int extra_smem = 0, int a_units = 4);
+// dense: size the pipeline for the form that writes the logits to global memory (wide beams; see lm_head_tc.cu).
+int tc_plan_create(const Params& p, int sm_count, void* w_packed, TcPlan* plan, int extra_smem = 0, int a_units = 4,
+                   bool dense = false);
 // pdl: launch with programmatic stream serialisation (see griddep_wait in ddd_common.cuh).
-cudaError_t launch_lm_head_tc(const Params& p, const TcPlan& plan, int d, int force_all, bool pdl, cudaStream_t st);
+// logits / ldl: with a plan sized `dense`, where the scaled logits go ([R][ldl] fp32); else ignored.
+cudaError_t launch_lm_head_tc(const Params& p, const TcPlan& plan, int d, int force_all, bool pdl, cudaStream_t st,
+                              float* logits = nullptr, size_t ldl = 0);
+
+// row_topk.cu: the record of every live row of pass d ([R][k] keys, then [R] (max, sum exp)) from its logits [R][ldl].
+cudaError_t launch_row_topk(const Params& p, int d, const float* logits, size_t ldl, void* record, cudaStream_t st);
 
 }  // namespace ddd

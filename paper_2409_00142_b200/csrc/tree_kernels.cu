@@ -98,12 +98,14 @@ __device__ __forceinline__ unsigned long long merge_row_kway(const Params& p, in
 // threads; a warp's 32 chunks lie in one row (the caller checks that a row has a multiple of
 // 32 chunks).  Every warp sends its partial sum of squares to all blocks through distributed
 // shared memory, and each block adds a row's partials in the same fixed order.
-template <typename T>
+// kBatch: chunks a thread has in flight at once (two loads each).  A narrow beam has one or two
+// chunks per thread in all; with a wide one (100 rows: 12.5 chunks per thread) the step is bound by the
+// latency of those loads, so more of them go out together (measured at width 100: 25 us with 2, see below).
+template <typename T, int kBatch>
 __device__ void draft_step_cluster(const Params& p, int b, int d, const int* sel_flat, const int* sel_tok,
                                    double* row_part /* [k][slots] */, double* row_inv /* [k] */) {
   cg::cluster_group cluster = cg::this_cluster();
   constexpr int N = Chunk<T>::N;
-  constexpr int kBatch = 2;
   const int k = p.k, lane = threadIdx.x & 31;
   const int cpr = p.Hd / N;            // chunks per row
   const int slots = cpr / 32;          // warp-sized groups of chunks per row
@@ -221,12 +223,12 @@ __device__ void draft_step_warp(const Params& p, int b, int d, const int* sel_fl
 }
 
 // Called by every block of the cluster (the choice below is the same in all of them).
-template <typename T>
+template <typename T, int kBatch = 2>
 __device__ void draft_step(const Params& p, int b, int d, const int* sel_flat, const int* sel_tok, double* row_part,
                            double* row_inv) {
   const int cpr = p.Hd / Chunk<T>::N;
   if (cpr % 32 == 0 && cpr / 32 <= 64)
-    draft_step_cluster<T>(p, b, d, sel_flat, sel_tok, row_part, row_inv);
+    draft_step_cluster<T, kBatch>(p, b, d, sel_flat, sel_tok, row_part, row_inv);
   else if (cg::this_cluster().block_rank() == 0)
     draft_step_warp<T>(p, b, d, sel_flat, sel_tok);
 }
@@ -498,6 +500,69 @@ __global__ void __launch_bounds__(kSelThreads) select_gate_step_kernel(const Par
 // pairwise in four rounds.
 // Dynamic shared memory: candidate records [k*k], merge buffers [16][128], partial sums of squares
 // of the draft step [k][slots]; after a stop the same memory serves the rerank.
+// The best k of n candidate records (score bits << 32 | token, token < 0 = no candidate) of a
+// sequence, as a sorted wide list in warp 0's `acc` (keys: score, then lower candidate index).
+// Merging the P sorted rows of 128-key lists took 22 us at width 100; here every thread keeps
+// the best score among its share of the candidates, the smallest over the 16 warps of the
+// warp's j-th largest thread maximum (j = k / 16 rounded up) has k candidates at or above it,
+// those are gathered (a few hundred) and each is placed by counting the better ones.  Returns
+// false, with nothing changed, when more than kPickCap candidates reach the floor (equal
+// scores).  Called by the whole block; scratch: kWideWarps * kWideK 8-byte words.
+constexpr int kPickCap = 1024;
+__device__ bool pick_beam_by_floor(const unsigned long long* cand_rec, const int n, const int k,
+                                   unsigned long long* scratch, unsigned long long (&acc)[4]) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  unsigned long long* gathered = scratch;                            // [kPickCap]
+  unsigned long long* chosen = scratch + kPickCap;                   // [kWideK]
+  uint32_t* warp_floor = reinterpret_cast<uint32_t*>(chosen + kWideK);   // [kWideWarps]
+  int* count_s = reinterpret_cast<int*>(warp_floor + kWideWarps);
+  uint32_t best = 0u;
+  for (int f = tid; f < n; f += kWideThreads) {
+    const unsigned long long rec = cand_rec[f];
+    if ((int)(uint32_t)rec >= 0) best = max(best, float_to_ordered(__uint_as_float((uint32_t)(rec >> 32))));
+  }
+  {
+    const int j = (k + kWideWarps - 1) / kWideWarps;
+    uint32_t cur = best, jth = 0u;
+    for (int t = 0; t < j; ++t) {
+      jth = __reduce_max_sync(kFullMask, cur);
+      const unsigned who = __ballot_sync(kFullMask, cur == jth);
+      if (lane == __ffs(who) - 1) cur = 0u;
+    }
+    if (lane == 0) warp_floor[warp] = jth;
+  }
+  if (tid == 0) *count_s = 0;
+  if (tid < kWideK) chosen[tid] = 0ull;
+  __syncthreads();
+  uint32_t floor_o = warp_floor[0];
+  for (int w = 1; w < kWideWarps; ++w) floor_o = min(floor_o, warp_floor[w]);
+  // a warp with fewer than j candidates says nothing: then everything counts
+  for (int f = tid; f < n; f += kWideThreads) {
+    const unsigned long long rec = cand_rec[f];
+    if ((int)(uint32_t)rec < 0) continue;
+    const float score = __uint_as_float((uint32_t)(rec >> 32));
+    if (float_to_ordered(score) < floor_o) continue;
+    const int at = atomicAdd(count_s, 1);
+    if (at < kPickCap) gathered[at] = make_key(score, (uint32_t)f);
+  }
+  __syncthreads();
+  const int count = *count_s;
+  if (count > kPickCap) {
+    __syncthreads();
+    return false;
+  }
+  for (int e = tid; e < count; e += kWideThreads) {
+    const unsigned long long mine = gathered[e];
+    int place = 0;
+    for (int i = 0; i < count; ++i) place += gathered[i] > mine ? 1 : 0;
+    if (place < k) chosen[place] = mine;
+  }
+  __syncthreads();
+  if (warp == 0) wide_load(acc, chosen, k);
+  __syncthreads();
+  return true;
+}
+
 __global__ void __launch_bounds__(kWideThreads) select_gate_step_wide_kernel(const Params p, const DraftIO io,
                                                                              const int d, const int part_slots,
                                                                              const cudaGraphConditionalHandle cond,
@@ -606,23 +671,26 @@ __global__ void __launch_bounds__(kWideThreads) select_gate_step_wide_kernel(con
   if (!waited) asm volatile("barrier.cluster.wait.aligned;" ::: "memory");
   cluster.sync();
 
-  // ---- phase 2: the new beam = best k of the P sorted candidate rows (every block, same result)
+  // ---- phase 2: the new beam = best k of the P * k candidates (every block, same result)
   {
     unsigned long long acc[4] = {0ull, 0ull, 0ull, 0ull};
-    for (int row = warp; row < P; row += kWideWarps) {
-      unsigned long long t[4];
+    if (!pick_beam_by_floor(cand_rec, P * k, k, buf, acc)) {
+      // many equal scores: merge the P sorted candidate rows instead
+      for (int row = warp; row < P; row += kWideWarps) {
+        unsigned long long t[4];
 #pragma unroll
-      for (int s4 = 0; s4 < 4; ++s4) {
-        const int e = 4 * lane + s4;
-        t[s4] = 0ull;
-        if (e < k) {
-          const unsigned long long rec = cand_rec[row * k + e];
-          if ((int)(uint32_t)rec >= 0) t[s4] = make_key(__uint_as_float((uint32_t)(rec >> 32)), (uint32_t)(row * k + e));
+        for (int s4 = 0; s4 < 4; ++s4) {
+          const int e = 4 * lane + s4;
+          t[s4] = 0ull;
+          if (e < k) {
+            const unsigned long long rec = cand_rec[row * k + e];
+            if ((int)(uint32_t)rec >= 0) t[s4] = make_key(__uint_as_float((uint32_t)(rec >> 32)), (uint32_t)(row * k + e));
+          }
         }
+        wide_merge(acc, t);
       }
-      wide_merge(acc, t);
+      block_merge_lists(acc, buf);
     }
-    block_merge_lists(acc, buf);
     if (warp == 0) {
       float cum[4];
       int flat[4], tok[4];
@@ -678,10 +746,54 @@ __global__ void __launch_bounds__(kWideThreads) select_gate_step_wide_kernel(con
     }
     return;
   }
-  if (p.dtype == DDD_DTYPE_BF16)
-    draft_step<__nv_bfloat16>(p, b, d, sel_flat, sel_tok, row_part, row_inv);
-  else
-    draft_step<float>(p, b, d, sel_flat, sel_tok, row_part, row_inv);
+  // the draft step of the k new rows is a kernel of its own behind this one (draft_rows_kernel)
+  (void)row_part;
+  (void)row_inv;
+  (void)sel_tok;
+}
+
+// The synthetic draft step of a wide beam, one block per new beam row (Algorithm 1, "Run draft model on
+// beam"; here h = round(u / sqrt(mean(u^2) + eps)), u = h_parent + E[token], in fp64).  Inside the
+// select kernel the step had the eight SMs of a sequence's cluster: at width 100 its 100 rows of
+// fp64 conversions and sums took 25 us of the kernel's 43; as B * k blocks it has the whole device.
+// The row's token and parent come from the beam state the select kernel has just written.
+constexpr int kRowThreads = 256;
+template <typename T>
+__global__ void __launch_bounds__(kRowThreads) draft_rows_kernel(const Params p, const int d) {
+  griddep_wait();
+  griddep_launch_dependents();
+  constexpr int N = Chunk<T>::N;
+  const int k = p.k, r = blockIdx.x, b = r / k;
+  if (d >= p.n || p.active[b] == 0) return;          // no step after the last pass or after a stop
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int base = (d == 1) ? 1 : 1 + k + (d - 2) * k * k;
+  const int parent_slot = (p.beam_node[r] - base) / k;
+  const int tok = p.beam_tok[r];
+  const int cpr = p.Hd / N;
+  const uint4* hp = reinterpret_cast<const uint4*>(p.hbuf[(d - 1) & 1]) + (size_t)(b * k + parent_slot) * cpr;
+  const uint4* er = reinterpret_cast<const uint4*>(p.E) + (size_t)(tok >= 0 && tok < p.V ? tok : 0) * cpr;
+  uint4* out = reinterpret_cast<uint4*>(p.hbuf[d & 1]) + (size_t)r * cpr;
+  __shared__ double red[kRowThreads / 32];
+  double ss = 0.0;
+  for (int q = threadIdx.x; q < cpr; q += kRowThreads) {
+    double u[N];
+    Chunk<T>::sum(hp[q], er[q], u);
+#pragma unroll
+    for (int e = 0; e < N; ++e) ss = fma(u[e], u[e], ss);
+  }
+  ss = warp_sum_f64(ss);
+  if (lane == 0) red[warp] = ss;
+  __syncthreads();
+  double total = 0.0;
+  for (int w = 0; w < kRowThreads / 32; ++w) total += red[w];
+  const double inv = 1.0 / sqrt(total / (double)p.Hd + (double)p.eps);
+  for (int q = threadIdx.x; q < cpr; q += kRowThreads) {
+    double u[N];
+    Chunk<T>::sum(hp[q], er[q], u);
+#pragma unroll
+    for (int e = 0; e < N; ++e) u[e] *= inv;
+    out[q] = Chunk<T>::round(u);
+  }
 }
 
 // Can the partial lists of a block's rows live in its shared memory?  (Host and device agree
@@ -763,8 +875,18 @@ cudaError_t launch_select(const Params& p, const DraftIO& io, int d, bool pdl, c
   cfg.attrs = attr;
   cfg.numAttrs = pdl ? 2 : 1;
   const int lists = select_lists_in_smem(p) ? 1 : 0, sc = set_cond ? 1 : 0;
-  if (is_wide(p))
-    return cudaLaunchKernelEx(&cfg, select_gate_step_wide_kernel, p, io, d, wide_part_slots(p), cond, sc);
+  if (is_wide(p)) {
+    cudaError_t e = cudaLaunchKernelEx(&cfg, select_gate_step_wide_kernel, p, io, d, wide_part_slots(p), cond, sc);
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t rows = {};
+    rows.gridDim = dim3((unsigned)p.R, 1, 1);
+    rows.blockDim = dim3(kRowThreads, 1, 1);
+    rows.stream = st;
+    rows.attrs = attr + 1;                    // the programmatic-serialisation attribute alone
+    rows.numAttrs = pdl ? 1 : 0;
+    if (p.dtype == DDD_DTYPE_BF16) return cudaLaunchKernelEx(&rows, draft_rows_kernel<__nv_bfloat16>, p, d);
+    return cudaLaunchKernelEx(&rows, draft_rows_kernel<float>, p, d);
+  }
   if (wide) return cudaLaunchKernelEx(&cfg, select_gate_step_kernel<kSelThreadsWide>, p, io, d, lists, cond, sc);
   return cudaLaunchKernelEx(&cfg, select_gate_step_kernel<kSelThreadsNarrow>, p, io, d, lists, cond, sc);
 }
