@@ -618,7 +618,7 @@ __global__ void __launch_bounds__(kWideThreads) select_gate_step_wide_kernel(con
       const float cand = cum0 + lp;
       const int flat = pr * k + e;
       const unsigned long long rec = ((unsigned long long)__float_as_uint(cand) << 32) | (uint32_t)tok;
-      for (int rk = 0; rk < kSelCluster; ++rk) cluster.map_shared_rank(cand_rec, rk)[flat] = rec;
+      cluster.map_shared_rank(cand_rec, 0)[flat] = rec;          // block 0 of the cluster picks the beam
       const size_t node = (size_t)b * p.Nn + base + flat;
       p.tree_token[node] = tok;
       p.tree_parent[node] = parent_node;
@@ -670,8 +670,12 @@ __global__ void __launch_bounds__(kWideThreads) select_gate_step_wide_kernel(con
   }
   if (!waited) asm volatile("barrier.cluster.wait.aligned;" ::: "memory");
   cluster.sync();
+  // The candidates and the tree nodes of all rows are in place.  The draft step is a kernel of
+  // its own, so nothing is left for the other blocks: block 0 picks the beam, takes the stop
+  // decision, keeps the books and reranks at a stop.
+  if (crank != 0) return;
 
-  // ---- phase 2: the new beam = best k of the P * k candidates (every block, same result)
+  // ---- phase 2: the new beam = best k of the P * k candidates
   {
     unsigned long long acc[4] = {0ull, 0ull, 0ull, 0ull};
     if (!pick_beam_by_floor(cand_rec, P * k, k, buf, acc)) {
@@ -739,11 +743,9 @@ __global__ void __launch_bounds__(kWideThreads) select_gate_step_wide_kernel(con
   __syncthreads();
   if (set_cond && !s_stop && crank == 0 && threadIdx.x == 0) cudaGraphSetConditional(cond, 1);
   if (s_stop) {
-    cluster.sync();          // the nodes the other blocks appended in this pass are visible to block 0
-    if (crank == 0) {
-      if (p.Nn * 6 <= 160 * 1024) rerank_mask_block<kWideThreads, true>(p, io, b, d, s_last, smem_raw);
-      else rerank_mask_block<kWideThreads, false>(p, io, b, d, s_last, smem_raw);
-    }
+    // the nodes the other blocks appended in this pass were written before the cluster barrier above
+    if (p.Nn * 6 <= 160 * 1024) rerank_mask_block<kWideThreads, true>(p, io, b, d, s_last, smem_raw);
+    else rerank_mask_block<kWideThreads, false>(p, io, b, d, s_last, smem_raw);
     return;
   }
   // the draft step of the k new rows is a kernel of its own behind this one (draft_rows_kernel)
