@@ -54,6 +54,9 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama2_7b", choices=list(S.CONFIGS))
     ap.add_argument("--threshold", type=float, default=None, help="override the workload's threshold x")
+    ap.add_argument("--beam-width", type=int, default=None,
+                    help="override the workload's beam width k (beyond 32: not with --launch-mode fused)")
+    ap.add_argument("--max-depth", type=int, default=None, help="override the workload's maximum depth n")
     ap.add_argument("--drafts-per-step", type=int, default=1000,
                     help="distinct seeded roots drafted per step and rank (the 7B workload is stated on 1000 drafts)")
     ap.add_argument("--lm-head-reps", type=int, default=200)
@@ -331,6 +334,10 @@ def main():
     cfg = S.CONFIGS[args.workload]
     if args.threshold is not None:
         cfg = cfg.replace(threshold=args.threshold)
+    if args.beam_width is not None:
+        cfg = cfg.replace(k=args.beam_width)
+    if args.max_depth is not None:
+        cfg = cfg.replace(max_depth=args.max_depth)
     weights = S.make_weights(cfg)
     n_per_rank = args.drafts_per_step
     my_indices = S.shard_draft_indices(n_per_rank * world, rank, world)

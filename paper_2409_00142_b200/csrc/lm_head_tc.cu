@@ -17,7 +17,8 @@
 //              and transpose it through shared memory; then every warp folds one beam row's
 //              128 values into that row's online max / sum-exp and running top-k
 // Each thread block owns a contiguous range of vocab rows (a multiple of 32) and publishes
-// one partial (max, sum-exp, top-k list) per beam row; logits never reach global memory.
+// one partial (max, sum-exp, top-k list) per beam row; logits never reach global memory
+// (except for beams wider than 32, see DENSE below).
 // Every wait is bounded: when one runs out the block records DDD_ERR_TIMEOUT, drains what
 // it has in flight, frees its tensor memory and returns.
 #include "lm_head_tc.cuh"
