@@ -148,6 +148,9 @@ def wide_cases():
         "k75_two_sequences": base.replace(k=75, batch=2, max_depth=2, threshold=-9.0),   # 150 rows in a pass
         "k100": base.replace(k=100),
         "k128": base.replace(k=128, max_depth=2),                    # the limit
+        # fewer logits per row than the per-row top-k kernel has threads: every logit is a candidate
+        "k40_small_vocab": S.scaled_down(S.CONFIGS["llama2_7b"], 128, 1000, threshold=NEG, max_depth=3, total_tokens=100,
+                                         k=40),
         "k100_zipf": zipf.replace(k=100, batch=1),                   # winners cluster in the first vocab tiles
         # 28,737 tree nodes: more than the rerank keeps keys for in shared memory
         "k64_large_tree": S.scaled_down(S.CONFIGS["vicuna_13b"], 128, 2000, threshold=NEG, k=64, max_depth=8,
@@ -167,6 +170,30 @@ def test_wide_beams_match_oracle(case, kernel):
             roots = S.make_roots(cfg, i)
             g = parity.run_gpu(eng, roots)
             parity.compare_with_oracle(cfg, weights_for(cfg), roots, g)
+    eng.close()
+
+
+@pytest.mark.parametrize("k", [40, 100])
+def test_wide_beams_with_equal_logits_take_the_exact_slow_ways(k):
+    # W = 0 on the tensor-core path: every logit of a row is the same, so far more than 1024 of them lie
+    # on the floor the per-row top-k kernel derives (it falls back to a radix select over the row and takes
+    # the lowest tokens among the ties), and all k * k candidates of a pass tie as well (the select kernel
+    # falls back to merging the sorted candidate rows).  The closed form: tokens 0..k-1, candidates
+    # 0..k-1, H_d = ln k - d ln V.
+    cfg = S.scaled_down(S.CONFIGS["llama2_7b"], 256, 3000 + 24, threshold=NEG, max_depth=3, total_tokens=120, k=k)
+    w = dict(weights_for(cfg))
+    w["W"] = torch.zeros_like(w["W"])
+    eng = P.DraftEngine(cfg, w, lm_head_kernel=TC, launch_mode=P.DDD_LAUNCH_STREAM)
+    with torch.cuda.stream(torch.cuda.Stream()):
+        roots = S.make_roots(cfg, 0)
+        g = parity.run_gpu(eng, roots)
+    V = cfg.vocab
+    assert int(g["stop_depth"][0]) == cfg.max_depth
+    for d in range(1, cfg.max_depth + 1):
+        assert abs(g["H_trace"][0, d - 1] - (math.log(k) - d * math.log(V))) < 1e-3
+        assert g["beam_sel"][0, d - 1].tolist() == list(range(k))
+    assert g["tree_token"][0, 1:k + 1].tolist() == list(range(k))
+    parity.compare_with_oracle(cfg, w, roots, g, strict=True)
     eng.close()
 
 
