@@ -551,6 +551,11 @@ def main():
                     "lm_head_gbs": o_bytes / (o_period * 1e-6) / 1e9, "lm_head_frac": o_bytes / (o_period * 1e-6) / 1e9 / peak,
                     "us_per_expansion_step_full_depth": o_step,
                     "step_frac": o_bytes / (o_step * 1e-6) / 1e9 / peak}
+                if others[name]["fused_pass_kind"]:
+                    others[name]["lm_head_note"] = ("lm_head_* time the LM-head kernel of the kernel-by-kernel path; the "
+                                                    "persistent kernel's pass for many beam rows is organised differently "
+                                                    "(both tiles of a block per stage, a floor per row) and is timed by "
+                                                    "us_per_expansion_step_full_depth")
                 of.close()
                 oe.close()
                 del oe, of, ow, odw, oroots
