@@ -304,6 +304,44 @@ def test_random_shapes_match_oracle(index):
 
 
 # ----------------------------------------------------------------------------- launch modes
+def _random_many_rows_or_wide(index):
+    """Seeded random shapes for the two paths the ordinary random shapes do not reach: the many-rows
+    form of the persistent kernel (48 beam rows or more, 23,700-37,800 vocabulary rows on a 148-SM
+    device) for even indices, beams wider than 32 for odd ones."""
+    rng = np.random.default_rng([20240900142, index])
+    if index % 2 == 0:
+        k = int(rng.choice([8, 10, 12, 16, 24, 32]))
+        batch = int(rng.integers(max(2, -(-48 // k)), min(256 // k, max(3, 200 // k)) + 1))
+        vocab = int(rng.integers(23700, 37800) // 8 * 8 + int(rng.choice([0, 8, 16, 24])))
+        cfg = S.scaled_down(S.CONFIGS["llama2_70b_b16"], int(rng.choice([128, 256, 512])), vocab, batch=batch, k=k,
+                            total_tokens=int(rng.integers(10, 80)), threshold=float(rng.choice([NEG, -2.0, -3.0, -4.0])),
+                            max_depth=int(rng.integers(2, 6)), plant_frac=float(rng.choice([0.0, 0.0, 0.3])),
+                            plant_delta=8.0, bias_kind=str(rng.choice(["none", "none", "zipf"])),
+                            seed=int(rng.integers(0, 1000)))
+        return cfg, P.DDD_LAUNCH_FUSED
+    k = int(rng.choice([33, 40, 50, 64, 75, 100, 128]))
+    batch = int(rng.integers(1, max(1, 256 // k) + 1))
+    vocab = max(k + 64, int(rng.integers(600, 12000) // 8 * 8 + int(rng.choice([0, 8, 16]))))
+    cfg = S.scaled_down(S.CONFIGS["llama2_7b"], int(rng.choice([128, 256])), vocab, batch=batch, k=k,
+                        total_tokens=int(rng.integers(20, 300)), threshold=float(rng.choice([NEG, -6.0, -9.0])),
+                        max_depth=int(rng.integers(2, 5)), plant_frac=float(rng.choice([0.0, 0.0, 0.3])), plant_delta=8.0,
+                        bias_kind=str(rng.choice(["none", "none", "zipf"])), seed=int(rng.integers(0, 1000)))
+    return cfg, int(rng.choice([P.DDD_LAUNCH_STREAM, P.DDD_LAUNCH_GRAPH, P.DDD_LAUNCH_PLAIN]))
+
+
+@pytest.mark.parametrize("index", range(24))
+def test_random_many_rows_and_wide_shapes_match_oracle(index):
+    cfg, mode = _random_many_rows_or_wide(index)
+    w = S.make_weights(cfg)
+    eng = P.DraftEngine(cfg, w, lm_head_kernel=TC, launch_mode=mode)
+    with torch.cuda.stream(torch.cuda.Stream()):
+        for i in range(2):
+            roots = S.make_roots(cfg, 500 + i)
+            g = parity.run_gpu(eng, roots)
+            parity.compare_with_oracle(cfg, w, roots, g)
+    eng.close()
+
+
 def test_graph_mode_host_variant_and_determinism():
     cfg = small_cases()["7b"]
     roots = S.make_roots(cfg, 1)
