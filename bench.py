@@ -35,9 +35,9 @@ NEG = -1e30
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes (read + write) of one launch of the persistent draft kernel (a full-depth draft) from the
 # ncu capture summarised under profiles/, valid only while the kernel source is the one that was profiled.
-NCU_TRAFFIC = {"llama2_7b": {"bytes": 2941.7e6, "source_sha256_16": "7bf6dc11df120345",
+NCU_TRAFFIC = {"llama2_7b": {"bytes": 2942.2e6, "source_sha256_16": "f7456c78b72c5525",
                              "profile": "profiles/draft_fused_llama2_7b.md"},
-               "llama2_70b_b16": {"bytes": 5128.1e6, "source_sha256_16": "7bf6dc11df120345",
+               "llama2_70b_b16": {"bytes": 5131.3e6, "source_sha256_16": "f7456c78b72c5525",
                                   "profile": "profiles/draft_fused_llama2_70b_b16.md"}}
 BEAM_WIDTHS = (5, 10, 20, 50, 75, 100)      # fixed-depth-6 sweep: the widths of the paper's appendix table
 OTHER_WORKLOADS = ("vicuna_13b", "llama2_70b_b16", "llama3_8b_128k")

@@ -1,8 +1,9 @@
 // One persistent kernel per draft (launch mode DDD_LAUNCH_FUSED).
 //
 // Every pass of Algorithm 1 - LM head, log-softmax statistics, per-row top-k, merge, beam choice,
-// Eq. 1 and the gate, draft step - runs inside ONE cooperative launch of one thread block per SM.
-// The blocks never leave between passes, so the two kernel boundaries per pass of the other launch
+// Eq. 1 and the gate, draft step - runs inside ONE launch of one thread block per SM (all of them
+// resident at once: checked at ddd_create; launched as a programmatic dependent of the kernel
+// before it, see launch_draft_fused).  The blocks never leave between passes, so the two kernel boundaries per pass of the other launch
 // modes become two grid-wide hand-overs through counters in global memory, and a draft that
 // stops after d passes has launched nothing for the passes it does not run:
 //
@@ -24,6 +25,10 @@
 // twice, by pass parity: a block may still read the old beam while the book-keeper writes the new.
 // After the last pass the blocks that kept a sequence's books rerank its tree and write the rows
 // and the mask (in the epilogue's transpose buffer; a tree too large for it goes to rerank_kernel).
+//
+// With many beam rows (48 or more, two tiles per block) the instantiation <true> feeds both tiles
+// of a block from one fetch of the hidden rows and replaces the per-tile top-k of the epilogue by a
+// floor per row that the blocks agree on (floor_epilogue below).
 //
 // Every wait is bounded.  A wait that runs out records DDD_ERR_TIMEOUT, raises a grid-wide abort
 // word that ends every other wait, and each block drains its copies, frees its tensor memory and
