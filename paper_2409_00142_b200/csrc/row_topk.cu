@@ -155,15 +155,14 @@ __global__ void __launch_bounds__(kTopkThreads) row_topk_kernel(const Params p, 
   }
   if (tid == 0) s_count = 0;
   __syncthreads();
-  if (tid == 0) {
-    float M = neg_inf();
-    int n = 0;
-    for (int w = 0; w < kTopkThreads / 32; ++w) { M = fmaxf(M, red_m[w]); n += red_n[w]; }
-    float S = 0.f;
-    for (int w = 0; w < kTopkThreads / 32; ++w)
-      if (red_s[w] > 0.f) S += red_s[w] * __expf(red_m[w] - M);
-    rec_ms[r] = make_float2(M, S);
-    s_need = n < k ? n : k;
+  if (warp == 0) {                 // 32 warps' results, one per lane
+    const float M = ordered_to_float(__reduce_max_sync(kFullMask, float_to_ordered(red_m[lane])));
+    const float S = warp_sum(red_s[lane] > 0.f ? red_s[lane] * __expf(red_m[lane] - M) : 0.f);
+    const int n = __reduce_add_sync(kFullMask, red_n[lane]);
+    if (lane == 0) {
+      rec_ms[r] = make_float2(M, S);
+      s_need = n < k ? n : k;
+    }
   }
   __syncthreads();
   const int need = s_need;                 // entries the list will hold
