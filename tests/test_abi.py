@@ -42,6 +42,22 @@ def test_workspace_bytes_and_config_validation():
     assert big > P.ddd_workspace_bytes(good_config())
 
 
+def test_workspace_of_wide_beams_holds_the_logits_where_the_lm_head_writes_them_out():
+    # beams wider than 32 on the tensor-core kernel with an unsliced vocabulary: [B k][V rounded up to 32] fp32
+    shape = dict(batch=1, hidden=64, vocab=3000, max_depth=3, total_tokens=30, dtype=P.DDD_DTYPE_BF16)
+    logits = 100 * 3008 * 4
+    packed_w = 3008 * 64 * 2            # the tensor-core kernel's own copy of W (whole 32-row units): well under the logits here
+
+    def extra(**kw):                    # what the tensor-core path adds over the CUDA-core path
+        return (P.ddd_workspace_bytes(good_config(**shape, **kw)) -
+                P.ddd_workspace_bytes(good_config(**shape, **kw, lm_head_kernel=P.DDD_LM_HEAD_SIMT)))
+
+    assert extra(k=32) == packed_w
+    assert extra(k=100) == logits + packed_w
+    # a slice of a vocabulary-parallel head keeps per-block lists instead
+    assert extra(k=100, vocab_begin=0, vocab_count=1504) == 1504 * 64 * 2
+
+
 def test_create_rejects_bad_arguments_without_a_device():
     lib = P.load_library()
     cfg = good_config()
